@@ -1,0 +1,59 @@
+// Shared device helpers and internal types of libsnlp (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace snlp {
+
+constexpr int kMaxStreams = 8;
+
+// Per-layer stream-mixing coefficients derived on the host (in double) from the mHC maps of
+// App. C.2.  With x' = Ra x + Qa a and x_next = Rm x' + Qm m the block is affine in (x, a, m):
+//   x_next = A x + ca * a + cm * m,  A = Rm Ra (the HCN surrogate, Eq. 8), ca = Rm Qa, cm = Qm;
+// the attention branch reads pa . x (pa = Pa) and the MLP branch reads Pm . x' = pmra . x + kappa a
+// with pmra = Pm Ra and kappa = Pm . Qa.  For a residual model (n = 1) every entry is 1.
+struct HcCoef {
+  float A[kMaxStreams * kMaxStreams];
+  float ca[kMaxStreams];
+  float cm[kMaxStreams];
+  float pa[kMaxStreams];
+  float pmra[kMaxStreams];
+  float kappa;
+  float pad[3];
+};
+
+template <typename T>
+__device__ __forceinline__ float to_f(T v);
+template <>
+__device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T>
+__device__ __forceinline__ T from_f(float v);
+template <>
+__device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Deterministic block-wide sum (fixed order: lanes by butterfly, warps in index order).
+// `red` must hold at least 32 floats of shared memory.  All threads get the result.
+__device__ __forceinline__ float block_sum(float v, float *red) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  v = warp_sum(v);
+  __syncthreads();
+  if (lane == 0) red[w] = v;
+  __syncthreads();
+  float s = 0.f;
+  for (int i = 0; i < nw; ++i) s += red[i];
+  return s;
+}
+
+}  // namespace snlp

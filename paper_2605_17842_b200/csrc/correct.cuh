@@ -1,0 +1,145 @@
+// Fused structured correction along the layer axis (Alg. 2 lines 8-10, Eq. 5), one coalesced pass
+// over the trace: per (row, 4-column) thread a serial loop over the layers of the range; no
+// dependency between threads along L.  Also produces the residual norms of Eq. (2) and, for mHC
+// models, the two pre-mapped branch inputs of every layer for the next sweep.
+#pragma once
+#include "common.cuh"
+
+namespace snlp {
+
+struct CorrParams {
+  float *trace;      // [L+1][M][n][d], updated in place for states l0+1 .. l0+nl
+  const float *a;    // [a_splits][L][M][d] attention-branch outputs (partial sums over splits)
+  const float *m;    // [m_splits][L][M][d] MLP-branch outputs
+  size_t a_ss, m_ss; // split strides (elements)
+  int a_splits, m_splits;
+  int l0, nl, L;
+  int M, d;
+  int mode;          // SNLP_MODE_*
+  const HcCoef *coef;
+  float *xa, *xm;    // [L][M][d] pre-mapped inputs for the next sweep (n > 1 only)
+  float *partial;    // [gridDim.x][nl][2] scratch for the norms (nullable => no norms)
+  float *resnorm;    // [L][2] (entries l0 .. l0+nl-1 written)
+  unsigned *counter; // zero on entry, left zero on exit
+};
+
+__device__ __forceinline__ float4 f4_add(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
+__device__ __forceinline__ float4 f4_sub(float4 a, float4 b) { return make_float4(a.x - b.x, a.y - b.y, a.z - b.z, a.w - b.w); }
+__device__ __forceinline__ float4 f4_fma(float s, float4 a, float4 b) {
+  return make_float4(fmaf(s, a.x, b.x), fmaf(s, a.y, b.y), fmaf(s, a.z, b.z), fmaf(s, a.w, b.w));
+}
+__device__ __forceinline__ float4 f4_scale(float s, float4 a) { return make_float4(s * a.x, s * a.y, s * a.z, s * a.w); }
+__device__ __forceinline__ float f4_sq(float4 a) { return a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w; }
+
+// NS = number of residual streams (compile time so the per-thread state stays in registers).
+template <int NS>
+__global__ void __launch_bounds__(256) k_correct(CorrParams p) {
+  extern __shared__ float s_norm[];  // [warps][nl][2]
+  const int d4 = p.d >> 2;
+  const size_t total = (size_t)p.M * d4;
+  const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const bool active = idx < total;
+  const size_t row = active ? idx / d4 : 0;
+  const int c4 = active ? (int)(idx % d4) : 0;
+  const size_t Md4 = (size_t)p.M * d4;             // float4 per [M][d] plane
+  const size_t state4 = Md4 * NS;                  // float4 per trace state
+  const float4 *a4 = reinterpret_cast<const float4 *>(p.a);
+  const float4 *m4 = reinterpret_cast<const float4 *>(p.m);
+  float4 *tr4 = reinterpret_cast<float4 *>(p.trace);
+  const size_t bm_off = row * d4 + c4;             // offset inside an [M][d] plane
+  const size_t st_off = row * NS * d4 + c4;        // offset of stream 0 inside a state
+  const bool native = (NS == 1) ? (p.mode != 2) : (p.mode == 1);  // direct form == the block itself
+  const bool want_norm = p.partial != nullptr;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+
+  float4 oldp[NS], newp[NS];
+  if (active) {
+#pragma unroll
+    for (int s = 0; s < NS; ++s) oldp[s] = newp[s] = tr4[(size_t)p.l0 * state4 + st_off + (size_t)s * d4];
+  }
+  for (int i = 0; i < p.nl; ++i) {
+    const int l = p.l0 + i;
+    float rs = 0.f, hs = 0.f;
+    if (active) {
+      float4 av = a4[(size_t)l * Md4 + bm_off];
+      for (int q = 1; q < p.a_splits; ++q) av = f4_add(av, a4[(size_t)q * (p.a_ss >> 2) + (size_t)l * Md4 + bm_off]);
+      float4 mv = m4[(size_t)l * Md4 + bm_off];
+      for (int q = 1; q < p.m_splits; ++q) mv = f4_add(mv, m4[(size_t)q * (p.m_ss >> 2) + (size_t)l * Md4 + bm_off]);
+      const HcCoef &c = p.coef[l];
+      float4 oldn[NS], newn[NS], tilde[NS];
+#pragma unroll
+      for (int r = 0; r < NS; ++r) {
+        oldn[r] = tr4[(size_t)(l + 1) * state4 + st_off + (size_t)r * d4];
+        if (NS == 1) {
+          tilde[r] = f4_add(f4_add(oldp[0], av), mv);  // F_l(h_l^k) = (h + a) + m
+        } else {
+          float4 t = f4_scale(c.A[r * NS], oldp[0]);
+#pragma unroll
+          for (int s = 1; s < NS; ++s) t = f4_fma(c.A[r * NS + s], oldp[s], t);
+          tilde[r] = f4_fma(c.cm[r], mv, f4_fma(c.ca[r], av, t));
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < NS; ++r) {
+        if (p.mode == 2) {
+          newn[r] = tilde[r];                                        // A = 0
+        } else if (native) {
+          if (NS == 1) {
+            newn[r] = f4_add(f4_add(newp[0], av), mv);               // prefix sum over depth
+          } else {
+            float4 t = f4_scale(c.A[r * NS], newp[0]);
+#pragma unroll
+            for (int s = 1; s < NS; ++s) t = f4_fma(c.A[r * NS + s], newp[s], t);
+            newn[r] = f4_fma(c.cm[r], mv, f4_fma(c.ca[r], av, t));   // affine scan with A_l
+          }
+        } else {
+          newn[r] = f4_add(tilde[r], f4_sub(newp[r], oldp[r]));      // identity surrogate on n streams
+        }
+        const float4 rr = f4_sub(tilde[r], oldn[r]);
+        rs += f4_sq(rr);
+        hs += f4_sq(oldn[r]);
+        tr4[(size_t)(l + 1) * state4 + st_off + (size_t)r * d4] = newn[r];
+      }
+      if (NS > 1 && l + 1 < p.L) {
+        const HcCoef &cn = p.coef[l + 1];
+        float4 sa = f4_scale(cn.pa[0], newn[0]), sm = f4_scale(cn.pmra[0], newn[0]);
+#pragma unroll
+        for (int s = 1; s < NS; ++s) {
+          sa = f4_fma(cn.pa[s], newn[s], sa);
+          sm = f4_fma(cn.pmra[s], newn[s], sm);
+        }
+        reinterpret_cast<float4 *>(p.xa)[(size_t)(l + 1) * Md4 + bm_off] = sa;
+        reinterpret_cast<float4 *>(p.xm)[(size_t)(l + 1) * Md4 + bm_off] = sm;
+      }
+#pragma unroll
+      for (int r = 0; r < NS; ++r) { oldp[r] = oldn[r]; newp[r] = newn[r]; }
+    }
+    if (want_norm) {
+      rs = warp_sum(rs);
+      hs = warp_sum(hs);
+      if (lane == 0) { s_norm[(warp * p.nl + i) * 2] = rs; s_norm[(warp * p.nl + i) * 2 + 1] = hs; }
+    }
+  }
+  if (!want_norm) return;
+  __syncthreads();
+  for (int i = threadIdx.x; i < p.nl * 2; i += blockDim.x) {
+    float s = 0.f;
+    for (int w = 0; w < nwarp; ++w) s += s_norm[w * p.nl * 2 + i];
+    p.partial[(size_t)blockIdx.x * p.nl * 2 + i] = s;
+  }
+  __threadfence();
+  __syncthreads();
+  __shared__ bool last;
+  if (threadIdx.x == 0) last = (atomicAdd(p.counter, 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (!last) return;
+  __threadfence();
+  for (int i = threadIdx.x; i < p.nl * 2; i += blockDim.x) {
+    double s = 0.0;
+    for (unsigned b = 0; b < gridDim.x; ++b) s += (double)__ldcg(&p.partial[(size_t)b * p.nl * 2 + i]);
+    p.resnorm[(size_t)p.l0 * 2 + i] = (float)s;
+  }
+  if (threadIdx.x == 0) *p.counter = 0u;
+}
+
+}  // namespace snlp

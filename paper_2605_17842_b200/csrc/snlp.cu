@@ -1,0 +1,854 @@
+// libsnlp: host side of the C ABI declared in include/snlp.h -- handles, workspace, launch sequences.
+// Every arithmetic step of the path runs in the CUDA kernels of generic.cuh / decode.cuh / correct.cuh.
+#include "../../include/snlp.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <string>
+#include <tuple>
+#include <vector>
+
+#include "common.cuh"
+#include "correct.cuh"
+#include "decode.cuh"
+#include "generic.cuh"
+
+using namespace snlp;
+
+// ------------------------------------------------------------------------------------------------
+// errors
+static thread_local std::string g_err;
+
+static int fail(int code, const char *fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  g_err = buf;
+  return code;
+}
+
+#define CU(call)                                                                                     \
+  do {                                                                                               \
+    cudaError_t e_ = (call);                                                                         \
+    if (e_ != cudaSuccess) return fail(SNLP_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+#define TRY(call)            \
+  do {                       \
+    int r_ = (call);         \
+    if (r_ != SNLP_OK) return r_; \
+  } while (0)
+
+extern "C" const char *snlp_last_error(void) { return g_err.c_str(); }
+
+// ------------------------------------------------------------------------------------------------
+// handles
+constexpr int kAttnChunk = 64;   // key positions per split-KV chunk
+constexpr int kMaxSplits = 4;    // K-splits of the partial-sum GEMV outputs
+constexpr int kDecodeRows = 16;  // largest row count served by the decode-regime kernels
+constexpr size_t kGemvMaxSmem = 200 * 1024;
+
+struct GraphKey {
+  int B, K, mode, nchunk;
+  const void *tin, *tout, *res;
+  const void *kv;
+  bool operator<(const GraphKey &o) const {
+    return std::tie(B, K, mode, nchunk, tin, tout, res, kv) < std::tie(o.B, o.K, o.mode, o.nchunk, o.tin, o.tout, o.res, o.kv);
+  }
+};
+struct GraphEntry { cudaGraphExec_t exec; int64_t nodes; };
+
+struct snlp_model {
+  snlp_config cfg{};
+  int device = 0;
+  bool loaded = false;
+  size_t esz = 4;  // operand element size
+  // weights
+  void *embed = nullptr, *lm_head = nullptr, *wqkv = nullptr, *wo = nullptr, *wup = nullptr, *wdn = nullptr;
+  HcCoef *coef = nullptr;
+  float2 *rope = nullptr;
+  // workspace (R = max_rows)
+  float *trace = nullptr, *xa = nullptr, *xm = nullptr, *qkv_raw = nullptr, *a = nullptr, *y_raw = nullptr, *mb = nullptr;
+  void *xn = nullptr, *q = nullptr, *att = nullptr, *z = nullptr, *sk = nullptr, *sv = nullptr, *xlm = nullptr;
+  float *attn_part = nullptr, *corr_part = nullptr, *logits = nullptr, *pm_val = nullptr;
+  int *pm_idx = nullptr;
+  unsigned *counter = nullptr;
+  int *zero = nullptr;
+  int32_t *spec = nullptr;  // [2 * (max_rows + 1)] ids / verifier tokens for draft-and-verify
+  int logit_rows = 0;
+  std::vector<void *> allocs;
+  // flags / stats
+  int use_graphs = 1, force_generic = 0;
+  int64_t launches = 0;
+  bool capturing = false;
+  int64_t cap_nodes = 0;
+  std::map<GraphKey, GraphEntry> graphs;
+  cudaStream_t cap_stream = nullptr;  // capture target: graphs are recorded here and replayed on the caller's stream
+};
+
+struct snlp_kv {
+  snlp_model *m = nullptr;
+  int B = 0, max_ctx = 0, len = 0;
+  void *k = nullptr, *v = nullptr;
+  int *pos = nullptr;
+};
+
+// a forward call's geometry and key/value store
+struct Fwd {
+  int M, B, T;
+  void *kc, *vc;
+  size_t kv_ls, kv_bs;  // elements
+  const int *pos;       // device: first position of this call
+  int pos_hi;           // host copy of *pos
+  cudaStream_t st;
+};
+
+static inline void count(snlp_model *m, int n = 1) {
+  if (m->capturing) m->cap_nodes += n;
+  else m->launches += n;
+}
+
+#define LAUNCH_CHECK()                                                                              \
+  do {                                                                                              \
+    cudaError_t e_ = cudaGetLastError();                                                            \
+    if (e_ != cudaSuccess) return fail(SNLP_ERR_CUDA, "kernel launch failed (%s:%d): %s", __FILE__, __LINE__, cudaGetErrorString(e_)); \
+  } while (0)
+
+template <typename P>
+static int dalloc(snlp_model *m, P **p, size_t bytes) {
+  void *q = nullptr;
+  if (bytes == 0) bytes = 16;
+  cudaError_t e = cudaMalloc(&q, bytes);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return fail(SNLP_ERR_OOM, "cudaMalloc of %zu bytes failed: %s", bytes, cudaGetErrorString(e));
+  }
+  m->allocs.push_back(q);
+  *p = reinterpret_cast<P *>(q);
+  return SNLP_OK;
+}
+
+static int init_kernel_attributes();
+
+static bool fast_decode_ok(const snlp_model *m, int M) {
+  const snlp_config &c = m->cfg;
+  return !m->force_generic && c.dtype == SNLP_DTYPE_BF16 && c.head_dim == 128 && M <= kDecodeRows && c.d_model % 128 == 0 &&
+         c.d_ff % 128 == 0 && (c.d_ff / kMaxSplits) % 32 == 0 && (c.d_model / kMaxSplits) % 32 == 0;
+}
+
+extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
+  if (!cfg || !out) return fail(SNLP_ERR_ARG, "snlp_create: NULL argument");
+  const snlp_config &c = *cfg;
+  if (c.n_layer < 1 || c.d_model < 1 || c.n_head < 1 || c.head_dim < 2 || c.d_ff < 1 || c.vocab < 1 || c.max_rows < 1 ||
+      c.max_batch < 1 || c.max_ctx < 1)
+    return fail(SNLP_ERR_ARG, "snlp_create: sizes must be positive");
+  if (c.n_head * c.head_dim != c.d_model) return fail(SNLP_ERR_ARG, "snlp_create: n_head*head_dim != d_model");
+  if (c.head_dim % 2 || c.head_dim > 256) return fail(SNLP_ERR_ARG, "snlp_create: head_dim must be even and <= 256");
+  if (c.d_model % 4) return fail(SNLP_ERR_ARG, "snlp_create: d_model must be a multiple of 4");
+  if (c.n_streams < 1 || c.n_streams > kMaxStreams) return fail(SNLP_ERR_ARG, "snlp_create: n_streams must be in 1..8");
+  if (c.dtype != SNLP_DTYPE_FP32 && c.dtype != SNLP_DTYPE_BF16) return fail(SNLP_ERR_ARG, "snlp_create: unknown dtype");
+  if (c.max_batch > c.max_rows) return fail(SNLP_ERR_ARG, "snlp_create: max_batch > max_rows");
+  snlp_model *m = new (std::nothrow) snlp_model;
+  if (!m) return fail(SNLP_ERR_OOM, "snlp_create: host allocation failed");
+  m->cfg = c;
+  m->esz = c.dtype == SNLP_DTYPE_BF16 ? 2 : 4;
+  cudaError_t e = cudaGetDevice(&m->device);
+  if (e != cudaSuccess) {
+    delete m;
+    return fail(SNLP_ERR_CUDA, "cudaGetDevice failed: %s", cudaGetErrorString(e));
+  }
+  const size_t L = c.n_layer, d = c.d_model, ff = c.d_ff, V = c.vocab, n = c.n_streams, R = c.max_rows, es = m->esz;
+  int rc = SNLP_OK;
+  auto A = [&](auto **p, size_t bytes) { if (rc == SNLP_OK) rc = dalloc(m, p, bytes); };
+  A(&m->embed, V * d * es);
+  A(&m->lm_head, V * d * es);
+  A(&m->wqkv, L * 3 * d * d * es);
+  A(&m->wo, L * d * d * es);
+  A(&m->wup, L * ff * d * es);
+  A(&m->wdn, L * d * ff * es);
+  A(&m->coef, L * sizeof(HcCoef));
+  A(&m->rope, (size_t)c.max_ctx * (c.head_dim / 2) * sizeof(float2));
+  A(&m->trace, (L + 1) * R * n * d * 4);
+  if (n > 1) {
+    A(&m->xa, L * R * d * 4);
+    A(&m->xm, L * R * d * 4);
+  }
+  A(&m->qkv_raw, L * R * 3 * d * 4);
+  // the decode-regime kernels write up to kMaxSplits partial sums for at most kDecodeRows rows
+  const size_t split_rows = std::max<size_t>(R, (size_t)kMaxSplits * std::min<size_t>(R, kDecodeRows));
+  A(&m->a, L * split_rows * d * 4);
+  A(&m->y_raw, L * R * ff * 4);
+  A(&m->mb, L * split_rows * d * 4);
+  A(&m->xn, L * R * d * es);
+  A(&m->q, L * R * d * es);
+  A(&m->att, L * R * d * es);
+  A(&m->z, L * R * ff * es);
+  A(&m->sk, L * R * d * es);
+  A(&m->sv, L * R * d * es);
+  A(&m->xlm, R * d * es);
+  const size_t nchunk_max = ((size_t)c.max_ctx + kAttnChunk - 1) / kAttnChunk;
+  A(&m->attn_part, L * (size_t)kDecodeRows * c.n_head * nchunk_max * kAttnPartStride * 4);
+  const size_t corr_blocks = (R * (d / 4) + 255) / 256;
+  A(&m->corr_part, corr_blocks * L * 2 * 4);
+  m->logit_rows = (int)(R < 64 ? R : 64);
+  A(&m->logits, (size_t)m->logit_rows * V * 4);
+  A(&m->pm_val, (size_t)kDecodeRows * ((V + 127) / 128) * 4);
+  A(&m->pm_idx, (size_t)kDecodeRows * ((V + 127) / 128) * 4);
+  A(&m->counter, 16);
+  A(&m->zero, 16);
+  A(&m->spec, 2 * (R + 1) * 4);
+  if (rc == SNLP_OK) {
+    if (cudaMemset(m->counter, 0, 16) != cudaSuccess || cudaMemset(m->zero, 0, 16) != cudaSuccess)
+      rc = fail(SNLP_ERR_CUDA, "cudaMemset failed");
+  }
+  if (rc == SNLP_OK) {
+    // rotary table in double on the host: (cos, sin)(pos * base^(-2i/hd))
+    const int half = c.head_dim / 2;
+    std::vector<float2> tab((size_t)c.max_ctx * half);
+    for (int pos = 0; pos < c.max_ctx; ++pos)
+      for (int i = 0; i < half; ++i) {
+        const double ang = (double)pos * std::pow((double)c.rope_base, -2.0 * i / c.head_dim);
+        tab[(size_t)pos * half + i] = make_float2((float)std::cos(ang), (float)std::sin(ang));
+      }
+    if (cudaMemcpy(m->rope, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice) != cudaSuccess)
+      rc = fail(SNLP_ERR_CUDA, "rotary table upload failed");
+  }
+  if (rc == SNLP_OK) rc = init_kernel_attributes();
+  if (rc == SNLP_OK && cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking) != cudaSuccess)
+    rc = fail(SNLP_ERR_CUDA, "cudaStreamCreateWithFlags failed");
+  if (rc != SNLP_OK) {
+    for (void *p : m->allocs) cudaFree(p);
+    delete m;
+    return rc;
+  }
+  *out = m;
+  return SNLP_OK;
+}
+
+extern "C" int snlp_destroy(snlp_model *m) {
+  if (!m) return fail(SNLP_ERR_ARG, "snlp_destroy: NULL handle");
+  cudaDeviceSynchronize();
+  for (auto &g : m->graphs) cudaGraphExecDestroy(g.second.exec);
+  if (m->cap_stream) cudaStreamDestroy(m->cap_stream);
+  for (void *p : m->allocs) cudaFree(p);
+  delete m;
+  return SNLP_OK;
+}
+
+extern "C" int snlp_load_weights(snlp_model *m, const snlp_weights *w) {
+  if (!m || !w) return fail(SNLP_ERR_ARG, "snlp_load_weights: NULL argument");
+  if (!w->embed || !w->lm_head || !w->wqkv || !w->wo || !w->wup || !w->wdn)
+    return fail(SNLP_ERR_ARG, "snlp_load_weights: NULL weight array");
+  const snlp_config &c = m->cfg;
+  const int n = c.n_streams;
+  if (n > 1 && (!w->hc_res_attn || !w->hc_res_mlp || !w->hc_pre_attn || !w->hc_pre_mlp || !w->hc_post_attn || !w->hc_post_mlp))
+    return fail(SNLP_ERR_ARG, "snlp_load_weights: n_streams > 1 needs all hc_* arrays");
+  const size_t L = c.n_layer, d = c.d_model, ff = c.d_ff, V = c.vocab, es = m->esz;
+  CU(cudaMemcpy(m->embed, w->embed, V * d * es, cudaMemcpyHostToDevice));
+  CU(cudaMemcpy(m->lm_head, w->lm_head, V * d * es, cudaMemcpyHostToDevice));
+  CU(cudaMemcpy(m->wqkv, w->wqkv, L * 3 * d * d * es, cudaMemcpyHostToDevice));
+  CU(cudaMemcpy(m->wo, w->wo, L * d * d * es, cudaMemcpyHostToDevice));
+  CU(cudaMemcpy(m->wup, w->wup, L * ff * d * es, cudaMemcpyHostToDevice));
+  CU(cudaMemcpy(m->wdn, w->wdn, L * d * ff * es, cudaMemcpyHostToDevice));
+  std::vector<HcCoef> co(L);
+  for (size_t l = 0; l < L; ++l) {
+    HcCoef &h = co[l];
+    std::memset(&h, 0, sizeof h);
+    if (n == 1) {
+      h.A[0] = h.ca[0] = h.cm[0] = h.pa[0] = h.pmra[0] = 1.f;
+      h.kappa = 1.f;
+      continue;
+    }
+    const float *Ra = w->hc_res_attn + l * n * n, *Rm = w->hc_res_mlp + l * n * n;
+    const float *Pa = w->hc_pre_attn + l * n, *Pm = w->hc_pre_mlp + l * n;
+    const float *Qa = w->hc_post_attn + l * n, *Qm = w->hc_post_mlp + l * n;
+    double kappa = 0.0;
+    for (int r = 0; r < n; ++r) {
+      double ca = 0.0, pm = 0.0;
+      for (int s = 0; s < n; ++s) {
+        double acc = 0.0;
+        for (int q = 0; q < n; ++q) acc += (double)Rm[r * n + q] * (double)Ra[q * n + s];
+        h.A[r * n + s] = (float)acc;       // A = Rm Ra
+        ca += (double)Rm[r * n + s] * (double)Qa[s];
+        pm += (double)Pm[s] * (double)Ra[s * n + r];  // (Pm Ra)[r]
+      }
+      h.ca[r] = (float)ca;
+      h.cm[r] = Qm[r];
+      h.pa[r] = Pa[r];
+      h.pmra[r] = (float)pm;
+      kappa += (double)Pm[r] * (double)Qa[r];
+    }
+    h.kappa = (float)kappa;
+  }
+  CU(cudaMemcpy(m->coef, co.data(), L * sizeof(HcCoef), cudaMemcpyHostToDevice));
+  m->loaded = true;
+  return SNLP_OK;
+}
+
+extern "C" int snlp_set_flag(snlp_model *m, int flag, int value) {
+  if (!m) return fail(SNLP_ERR_ARG, "snlp_set_flag: NULL handle");
+  if (flag == 0) m->use_graphs = value != 0;
+  else if (flag == 1) m->force_generic = value != 0;
+  else return fail(SNLP_ERR_ARG, "snlp_set_flag: unknown flag %d", flag);
+  return SNLP_OK;
+}
+
+extern "C" int snlp_launch_count(const snlp_model *m, int64_t *count_out) {
+  if (!m || !count_out) return fail(SNLP_ERR_ARG, "snlp_launch_count: NULL argument");
+  *count_out = m->launches;
+  return SNLP_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// launch sequences
+template <typename T>
+static int gemm(snlp_model *m, cudaStream_t st, const T *A, size_t a_ls, const T *W, size_t w_ls, float *C, size_t c_ls, int M, int N,
+                int K, int nl) {
+  dim3 grid((N + 63) / 64, (M + 63) / 64, nl);
+  k_gemm_nt<T><<<grid, 256, 0, st>>>(A, a_ls, W, w_ls, C, c_ls, M, N, K);
+  count(m);
+  LAUNCH_CHECK();
+  return SNLP_OK;
+}
+
+static int correct(snlp_model *m, const Fwd &f, int l0, int nl, int mode, int a_splits, int m_splits, float *resnorm) {
+  const snlp_config &c = m->cfg;
+  CorrParams p{};
+  p.trace = m->trace;
+  p.a = m->a;
+  p.m = m->mb;
+  p.a_ss = p.m_ss = (size_t)c.n_layer * f.M * c.d_model;
+  p.a_splits = a_splits;
+  p.m_splits = m_splits;
+  p.l0 = l0;
+  p.nl = nl;
+  p.L = c.n_layer;
+  p.M = f.M;
+  p.d = c.d_model;
+  p.mode = mode;
+  p.coef = m->coef;
+  p.xa = m->xa;
+  p.xm = m->xm;
+  p.partial = resnorm ? m->corr_part : nullptr;
+  p.resnorm = resnorm;
+  p.counter = m->counter;
+  const size_t total = (size_t)f.M * (c.d_model / 4);
+  const int threads = 256;
+  const unsigned blocks = (unsigned)((total + threads - 1) / threads);
+  const size_t sm = resnorm ? (size_t)(threads / 32) * nl * 2 * sizeof(float) : 0;
+  switch (c.n_streams) {
+#define CASE(NS) case NS: k_correct<NS><<<blocks, threads, sm, f.st>>>(p); break;
+    CASE(1) CASE(2) CASE(3) CASE(4) CASE(5) CASE(6) CASE(7) CASE(8)
+#undef CASE
+  }
+  count(m);
+  LAUNCH_CHECK();
+  return SNLP_OK;
+}
+
+// Blocks l0 .. l0+nl-1, each on its own current input state, then the correction over that range.
+template <typename T>
+static int run_generic(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float *resnorm) {
+  const snlp_config &c = m->cfg;
+  const int M = f.M, d = c.d_model, ff = c.d_ff, H = c.n_head, hd = c.head_dim, n = c.n_streams;
+  const size_t Md = (size_t)M * d;
+  cudaStream_t st = f.st;
+  const float *xa_src = n == 1 ? m->trace + l0 * Md : m->xa + l0 * Md;
+  const float *xm_src = n == 1 ? m->trace + l0 * Md : m->xm + l0 * Md;
+  T *xn = (T *)m->xn + l0 * Md, *q = (T *)m->q + l0 * Md, *att = (T *)m->att + l0 * Md;
+  T *z = (T *)m->z + (size_t)l0 * M * ff;
+  float *qkv = m->qkv_raw + (size_t)l0 * M * 3 * d, *a = m->a + l0 * Md, *y = m->y_raw + (size_t)l0 * M * ff, *mb = m->mb + l0 * Md;
+  T *kc = (T *)f.kc + (size_t)l0 * f.kv_ls, *vc = (T *)f.vc + (size_t)l0 * f.kv_ls;
+
+  k_rmsnorm_cast<T><<<dim3(M, nl), 256, 0, st>>>(xa_src, Md, (size_t)d, 1, xn, Md, d, c.rms_eps);
+  count(m);
+  LAUNCH_CHECK();
+  TRY(gemm<T>(m, st, xn, Md, (const T *)m->wqkv + (size_t)l0 * 3 * d * d, (size_t)3 * d * d, qkv, (size_t)M * 3 * d, M, 3 * d, d, nl));
+  k_rope_qknorm_store<T><<<dim3(M, 3 * H, nl), 128, 0, st>>>(qkv, (size_t)M * 3 * d, q, Md, kc, vc, f.kv_ls, f.kv_bs, f.T, H, hd, f.pos,
+                                                             m->rope, c.rms_eps);
+  count(m);
+  LAUNCH_CHECK();
+  k_attn_generic<T><<<dim3((M * H + 3) / 4, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, att, Md, M, f.T, H, hd, f.pos);
+  count(m);
+  LAUNCH_CHECK();
+  TRY(gemm<T>(m, st, att, Md, (const T *)m->wo + (size_t)l0 * d * d, (size_t)d * d, a, Md, M, d, d, nl));
+  k_resid_rmsnorm_cast<T><<<dim3(M, nl), 256, 0, st>>>(xm_src, Md, (size_t)d, a, Md, 1, 0, m->coef, l0, xn, Md, d, c.rms_eps);
+  count(m);
+  LAUNCH_CHECK();
+  TRY(gemm<T>(m, st, xn, Md, (const T *)m->wup + (size_t)l0 * ff * d, (size_t)ff * d, y, (size_t)M * ff, M, ff, d, nl));
+  {
+    const size_t tot = (size_t)nl * M * ff;
+    k_relu2_cast<T><<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(y, z, tot);
+    count(m);
+    LAUNCH_CHECK();
+  }
+  TRY(gemm<T>(m, st, z, (size_t)M * ff, (const T *)m->wdn + (size_t)l0 * d * ff, (size_t)d * ff, mb, Md, M, d, ff, nl));
+  return correct(m, f, l0, nl, mode, 1, 1, resnorm);
+}
+
+template <int PRO, int EPI>
+static int launch_gemv(snlp_model *m, cudaStream_t st, GemvParams &p, int ksplit, int nl) {
+  const int NT = p.M <= 8 ? 1 : 2;
+  p.kslice = p.Kd / ksplit;
+  const size_t sm = (size_t)NT * 8 * (p.kslice + kGemvPad) * 2 + (size_t)NT * 8 * (kGemvRows + 1) * 4 + 16 * 4;
+  if (sm > kGemvMaxSmem) return fail(SNLP_ERR_UNSUPPORTED, "gemv: K slice of %d needs %zu bytes of shared memory", p.kslice, sm);
+  dim3 grid(p.N / kGemvRows, ksplit, nl);
+  if (NT == 1) k_gemv_mma<1, PRO, EPI><<<grid, kGemvThreads, sm, st>>>(p);
+  else k_gemv_mma<2, PRO, EPI><<<grid, kGemvThreads, sm, st>>>(p);
+  count(m);
+  LAUNCH_CHECK();
+  return SNLP_OK;
+}
+
+template <int PRO, int EPI>
+static cudaError_t gemv_attr() {
+  cudaError_t e = cudaFuncSetAttribute(k_gemv_mma<1, PRO, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemvMaxSmem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_gemv_mma<2, PRO, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemvMaxSmem);
+}
+
+static int init_kernel_attributes() {
+  CU((gemv_attr<PRO_NORM, EPI_QKV>()));
+  CU((gemv_attr<PRO_BF16, EPI_PARTIAL>()));
+  CU((gemv_attr<PRO_RESID_NORM, EPI_RELU2>()));
+  CU((gemv_attr<PRO_NORM, EPI_LMHEAD>()));
+  return SNLP_OK;
+}
+
+// Decode-regime sweep over layers l0 .. l0+nl-1 (bf16, <= 16 rows): 7 launches independent of nl.
+static int run_decode(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float *resnorm) {
+  typedef __nv_bfloat16 bf;
+  const snlp_config &c = m->cfg;
+  const int M = f.M, d = c.d_model, ff = c.d_ff, H = c.n_head, n = c.n_streams, L = c.n_layer;
+  const size_t Md = (size_t)M * d;
+  cudaStream_t st = f.st;
+  const float *xa_src = n == 1 ? m->trace + l0 * Md : m->xa + l0 * Md;
+  const float *xm_src = n == 1 ? m->trace + l0 * Md : m->xm + l0 * Md;
+  bf *q = (bf *)m->q + l0 * Md, *att = (bf *)m->att + l0 * Md, *z = (bf *)m->z + (size_t)l0 * M * ff;
+  bf *kc = (bf *)f.kc + (size_t)l0 * f.kv_ls, *vc = (bf *)f.vc + (size_t)l0 * f.kv_ls;
+  const int so = d >= 1024 ? 2 : 1;          // K-splits of the out-projection
+  const int sd = kMaxSplits;                 // K-splits of the down-projection
+  {
+    GemvParams p{};
+    p.W = (const bf *)m->wqkv + (size_t)l0 * 3 * d * d; p.w_ls = (size_t)3 * d * d;
+    p.N = 3 * d; p.Kd = d; p.M = M;
+    p.xf = xa_src; p.xf_ls = Md; p.xf_rs = d; p.nsum = 1; p.eps = c.rms_eps;
+    p.q = q; p.q_ls = Md; p.kc = kc; p.vc = vc; p.kv_ls = f.kv_ls; p.kv_bs = f.kv_bs;
+    p.T = f.T; p.H = H; p.pos_base = f.pos; p.rope = m->rope; p.qk_eps = c.rms_eps;
+    TRY((launch_gemv<PRO_NORM, EPI_QKV>(m, st, p, 1, nl)));
+  }
+  const int nchunk = (f.pos_hi + f.T - 1) / kAttnChunk + 1;
+  k_attn_decode<kAttnChunk><<<dim3(nchunk, f.B * H, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, m->attn_part, f.T, H, f.pos);
+  count(m);
+  LAUNCH_CHECK();
+  k_attn_combine<<<dim3(M * H, nl), 128, 0, st>>>(m->attn_part, nchunk, f.T, H, att, Md);
+  count(m);
+  LAUNCH_CHECK();
+  {
+    GemvParams p{};
+    p.W = (const bf *)m->wo + (size_t)l0 * d * d; p.w_ls = (size_t)d * d;
+    p.N = d; p.Kd = d; p.M = M;
+    p.xb = att; p.xb_ls = Md;
+    p.out = m->a + l0 * Md; p.out_ls = Md; p.out_ss = (size_t)L * Md;
+    TRY((launch_gemv<PRO_BF16, EPI_PARTIAL>(m, st, p, so, nl)));
+  }
+  {
+    GemvParams p{};
+    p.W = (const bf *)m->wup + (size_t)l0 * ff * d; p.w_ls = (size_t)ff * d;
+    p.N = ff; p.Kd = d; p.M = M;
+    p.xf = xm_src; p.xf_ls = Md; p.xf_rs = d; p.nsum = 1; p.eps = c.rms_eps;
+    p.ap = m->a + l0 * Md; p.ap_ls = Md; p.ap_ss = (size_t)L * Md; p.ap_splits = so; p.coef = m->coef + l0;
+    p.zout = z; p.z_ls = (size_t)M * ff;
+    TRY((launch_gemv<PRO_RESID_NORM, EPI_RELU2>(m, st, p, 1, nl)));
+  }
+  {
+    GemvParams p{};
+    p.W = (const bf *)m->wdn + (size_t)l0 * d * ff; p.w_ls = (size_t)d * ff;
+    p.N = d; p.Kd = ff; p.M = M;
+    p.xb = z; p.xb_ls = (size_t)M * ff;
+    p.out = m->mb + l0 * Md; p.out_ls = Md; p.out_ss = (size_t)L * Md;
+    TRY((launch_gemv<PRO_BF16, EPI_PARTIAL>(m, st, p, sd, nl)));
+  }
+  return correct(m, f, l0, nl, mode, so, sd, resnorm);
+}
+
+static int run_layers(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float *resnorm) {
+  if (fast_decode_ok(m, f.M)) return run_decode(m, f, l0, nl, mode, resnorm);
+  if (m->cfg.dtype == SNLP_DTYPE_BF16) return run_generic<__nv_bfloat16>(m, f, l0, nl, mode, resnorm);
+  return run_generic<float>(m, f, l0, nl, mode, resnorm);
+}
+
+static int native_mode(const snlp_model *m) { return m->cfg.n_streams > 1 ? SNLP_MODE_HCN : SNLP_MODE_IDN; }
+
+static int premix(snlp_model *m, const Fwd &f, int l0, int nl) {
+  const snlp_config &c = m->cfg;
+  if (c.n_streams == 1) return SNLP_OK;
+  const size_t Md = (size_t)f.M * c.d_model;
+  k_premix<<<dim3((unsigned)((Md + 255) / 256), nl), 256, 0, f.st>>>(m->trace, Md * c.n_streams, c.n_streams, c.d_model, Md, m->coef, l0,
+                                                                    m->xa, m->xm, Md);
+  count(m);
+  LAUNCH_CHECK();
+  return SNLP_OK;
+}
+
+// Alg. 1 over the internal trace (trace[0] must hold h_0).
+static int sequential(snlp_model *m, const Fwd &f) {
+  TRY(premix(m, f, 0, 1));
+  for (int l = 0; l < m->cfg.n_layer; ++l) TRY(run_layers(m, f, l, 1, native_mode(m), nullptr));
+  return SNLP_OK;
+}
+
+// Alg. 2 (S = 0, h0 init) over the internal trace (trace[0] must hold h_0).
+static int parallel(snlp_model *m, const Fwd &f, int K, int mode, float *resnorm_out) {
+  const snlp_config &c = m->cfg;
+  const size_t n4 = (size_t)f.M * c.n_streams * c.d_model / 4;
+  k_bcast_trace<<<(unsigned)((n4 + 255) / 256), 256, 0, f.st>>>(reinterpret_cast<const float4 *>(m->trace),
+                                                               reinterpret_cast<float4 *>(m->trace) + n4, n4, c.n_layer);
+  count(m);
+  LAUNCH_CHECK();
+  TRY(premix(m, f, 0, c.n_layer));
+  for (int k = 0; k < K; ++k)
+    TRY(run_layers(m, f, 0, c.n_layer, mode, resnorm_out ? resnorm_out + (size_t)k * c.n_layer * 2 : nullptr));
+  return SNLP_OK;
+}
+
+static int lm_head_impl(snlp_model *m, cudaStream_t st, const float *hL, size_t row_stride, int rows, float *logits, int32_t *argmax) {
+  const snlp_config &c = m->cfg;
+  const int d = c.d_model, V = c.vocab, n = c.n_streams;
+  if (!m->force_generic && c.dtype == SNLP_DTYPE_BF16 && rows <= kDecodeRows && d % 32 == 0 && V % 128 == 0) {
+    GemvParams p{};
+    p.W = (const __nv_bfloat16 *)m->lm_head; p.w_ls = 0;
+    p.N = V; p.Kd = d; p.M = rows;
+    p.xf = hL; p.xf_ls = 0; p.xf_rs = row_stride; p.nsum = n; p.eps = c.rms_eps;
+    p.logits = logits; p.pm_val = m->pm_val; p.pm_idx = m->pm_idx; p.ntile = V / 128;
+    TRY((launch_gemv<PRO_NORM, EPI_LMHEAD>(m, st, p, 1, 1)));
+    if (argmax) {
+      k_argmax_tiles<<<rows, 256, 0, st>>>(m->pm_val, m->pm_idx, V / 128, argmax);
+      count(m);
+      LAUNCH_CHECK();
+    }
+    return SNLP_OK;
+  }
+  for (int r0 = 0; r0 < rows; r0 += m->logit_rows) {
+    const int nr = rows - r0 < m->logit_rows ? rows - r0 : m->logit_rows;
+    float *lg = logits ? logits + (size_t)r0 * V : m->logits;
+    const float *src = hL + (size_t)r0 * row_stride;
+    if (c.dtype == SNLP_DTYPE_BF16) {
+      typedef __nv_bfloat16 T;
+      k_rmsnorm_cast<T><<<dim3(nr, 1), 256, 0, st>>>(src, 0, row_stride, n, (T *)m->xlm, 0, d, c.rms_eps);
+      count(m);
+      LAUNCH_CHECK();
+      TRY(gemm<T>(m, st, (const T *)m->xlm, 0, (const T *)m->lm_head, 0, lg, 0, nr, V, d, 1));
+    } else {
+      typedef float T;
+      k_rmsnorm_cast<T><<<dim3(nr, 1), 256, 0, st>>>(src, 0, row_stride, n, (T *)m->xlm, 0, d, c.rms_eps);
+      count(m);
+      LAUNCH_CHECK();
+      TRY(gemm<T>(m, st, (const T *)m->xlm, 0, (const T *)m->lm_head, 0, lg, 0, nr, V, d, 1));
+    }
+    if (argmax) {
+      k_argmax_rows<<<nr, 256, 0, st>>>(lg, V, argmax + r0);
+      count(m);
+      LAUNCH_CHECK();
+    }
+  }
+  return SNLP_OK;
+}
+
+static int embed_impl(snlp_model *m, cudaStream_t st, const int32_t *ids, int rows, float *h0) {
+  const snlp_config &c = m->cfg;
+  if (c.dtype == SNLP_DTYPE_BF16)
+    k_embed<__nv_bfloat16><<<rows, 128, 0, st>>>(ids, (const __nv_bfloat16 *)m->embed, h0, c.d_model, c.n_streams, c.vocab);
+  else
+    k_embed<float><<<rows, 128, 0, st>>>(ids, (const float *)m->embed, h0, c.d_model, c.n_streams, c.vocab);
+  count(m);
+  LAUNCH_CHECK();
+  return SNLP_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// public entry points
+static int check_model(const snlp_model *m, const char *who) {
+  if (!m) return fail(SNLP_ERR_ARG, "%s: NULL model handle", who);
+  if (!m->loaded) return fail(SNLP_ERR_STATE, "%s: weights not loaded", who);
+  return SNLP_OK;
+}
+
+static int check_shape(const snlp_model *m, int B, int T, const char *who) {
+  if (B < 1 || T < 1) return fail(SNLP_ERR_ARG, "%s: B and T must be >= 1", who);
+  const snlp_config &c = m->cfg;
+  if ((int64_t)B * T > c.max_rows) return fail(SNLP_ERR_SHAPE, "%s: B*T = %lld exceeds max_rows = %d", who, (long long)B * T, c.max_rows);
+  if (B > c.max_batch) return fail(SNLP_ERR_SHAPE, "%s: B = %d exceeds max_batch = %d", who, B, c.max_batch);
+  if (T > c.max_ctx) return fail(SNLP_ERR_SHAPE, "%s: T = %d exceeds max_ctx = %d", who, T, c.max_ctx);
+  return SNLP_OK;
+}
+
+extern "C" int snlp_embed(snlp_model *m, const int32_t *ids, int B, int T, float *h0, void *stream) {
+  TRY(check_model(m, "snlp_embed"));
+  if (!ids || !h0) return fail(SNLP_ERR_ARG, "snlp_embed: NULL pointer");
+  TRY(check_shape(m, B, T, "snlp_embed"));
+  return embed_impl(m, (cudaStream_t)stream, ids, B * T, h0);
+}
+
+static Fwd scratch_fwd(snlp_model *m, int B, int T, cudaStream_t st) {
+  Fwd f{};
+  f.M = B * T; f.B = B; f.T = T;
+  f.kc = m->sk; f.vc = m->sv;
+  f.kv_bs = (size_t)T * m->cfg.d_model;
+  f.kv_ls = (size_t)B * f.kv_bs;
+  f.pos = m->zero; f.pos_hi = 0; f.st = st;
+  return f;
+}
+
+extern "C" int snlp_forward_sequential(snlp_model *m, const float *h0, int B, int T, float *trace_out, void *stream) {
+  TRY(check_model(m, "snlp_forward_sequential"));
+  if (!h0) return fail(SNLP_ERR_ARG, "snlp_forward_sequential: NULL h0");
+  TRY(check_shape(m, B, T, "snlp_forward_sequential"));
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t state = (size_t)B * T * m->cfg.n_streams * m->cfg.d_model;
+  CU(cudaMemcpyAsync(m->trace, h0, state * 4, cudaMemcpyDeviceToDevice, st));
+  Fwd f = scratch_fwd(m, B, T, st);
+  TRY(sequential(m, f));
+  if (trace_out) CU(cudaMemcpyAsync(trace_out, m->trace, (m->cfg.n_layer + 1) * state * 4, cudaMemcpyDeviceToDevice, st));
+  return SNLP_OK;
+}
+
+static int check_mode(int mode, const char *who) {
+  if (mode != SNLP_MODE_IDN && mode != SNLP_MODE_HCN && mode != SNLP_MODE_NOCORR) return fail(SNLP_ERR_ARG, "%s: unknown mode %d", who, mode);
+  return SNLP_OK;
+}
+
+extern "C" int snlp_forward_parallel(snlp_model *m, const float *h0, int B, int T, int K, int mode, float *trace_out, float *resnorm_out,
+                                     void *stream) {
+  TRY(check_model(m, "snlp_forward_parallel"));
+  if (!h0) return fail(SNLP_ERR_ARG, "snlp_forward_parallel: NULL h0");
+  if (K < 1) return fail(SNLP_ERR_ARG, "snlp_forward_parallel: K must be >= 1 (got %d)", K);
+  TRY(check_mode(mode, "snlp_forward_parallel"));
+  TRY(check_shape(m, B, T, "snlp_forward_parallel"));
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t state = (size_t)B * T * m->cfg.n_streams * m->cfg.d_model;
+  CU(cudaMemcpyAsync(m->trace, h0, state * 4, cudaMemcpyDeviceToDevice, st));
+  Fwd f = scratch_fwd(m, B, T, st);
+  TRY(parallel(m, f, K, mode, resnorm_out));
+  if (trace_out) CU(cudaMemcpyAsync(trace_out, m->trace, (m->cfg.n_layer + 1) * state * 4, cudaMemcpyDeviceToDevice, st));
+  return SNLP_OK;
+}
+
+extern "C" int snlp_lm_head(snlp_model *m, const float *hL, int rows, float *logits, int32_t *argmax, void *stream) {
+  TRY(check_model(m, "snlp_lm_head"));
+  if (!hL || (!logits && !argmax)) return fail(SNLP_ERR_ARG, "snlp_lm_head: NULL pointer");
+  if (rows < 1) return fail(SNLP_ERR_ARG, "snlp_lm_head: rows must be >= 1");
+  if (rows > m->cfg.max_rows) return fail(SNLP_ERR_SHAPE, "snlp_lm_head: rows = %d exceeds max_rows = %d", rows, m->cfg.max_rows);
+  return lm_head_impl(m, (cudaStream_t)stream, hL, (size_t)m->cfg.n_streams * m->cfg.d_model, rows, logits, argmax);
+}
+
+extern "C" int snlp_kv_create(snlp_model *m, int B, int max_ctx, snlp_kv **out) {
+  if (!m || !out) return fail(SNLP_ERR_ARG, "snlp_kv_create: NULL argument");
+  if (B < 1 || max_ctx < 1) return fail(SNLP_ERR_ARG, "snlp_kv_create: B and max_ctx must be >= 1");
+  if (B > m->cfg.max_batch) return fail(SNLP_ERR_SHAPE, "snlp_kv_create: B = %d exceeds max_batch = %d", B, m->cfg.max_batch);
+  if (max_ctx > m->cfg.max_ctx) return fail(SNLP_ERR_SHAPE, "snlp_kv_create: max_ctx = %d exceeds the model's %d", max_ctx, m->cfg.max_ctx);
+  snlp_kv *kv = new (std::nothrow) snlp_kv;
+  if (!kv) return fail(SNLP_ERR_OOM, "snlp_kv_create: host allocation failed");
+  kv->m = m; kv->B = B; kv->max_ctx = max_ctx;
+  const size_t bytes = (size_t)m->cfg.n_layer * B * max_ctx * m->cfg.d_model * m->esz;
+  if (cudaMalloc(&kv->k, bytes) != cudaSuccess || cudaMalloc(&kv->v, bytes) != cudaSuccess || cudaMalloc(&kv->pos, 16) != cudaSuccess) {
+    cudaGetLastError();
+    cudaFree(kv->k); cudaFree(kv->v); cudaFree(kv->pos);
+    delete kv;
+    return fail(SNLP_ERR_OOM, "snlp_kv_create: cudaMalloc of 2 x %zu bytes failed", bytes);
+  }
+  if (cudaMemset(kv->k, 0, bytes) != cudaSuccess || cudaMemset(kv->v, 0, bytes) != cudaSuccess || cudaMemset(kv->pos, 0, 16) != cudaSuccess) {
+    cudaFree(kv->k); cudaFree(kv->v); cudaFree(kv->pos);
+    delete kv;
+    return fail(SNLP_ERR_CUDA, "snlp_kv_create: cudaMemset failed");
+  }
+  *out = kv;
+  return SNLP_OK;
+}
+
+extern "C" int snlp_kv_destroy(snlp_kv *kv) {
+  if (!kv) return fail(SNLP_ERR_ARG, "snlp_kv_destroy: NULL handle");
+  cudaDeviceSynchronize();
+  // graphs captured against this cache hold its pointers
+  for (auto it = kv->m->graphs.begin(); it != kv->m->graphs.end();) {
+    if (it->first.kv == kv) { cudaGraphExecDestroy(it->second.exec); it = kv->m->graphs.erase(it); }
+    else ++it;
+  }
+  cudaFree(kv->k); cudaFree(kv->v); cudaFree(kv->pos);
+  delete kv;
+  return SNLP_OK;
+}
+
+extern "C" int snlp_kv_len(const snlp_kv *kv, int32_t *len) {
+  if (!kv || !len) return fail(SNLP_ERR_ARG, "snlp_kv_len: NULL argument");
+  *len = kv->len;
+  return SNLP_OK;
+}
+
+extern "C" int snlp_kv_truncate(snlp_kv *kv, int new_len, void *stream) {
+  if (!kv) return fail(SNLP_ERR_ARG, "snlp_kv_truncate: NULL handle");
+  if (new_len < 0 || new_len > kv->len) return fail(SNLP_ERR_ARG, "snlp_kv_truncate: new_len = %d outside 0..%d", new_len, kv->len);
+  k_set_int<<<1, 1, 0, (cudaStream_t)stream>>>(kv->pos, new_len);
+  count(kv->m);
+  LAUNCH_CHECK();
+  kv->len = new_len;
+  return SNLP_OK;
+}
+
+static Fwd kv_fwd(snlp_model *m, snlp_kv *kv, int T, cudaStream_t st) {
+  Fwd f{};
+  f.M = kv->B * T; f.B = kv->B; f.T = T;
+  f.kc = kv->k; f.vc = kv->v;
+  f.kv_bs = (size_t)kv->max_ctx * m->cfg.d_model;
+  f.kv_ls = (size_t)kv->B * f.kv_bs;
+  f.pos = kv->pos; f.pos_hi = kv->len; f.st = st;
+  return f;
+}
+
+__global__ void k_gather_ids(const int32_t *__restrict__ ids, int32_t *__restrict__ out, int B, int Tc, int T, int t0) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < B * Tc) out[i] = ids[(size_t)(i / Tc) * T + t0 + (i % Tc)];
+}
+
+extern "C" int snlp_prefill(snlp_model *m, snlp_kv *kv, const int32_t *ids, int B, int T, int32_t *last_argmax, void *stream) {
+  TRY(check_model(m, "snlp_prefill"));
+  if (!kv || !ids) return fail(SNLP_ERR_ARG, "snlp_prefill: NULL pointer");
+  if (kv->m != m) return fail(SNLP_ERR_ARG, "snlp_prefill: cache belongs to another model");
+  if (B < 1 || T < 1) return fail(SNLP_ERR_ARG, "snlp_prefill: B and T must be >= 1");
+  if (B != kv->B) return fail(SNLP_ERR_SHAPE, "snlp_prefill: B = %d but the cache holds %d sequences", B, kv->B);
+  if (kv->len + T > kv->max_ctx) return fail(SNLP_ERR_SHAPE, "snlp_prefill: len %d + T %d exceeds max_ctx %d", kv->len, T, kv->max_ctx);
+  cudaStream_t st = (cudaStream_t)stream;
+  const snlp_config &c = m->cfg;
+  const int tc_max = c.max_rows / B;
+  if (tc_max < 1) return fail(SNLP_ERR_SHAPE, "snlp_prefill: B exceeds max_rows");
+  const size_t nd = (size_t)c.n_streams * c.d_model;
+  int Tc = 0;
+  for (int t0 = 0; t0 < T; t0 += Tc) {
+    Tc = T - t0 < tc_max ? T - t0 : tc_max;
+    k_gather_ids<<<(B * Tc + 255) / 256, 256, 0, st>>>(ids, m->spec, B, Tc, T, t0);
+    count(m);
+    LAUNCH_CHECK();
+    TRY(embed_impl(m, st, m->spec, B * Tc, m->trace));
+    Fwd f = kv_fwd(m, kv, Tc, st);
+    TRY(sequential(m, f));
+    k_add_int<<<1, 1, 0, st>>>(kv->pos, Tc);
+    count(m);
+    LAUNCH_CHECK();
+    kv->len += Tc;
+  }
+  if (last_argmax) {
+    const float *hL = m->trace + (size_t)c.n_layer * B * Tc * nd + (size_t)(Tc - 1) * nd;
+    TRY(lm_head_impl(m, st, hL, (size_t)Tc * nd, B, nullptr, last_argmax));
+  }
+  return SNLP_OK;
+}
+
+// enqueue one decode step (no graph handling, no host-side length update)
+static int decode_launches(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, int K, int mode, int32_t *tok_out, float *resnorm_out,
+                           cudaStream_t st) {
+  const snlp_config &c = m->cfg;
+  TRY(embed_impl(m, st, tok_in, kv->B, m->trace));
+  Fwd f = kv_fwd(m, kv, 1, st);
+  if (K == 0) TRY(sequential(m, f));
+  else TRY(parallel(m, f, K, mode, resnorm_out));
+  const size_t nd = (size_t)c.n_streams * c.d_model;
+  TRY(lm_head_impl(m, st, m->trace + (size_t)c.n_layer * kv->B * nd, nd, kv->B, nullptr, tok_out));
+  k_add_int<<<1, 1, 0, st>>>(kv->pos, 1);
+  count(m);
+  LAUNCH_CHECK();
+  return SNLP_OK;
+}
+
+static int decode_step_impl(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, int K, int mode, int32_t *tok_out, float *resnorm_out,
+                            cudaStream_t st) {
+  if (!m->use_graphs) {
+    TRY(decode_launches(m, kv, tok_in, K, mode, tok_out, resnorm_out, st));
+    kv->len += 1;
+    return SNLP_OK;
+  }
+  const bool fast = fast_decode_ok(m, kv->B);
+  GraphKey key{kv->B, K, mode, fast ? kv->len / kAttnChunk + 1 : 0, tok_in, tok_out, resnorm_out, kv};
+  auto it = m->graphs.find(key);
+  if (it == m->graphs.end()) {
+    if (m->graphs.size() >= 256) {
+      for (auto &g : m->graphs) cudaGraphExecDestroy(g.second.exec);
+      m->graphs.clear();
+    }
+    cudaGraph_t graph = nullptr;
+    CU(cudaStreamBeginCapture(m->cap_stream, cudaStreamCaptureModeThreadLocal));
+    m->capturing = true;
+    m->cap_nodes = 0;
+    const int rc = decode_launches(m, kv, tok_in, K, mode, tok_out, resnorm_out, m->cap_stream);
+    m->capturing = false;
+    cudaError_t e = cudaStreamEndCapture(m->cap_stream, &graph);
+    if (rc != SNLP_OK) {
+      if (graph) cudaGraphDestroy(graph);
+      return rc;
+    }
+    if (e != cudaSuccess) return fail(SNLP_ERR_CUDA, "cudaStreamEndCapture failed: %s", cudaGetErrorString(e));
+    GraphEntry ge{};
+    ge.nodes = m->cap_nodes;
+    e = cudaGraphInstantiate(&ge.exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e != cudaSuccess) return fail(SNLP_ERR_CUDA, "cudaGraphInstantiate failed: %s", cudaGetErrorString(e));
+    it = m->graphs.emplace(key, ge).first;
+  }
+  CU(cudaGraphLaunch(it->second.exec, st));
+  m->launches += it->second.nodes;
+  kv->len += 1;
+  return SNLP_OK;
+}
+
+extern "C" int snlp_decode_step(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, int K, int mode, int32_t *tok_out, float *resnorm_out,
+                                void *stream) {
+  TRY(check_model(m, "snlp_decode_step"));
+  if (!kv || !tok_in || !tok_out) return fail(SNLP_ERR_ARG, "snlp_decode_step: NULL pointer");
+  if (kv->m != m) return fail(SNLP_ERR_ARG, "snlp_decode_step: cache belongs to another model");
+  if (K < 0) return fail(SNLP_ERR_ARG, "snlp_decode_step: K must be >= 0 (got %d)", K);
+  TRY(check_mode(mode, "snlp_decode_step"));
+  if (kv->len + 1 > kv->max_ctx) return fail(SNLP_ERR_SHAPE, "snlp_decode_step: cache is full (len %d, max_ctx %d)", kv->len, kv->max_ctx);
+  return decode_step_impl(m, kv, tok_in, K, mode, tok_out, K > 0 ? resnorm_out : nullptr, (cudaStream_t)stream);
+}
+
+extern "C" int snlp_draft_and_verify(snlp_model *m, snlp_kv *kv, int32_t *last_tok, int block, int K, int mode, int32_t *emitted,
+                                     int32_t *n_emitted, int32_t *n_accepted, void *stream) {
+  TRY(check_model(m, "snlp_draft_and_verify"));
+  if (!kv || !last_tok || !emitted || !n_emitted || !n_accepted) return fail(SNLP_ERR_ARG, "snlp_draft_and_verify: NULL pointer");
+  if (kv->m != m) return fail(SNLP_ERR_ARG, "snlp_draft_and_verify: cache belongs to another model");
+  if (block < 1) return fail(SNLP_ERR_ARG, "snlp_draft_and_verify: block must be >= 1");
+  if (K < 1) return fail(SNLP_ERR_ARG, "snlp_draft_and_verify: K must be >= 1");
+  TRY(check_mode(mode, "snlp_draft_and_verify"));
+  if (kv->B != 1) return fail(SNLP_ERR_SHAPE, "snlp_draft_and_verify: batch must be 1 (cache holds %d)", kv->B);
+  if (block + 1 > m->cfg.max_rows) return fail(SNLP_ERR_SHAPE, "snlp_draft_and_verify: block+1 exceeds max_rows");
+  if (kv->len + block + 1 > kv->max_ctx) return fail(SNLP_ERR_SHAPE, "snlp_draft_and_verify: len %d + block+1 exceeds max_ctx %d", kv->len, kv->max_ctx);
+  cudaStream_t st = (cudaStream_t)stream;
+  const snlp_config &c = m->cfg;
+  const int len0 = kv->len;
+  int32_t *ids = m->spec;                          // [block+1]: last_tok, x_1..x_block
+  int32_t *y = m->spec + (c.max_rows + 1);         // [block+1]: verifier tokens
+  CU(cudaMemcpyAsync(ids, last_tok, 4, cudaMemcpyDeviceToDevice, st));
+  for (int i = 0; i < block; ++i) TRY(decode_step_impl(m, kv, ids + i, K, mode, ids + i + 1, nullptr, st));
+  k_set_int<<<1, 1, 0, st>>>(kv->pos, len0);
+  count(m);
+  LAUNCH_CHECK();
+  kv->len = len0;
+  TRY(embed_impl(m, st, ids, block + 1, m->trace));
+  Fwd f = kv_fwd(m, kv, block + 1, st);
+  TRY(sequential(m, f));
+  const size_t nd = (size_t)c.n_streams * c.d_model;
+  TRY(lm_head_impl(m, st, m->trace + (size_t)c.n_layer * (block + 1) * nd, nd, block + 1, nullptr, y));
+  k_accept<<<1, 32, 0, st>>>(ids + 1, y, block, emitted, n_emitted, n_accepted, last_tok, kv->pos, len0);
+  count(m);
+  LAUNCH_CHECK();
+  int32_t n = 0;
+  CU(cudaMemcpyAsync(&n, n_accepted, 4, cudaMemcpyDeviceToHost, st));
+  CU(cudaStreamSynchronize(st));
+  kv->len = len0 + n + 1;
+  return SNLP_OK;
+}

@@ -1,0 +1,209 @@
+"""GPU parity of KV-cached decoding and greedy self-speculative decoding against the oracle."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import snlp_oracle as O
+from paper_2605_17842_b200 import synth
+from tests.gpu_util import TOL, dev, make_model
+
+pytestmark = pytest.mark.gpu
+
+F32 = synth.ModelConfig(4, 64, 2, 32, 256, 256, 1, "fp32")
+F32_HC = synth.ModelConfig(3, 64, 2, 32, 128, 256, 4, "fp32")
+BF16 = synth.ModelConfig(4, 256, 2, 128, 512, 1024, 1, "bf16")       # decode-regime kernels
+BF16_GEN = synth.ModelConfig(3, 128, 2, 64, 256, 512, 1, "bf16")     # generic kernels
+
+
+def weights(cfg):
+    return synth.make_weights(cfg, seed=1234, std=0.05, embed_std=1.0)
+
+
+def oracle_kv(cfg, B, ctx):
+    return O.LayerKV(cfg.n_layer, B, ctx, cfg.n_head, cfg.head_dim)
+
+
+def margin_tau(cfg, W):
+    # |logit error| <= tol * ||x_norm|| * ||w_row||, for the two logits being compared
+    return 2.0 * TOL[cfg.dtype] * math.sqrt(cfg.d_model) * float(np.max(np.linalg.norm(W.lm_head.astype(np.float64), axis=1)))
+
+
+@pytest.mark.parametrize("cfg,K", [(F32, 0), (F32, 2), (F32_HC, 0), (F32_HC, 2)])
+def test_fp32_greedy_token_stream_is_bit_exact(cfg, K):
+    W = weights(cfg)
+    B, Tp, steps = 2, 9, 6
+    ids = synth.make_ids(cfg, B, Tp, seed=3)
+    mode = O.MODE_HCN if cfg.n_streams > 1 else O.MODE_IDN
+    kv_o = oracle_kv(cfg, B, 32)
+    tok = O.greedy(O.prefill(cfg, W, ids, kv_o))
+    want = [tok.copy()]
+    for _ in range(steps):
+        tok, _ = O.decode_step(cfg, W, kv_o, tok, K, mode)
+        want.append(tok.copy())
+    m = make_model(cfg, W, max_rows=B * Tp, max_batch=B, max_ctx=32)
+    kv = m.kv_cache(B, 32)
+    t = m.prefill(kv, dev(ids))
+    got = [t.cpu().numpy().copy()]
+    for _ in range(steps):
+        t = m.decode_step(kv, t, K, mode)
+        got.append(t.cpu().numpy().copy())
+    assert len(kv) == Tp + steps
+    assert np.array_equal(np.array(got), np.array(want))
+
+
+@pytest.mark.parametrize("cfg", [BF16, BF16_GEN])
+@pytest.mark.parametrize("K", [0, 2])
+def test_bf16_greedy_tokens_teacher_forced(cfg, K):
+    """The oracle replays the GPU's own token history; the GPU token must be the oracle's argmax
+    wherever the oracle's margin over it exceeds the logit error bound implied by the 2e-2 state
+    tolerance.  Sub-margin positions are counted, not silently passed."""
+    W = weights(cfg)
+    B, Tp, steps = 2, 40, 8
+    ids = synth.make_ids(cfg, B, Tp, seed=4)
+    m = make_model(cfg, W, max_rows=B * Tp, max_batch=B, max_ctx=64)
+    kv = m.kv_cache(B, 64)
+    t = m.prefill(kv, dev(ids))
+    hist = [t.cpu().numpy().copy()]
+    for _ in range(steps):
+        t = m.decode_step(kv, t, K, O.MODE_IDN)
+        hist.append(t.cpu().numpy().copy())
+    tau = margin_tau(cfg, W)
+    kv_o = oracle_kv(cfg, B, 64)
+    logits = O.prefill(cfg, W, ids, kv_o)
+    sub_margin = 0
+    for s in range(steps + 1):
+        g = hist[s]
+        top = logits[np.arange(B), np.argmax(logits, -1)]
+        marg = top - logits[np.arange(B), g]
+        assert np.all(marg <= tau), (s, marg, tau)
+        sub_margin += int(np.sum((marg > 0)))
+        if s < steps:
+            _, logits = O.decode_step(cfg, W, kv_o, g, K, O.MODE_IDN)
+    assert sub_margin <= (steps + 1) * B // 4  # near-ties are the exception
+
+
+@pytest.mark.parametrize("cfg", [F32, BF16, BF16_GEN, F32_HC])
+def test_decode_with_K_equal_L_equals_sequential_decode_on_gpu(cfg):
+    W = weights(cfg)
+    B, Tp = 2, 12
+    ids = dev(synth.make_ids(cfg, B, Tp, seed=5))
+    m = make_model(cfg, W, max_rows=B * Tp, max_batch=B, max_ctx=32)
+    mode = O.MODE_HCN if cfg.n_streams > 1 else O.MODE_IDN
+    outs = []
+    for K in (0, cfg.n_layer):
+        kv = m.kv_cache(B, 32)
+        t = m.prefill(kv, ids)
+        seq = [t.clone()]
+        for _ in range(5):
+            t = m.decode_step(kv, t, K, mode)
+            seq.append(t.clone())
+        outs.append(torch.stack(seq))
+        kv.close()
+    assert torch.equal(outs[0], outs[1])
+
+
+@pytest.mark.parametrize("cfg", [F32, BF16])
+def test_step_by_step_decode_agrees_with_chunked_prefill(cfg):
+    """Prefill of T tokens in one call, in chunks (max_rows smaller than B*T), and token by token all
+    leave a cache from which the next greedy token is the same."""
+    W = weights(cfg)
+    B, Tp = 2, 20
+    ids_np = synth.make_ids(cfg, B, Tp, seed=6)
+    ids = dev(ids_np)
+    big = make_model(cfg, W, max_rows=B * Tp, max_batch=B, max_ctx=32)
+    kv = big.kv_cache(B, 32)
+    t_one = big.prefill(kv, ids).cpu().numpy()
+    small = make_model(cfg, W, max_rows=B * 6, max_batch=B, max_ctx=32)   # 4 chunks: 6, 6, 6, 2
+    kv2 = small.kv_cache(B, 32)
+    t_chunk = small.prefill(kv2, ids).cpu().numpy()
+    assert len(kv2) == Tp
+    kv3 = big.kv_cache(B, 32)
+    for s in range(Tp):
+        t_step = big.decode_step(kv3, dev(ids_np[:, s].copy()), 0)
+    # the oracle's token (fp64) settles fp32; in bf16 the three library paths may differ only at near-ties
+    kv_o = oracle_kv(cfg, B, 32)
+    logits = O.prefill(cfg, W, ids_np, kv_o)
+    tau = margin_tau(cfg, W) if cfg.dtype == "bf16" else 0.0
+    for got in (t_one, t_chunk, t_step.cpu().numpy()):
+        top = logits[np.arange(B), np.argmax(logits, -1)]
+        assert np.all(top - logits[np.arange(B), got] <= tau)
+
+
+@pytest.mark.parametrize("cfg,K", [(F32, 1), (F32, 2), (BF16, 1), (BF16, 2), (BF16_GEN, 1)])
+def test_draft_and_verify_reproduces_sequential_greedy(cfg, K):
+    W = weights(cfg)
+    Tp, block, n_tokens = 10, 4, 24
+    ids_np = synth.make_ids(cfg, 1, Tp, seed=7)
+    m = make_model(cfg, W, max_rows=max(Tp, block + 1), max_batch=1, max_ctx=96)
+    # the library's own sequential greedy stream
+    kv = m.kv_cache(1, 96)
+    first = m.prefill(kv, dev(ids_np))
+    t, want = first.clone(), []
+    for _ in range(n_tokens + block + 1):
+        t = m.decode_step(kv, t, 0)
+        want.append(int(t.item()))
+    kv.close()
+    # self-speculative decoding must emit exactly that stream
+    kv = m.kv_cache(1, 96)
+    last = m.prefill(kv, dev(ids_np)).clone()
+    got, accepted, rounds = [], 0, 0
+    while len(got) < n_tokens:
+        emitted, n_acc = m.draft_and_verify(kv, last, block, K, O.MODE_IDN)
+        assert len(emitted) == n_acc + 1 and 1 <= len(emitted) <= block + 1
+        assert int(last.item()) == emitted[-1]
+        got += emitted
+        accepted += n_acc
+        rounds += 1
+        assert len(kv) == Tp + len(got)
+    assert got == want[:len(got)]
+    if cfg.dtype == "fp32":
+        # accept / reject decisions are bit-exact against the oracle under greedy decoding
+        kv_o = oracle_kv(cfg, 1, 96)
+        lt = int(O.greedy(O.prefill(cfg, W, ids_np, kv_o))[0])
+        o_got, o_acc = [], 0
+        for _ in range(rounds):
+            em, na, lt = O.draft_and_verify(cfg, W, kv_o, lt, block, K, O.MODE_IDN)
+            o_got += em
+            o_acc += na
+        assert o_got == got and o_acc == accepted
+    # K = L: the drafter is exact, every draft is accepted
+    kv2 = m.kv_cache(1, 96)
+    last2 = m.prefill(kv2, dev(ids_np)).clone()
+    emitted, n_acc = m.draft_and_verify(kv2, last2, block, cfg.n_layer, O.MODE_IDN)
+    assert n_acc == block and emitted == want[:block + 1]
+
+
+def test_decode_graphs_do_not_change_results():
+    cfg = BF16
+    W = weights(cfg)
+    ids = dev(synth.make_ids(cfg, 1, 70, seed=8))   # decode crosses the 64-key chunk boundary at 128? no: 70 -> 80
+    outs = []
+    for use_graphs in (1, 0):
+        m = make_model(cfg, W, max_rows=70, max_batch=1, max_ctx=160)
+        m.set_flag(0, use_graphs)
+        kv = m.kv_cache(1, 160)
+        t = m.prefill(kv, ids)
+        seq = []
+        for _ in range(70):   # positions 70 .. 139: crosses a chunk boundary at 128
+            t = m.decode_step(kv, t, 2)
+            seq.append(t.clone())
+        outs.append(torch.stack(seq))
+        assert m.launch_count() > 0
+    assert torch.equal(outs[0], outs[1])
+
+
+def test_kv_truncate_rewinds_decoding():
+    cfg = F32
+    W = weights(cfg)
+    m = make_model(cfg, W, max_rows=8, max_batch=1, max_ctx=32)
+    kv = m.kv_cache(1, 32)
+    t0 = m.prefill(kv, dev(synth.make_ids(cfg, 1, 8, seed=9)))
+    a = [m.decode_step(kv, t0, 0).clone()]
+    a.append(m.decode_step(kv, a[-1], 0).clone())
+    kv.truncate(8)
+    assert len(kv) == 8
+    b = [m.decode_step(kv, t0, 0).clone()]
+    b.append(m.decode_step(kv, b[-1], 0).clone())
+    assert torch.equal(torch.stack(a), torch.stack(b))
