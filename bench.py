@@ -1,0 +1,388 @@
+#!/usr/bin/env python
+"""Benchmark of the SNLP hot path: greedy decoding with the layer-parallel Newton sweep on the
+d20 (~0.5B) Nanochat-shaped model, random-init bf16 weights, KV cache of 2048 random-prefill tokens.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--quick]
+
+A "step" is one decode step of the whole path: embed -> K_sweeps x (all 20 blocks evaluated at once
+on the current trace + IDN correction along the layer axis + residual norms) -> LM head + argmax.
+`value` is tokens/s of SNLP(K=2) IDN decoding at batch 1 (inputs resident on the device); the same
+line also carries the library's own sequential decode and the other (B, K) points, the roofline of
+the dominant kernel, the whole-sweep HBM fraction, and the CPU oracle timed on the host cores.
+With N > 1 (torchrun) every rank runs an independent replica (the path does not shard).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+CTX = 2048          # random-prefill tokens in the cache before decoding starts
+K_MAIN = 2          # sweeps of the headline configuration
+WORKLOAD = "d20 decode: L20 d1280 H10x128 ff5120 V65536 bf16, KV cache of 2048 random-prefill tokens, greedy"
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+    return 6650.0, "fallback (6.65 TB/s)"
+
+
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.path = f"/tmp/snlp_bench_clocks_{os.getpid()}.csv"
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        try:
+            os.remove(self.path)
+        except OSError:
+            pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def d20():
+    from paper_2605_17842_b200 import synth
+    return synth.CONFIGS["d20"]
+
+
+def alg_bytes(cfg, B, ctx):
+    """Algorithmic HBM bytes (bf16): weights per sweep, KV per sweep, lm head per step."""
+    L, d, ff, V = cfg.n_layer, cfg.d_model, cfg.d_ff, cfg.vocab
+    w = {"qkv": L * 3 * d * d * 2, "out_proj": L * d * d * 2, "mlp_up": L * d * ff * 2, "mlp_down": L * d * ff * 2}
+    kv = L * B * 2 * ctx * d * 2
+    return w, kv, V * d * 2
+
+
+# ----------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2605_17842_b200 import build
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if rank == 0:
+        build.build()
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    from paper_2605_17842_b200 import snlp, synth
+
+    cfg = d20()
+    steps, warmup = args.steps, max(args.warmup, 3)
+    extra_steps = 32 if args.quick else 64
+    W = synth.make_weights(cfg, seed=1234)
+    max_ctx = CTX + warmup + max(steps, extra_steps) + 8
+    model = snlp.Model(cfg, max_rows=512 if args.only_main else 2048, max_batch=8, max_ctx=max_ctx)
+    model.load_weights(W)
+    stream = torch.cuda.Stream()
+    hbm_peak, peak_src = peaks()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed_decode(kv, first_tok, K, n_warm, n_steps):
+        """n_warm untimed + n_steps timed decode steps from a cache truncated to CTX.  Returns ms/step."""
+        kv.truncate(CTX)
+        tok = first_tok.clone()
+        for _ in range(n_warm):
+            model.decode_step(kv, tok, K, snlp.MODE_IDN, tok_out=tok)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n_steps):
+            model.decode_step(kv, tok, K, snlp.MODE_IDN, tok_out=tok)
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms / n_steps
+
+    results = {}
+    with torch.cuda.stream(stream):
+        caches = {}
+        for B in (1, 8):
+            if B == 8 and (args.quick or args.only_main):
+                continue
+            ids = torch.from_numpy(synth.make_ids(cfg, B, CTX, seed=3)).cuda()
+            kv = model.kv_cache(B, max_ctx)
+            first = model.prefill(kv, ids)
+            torch.cuda.synchronize()
+            caches[B] = (kv, first)
+
+        # ---- headline: SNLP(K=2) IDN, batch 1 ------------------------------------------------
+        kv, first = caches[1]
+        sampler = ClockSampler(local)
+        timed_decode(kv, first, K_MAIN, warmup, steps)  # untimed pass: CUDA graphs are captured here
+        sampler.start()
+        l0 = model.launch_count()
+        ms_main = timed_decode(kv, first, K_MAIN, warmup, steps)
+        launches = model.launch_count() - l0
+        clocks = sampler.stop()
+        launches_timed = int(round(launches * steps / (steps + warmup)))
+        results[(1, K_MAIN)] = ms_main
+
+        if args.only_main:
+            if rank == 0:
+                print(json.dumps({"metric": "d20 decode tokens/s SNLP(K) vs sequential; sweep HBM GB/s vs B200 peak",
+                                  "value": world * 1e3 / ms_main, "unit": "tokens/s", "ms_per_step": ms_main,
+                                  "steps": steps, "warmup": warmup, "note": "--only-main: headline point only"}))
+            return
+
+        # ---- the other points (fewer steps each) ---------------------------------------------
+        for B, (kv, first) in caches.items():
+            for K in (0, 2, 4, 8):
+                if (B, K) in results:
+                    continue
+                results[(B, K)] = timed_decode(kv, first, K, warmup, extra_steps)
+
+        # ---- end to end through the public call with HOST buffers ----------------------------
+        kv, first = caches[1]
+        kv.truncate(CTX)
+        host_in = torch.empty((1,), dtype=torch.int32).pin_memory()
+        host_out = torch.empty((1,), dtype=torch.int32).pin_memory()
+        host_in.copy_(first.cpu())
+        dev_tok = torch.empty((1,), dtype=torch.int32, device="cuda")
+        e2e_steps = min(steps, 128)
+
+        def e2e_step():
+            dev_tok.copy_(host_in, non_blocking=True)
+            model.decode_step(kv, dev_tok, K_MAIN, snlp.MODE_IDN, tok_out=dev_tok)
+            host_out.copy_(dev_tok, non_blocking=True)
+            stream.synchronize()
+            host_in.copy_(host_out)
+
+        for _ in range(warmup):
+            e2e_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        ms_e2e = e0.elapsed_time(e1) / e2e_steps
+        if world > 1:
+            t = torch.tensor([ms_e2e], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+
+        # ---- per-kernel device time (CUDA events inside the library, on its launch stream) ----
+        model.set_flag(2, 1)
+        kv.truncate(CTX)
+        tok = first.clone()
+        for _ in range(4):
+            model.decode_step(kv, tok, K_MAIN, snlp.MODE_IDN, tok_out=tok)
+        torch.cuda.synchronize()
+        model.kernel_times(reset=True)
+        n_prof = 32
+        for _ in range(n_prof):
+            model.decode_step(kv, tok, K_MAIN, snlp.MODE_IDN, tok_out=tok)
+        torch.cuda.synchronize()
+        ktimes = model.kernel_times(reset=True)
+        model.set_flag(2, 0)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    ctx_mid = CTX + warmup + steps / 2.0
+    wbytes, kvbytes, lmbytes = alg_bytes(cfg, 1, ctx_mid)
+    sweep_bytes = sum(wbytes.values()) + kvbytes
+    step_bytes = K_MAIN * sweep_bytes + lmbytes
+    # dominant kernel: the class with the largest summed device time
+    per_class = {k: {"ms_per_launch": (v[0] / v[1] if v[1] else None), "launches_per_step": v[1] / n_prof,
+                     "ms_per_step": v[0] / n_prof} for k, v in ktimes.items()}
+    cls_bytes = dict(wbytes)
+    cls_bytes["attention"] = alg_bytes(cfg, 1, CTX + 4 + n_prof / 2.0)[1]
+    cls_bytes["lm_head"] = lmbytes
+    gemv = [k for k in ("qkv", "out_proj", "mlp_up", "mlp_down")]
+    dom = max(gemv, key=lambda k: ktimes[k][0])
+    dom_ms = ktimes[dom][0] / ktimes[dom][1]
+    achieved = cls_bytes[dom] / (dom_ms * 1e-3) / 1e9
+    for k in per_class:
+        if k in cls_bytes and per_class[k]["ms_per_launch"]:
+            lp = per_class[k]["launches_per_step"] / K_MAIN if k != "lm_head" else per_class[k]["launches_per_step"]
+            # attention = 2 launches per sweep (split + combine): bytes are per sweep
+            ms_sweep = per_class[k]["ms_per_step"] / (K_MAIN if k != "lm_head" else 1)
+            per_class[k]["alg_GBs"] = cls_bytes[k] / (ms_sweep * 1e-3) / 1e9
+            per_class[k]["frac_of_hbm_peak"] = per_class[k]["alg_GBs"] / hbm_peak
+    step_gbs = step_bytes / (ms_main * 1e-3) / 1e9
+
+    def toks(B, K):
+        return B * 1e3 / results[(B, K)] if (B, K) in results else None
+
+    table = {}
+    for (B, K), ms in sorted(results.items()):
+        table[f"B{B}_" + ("seq" if K == 0 else f"K{K}")] = {"ms_per_step": ms, "tok_s": world * B * 1e3 / ms}
+    speedups = {f"B{B}_K{K}": results[(B, 0)] / results[(B, K)] for (B, K) in results if K > 0 and (B, 0) in results}
+
+    cpu = cpu_baseline_sample(cfg, W, seconds=8.0 if args.quick else 20.0)
+
+    line = {
+        "metric": "d20 decode tokens/s SNLP(K) vs sequential; sweep HBM GB/s vs B200 peak",
+        "value": world * 1e3 / ms_main,
+        "unit": "tokens/s",
+        "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms_main,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "point": f"SNLP IDN K={K_MAIN}, batch 1 per GPU", "parallelism": "replicas only",
+                   "l2": "no flush: each step streams 2.2 GB of weights + KV (> 126 MB L2)"},
+        "clocks": clocks,
+        "e2e": {"value": world * 1e3 / ms_e2e, "unit": "tokens/s", "h2d_bytes_per_step": 4, "d2h_bytes_per_step": 4,
+                "steps": e2e_steps, "note": "host token in pinned memory -> H2D, snlp_decode_step, D2H, stream sync, every step"},
+        "gpu_launches": launches_timed,
+        "roofline": {"bound": "hbm", "kernel": f"k_gemv_mma ({dom}, all 20 layers in one launch)", "achieved": achieved,
+                     "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak, "peak_source": peak_src,
+                     "traffic": NCU_TRAFFIC_BYTES.get(dom), "alg_bytes_per_launch": cls_bytes[dom],
+                     "ms_per_launch": dom_ms},
+        "sweep": {"alg_bytes_per_step": step_bytes, "achieved_GBs": step_gbs, "frac_of_hbm_peak": step_gbs / hbm_peak,
+                  "target_frac": 0.70, "note": "whole decode step (K sweeps + lm head) under CUDA-graph replay"},
+        "kernels": per_class,
+        "decode": table,
+        "speedup_vs_own_sequential": speedups,
+        "paper_context": "paper reports only relative speed-ups on H100 (up to 2.58x, 1.40x without PPL increase, 0.5B models)",
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under profiles/
+NCU_TRAFFIC_BYTES: dict = {}
+
+
+# ----------------------------------------------------------------------------------------------
+def oracle_decode_setup(cfg, W):
+    """The oracle's d20 decode state: a cache whose 2048 slots hold seeded random unit-RMS keys and
+    N(0,1)-scaled values (cost-equivalent stand-in for a 1.6 TFLOP fp64 prefill on the host)."""
+    from oracle import snlp_oracle as O
+    kv = O.LayerKV(cfg.n_layer, 1, CTX + 64, cfg.n_head, cfg.head_dim)
+    rng = np.random.Generator(np.random.Philox(11))
+    kv.k[:, :, :CTX] = rng.standard_normal(kv.k[:, :, :CTX].shape)
+    kv.v[:, :, :CTX] = 0.3 * rng.standard_normal(kv.v[:, :, :CTX].shape)
+    kv.len = CTX
+    return kv
+
+
+def cpu_baseline_sample(cfg, W, seconds):
+    from oracle import snlp_oracle as O
+    kv = oracle_decode_setup(cfg, W)
+    tok = np.array([17], dtype=np.int32)
+    n, t0 = 0, time.perf_counter()
+    while True:
+        tok, _ = O.decode_step(cfg, W, kv, tok, K_MAIN, O.MODE_IDN)
+        n += 1
+        dt = time.perf_counter() - t0
+        if dt >= seconds or n >= 32:
+            break
+    return {"value": n / dt, "unit": "tokens/s", "cores": os.cpu_count(), "kind": "oracle",
+            "sample": f"{n} greedy decode steps of the numpy fp64 oracle, IDN K={K_MAIN}, batch 1, d20, cache of {CTX} "
+                      f"seeded random keys/values (no prefill), {dt:.1f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import snlp_oracle as O
+    from paper_2605_17842_b200 import synth
+    cfg = d20()
+    W = synth.make_weights(cfg, seed=1234)
+    kv = oracle_decode_setup(cfg, W)
+    tok = np.array([17], dtype=np.int32)
+    warm = min(max(args.warmup, 1), 2)
+    for _ in range(warm):
+        tok, _ = O.decode_step(cfg, W, kv, tok, K_MAIN, O.MODE_IDN)
+    budget = 150.0
+    n, t0 = 0, time.perf_counter()
+    while n < args.steps:
+        tok, _ = O.decode_step(cfg, W, kv, tok, K_MAIN, O.MODE_IDN)
+        n += 1
+        if time.perf_counter() - t0 > budget:
+            break
+    dt = time.perf_counter() - t0
+    val = n / dt
+    sample = (f"{n} whole decode steps of the numpy fp64 oracle (IDN K={K_MAIN}, batch 1, d20, cache of {CTX} seeded random "
+              f"keys/values); the run stops after {budget:.0f} s, so fewer than --steps may be timed")
+    line = {"impl": "reference", "metric": "d20 decode tokens/s SNLP(K) vs sequential; sweep HBM GB/s vs B200 peak",
+            "value": val, "unit": "tokens/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": n, "warmup": warm,
+            "ms_per_step": 1e3 * dt / n, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": WORKLOAD, "point": f"SNLP IDN K={K_MAIN}, batch 1"},
+            "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": os.cpu_count(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=16)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--quick", action="store_true", help="batch 1 only, shorter side measurements")
+    ap.add_argument("--only-main", action="store_true",
+                    help="headline point only, small workspace: the light command used for ncu captures")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -158,8 +158,17 @@ int snlp_draft_and_verify(snlp_model *m, snlp_kv *kv, int32_t *last_tok, int blo
                           int32_t *emitted, int32_t *n_emitted, int32_t *n_accepted, void *stream);
 
 /* Tuning / introspection (no effect on results).  flag 0: use CUDA graphs for decode steps (default 1).
- * flag 1: force the generic SIMT kernels even where a specialised kernel exists (default 0; testing). */
+ * flag 1: force the generic SIMT kernels even where a specialised kernel exists (default 0; testing).
+ * flag 2: time every launch with CUDA events on its stream, accumulated per kernel class (default 0;
+ *         while on, decode steps are launched directly instead of replaying graphs). */
 int snlp_set_flag(snlp_model *m, int flag, int value);
+
+/* Kernel classes of snlp_kernel_times, in order: QKV projection, attention, out-projection, MLP up,
+ * MLP down, correction, lm head (+argmax), everything else (embed, casts, bookkeeping). */
+#define SNLP_NUM_KERNEL_CLASSES 8
+/* Waits for the timed launches recorded so far and returns, per class, the summed device time in
+ * milliseconds (host double[8]) and the number of launches (host int64[8]); reset != 0 clears them. */
+int snlp_kernel_times(snlp_model *m, double *ms, int64_t *launches, int reset);
 /* Number of kernel launches this handle has enqueued since creation (graph replays count their nodes). */
 int snlp_launch_count(const snlp_model *m, int64_t *count);
 

@@ -142,4 +142,129 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
   if (threadIdx.x == 0) *p.counter = 0u;
 }
 
+
+// Latency-oriented variant for the decode regime (a handful of rows): the per-thread loop over
+// layers above serialises ~7 dependent-latency loads per layer, which dominates when there are too
+// few threads to hide it.  Here a block owns 32 float4 columns of one row; its 8 warps first fetch
+// every layer's branch outputs and old states in parallel into shared memory, then warp 0 runs the
+// serial recurrence out of shared memory.  Same arithmetic, same summation order as k_correct.
+// grid (d/128, M), 256 threads; dynamic shared memory nl*32*(2+NS) float4 + nl*2 floats.
+template <int NS>
+__global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
+  extern __shared__ float4 s_buf[];
+  const int d4 = p.d >> 2;
+  const int c = threadIdx.x & 31, ll = threadIdx.x >> 5;
+  const int c4 = blockIdx.x * 32 + c;
+  const size_t row = blockIdx.y;
+  const bool active = c4 < d4;
+  const size_t Md4 = (size_t)p.M * d4, state4 = Md4 * NS;
+  const float4 *a4 = reinterpret_cast<const float4 *>(p.a);
+  const float4 *m4 = reinterpret_cast<const float4 *>(p.m);
+  float4 *tr4 = reinterpret_cast<float4 *>(p.trace);
+  const size_t bm_off = row * d4 + c4, st_off = row * NS * d4 + c4;
+  float4 *sa = s_buf, *sm = s_buf + (size_t)p.nl * 32, *so = s_buf + (size_t)p.nl * 64;  // so: [nl][NS][32]
+  float *snorm = reinterpret_cast<float *>(s_buf + (size_t)p.nl * 32 * (2 + NS));
+  const bool want_norm = p.partial != nullptr;
+  if (active) {
+    for (int i = ll; i < p.nl; i += 8) {
+      const int l = p.l0 + i;
+      float4 av = a4[(size_t)l * Md4 + bm_off];
+      for (int q = 1; q < p.a_splits; ++q) av = f4_add(av, a4[(size_t)q * (p.a_ss >> 2) + (size_t)l * Md4 + bm_off]);
+      float4 mv = m4[(size_t)l * Md4 + bm_off];
+      for (int q = 1; q < p.m_splits; ++q) mv = f4_add(mv, m4[(size_t)q * (p.m_ss >> 2) + (size_t)l * Md4 + bm_off]);
+      sa[i * 32 + c] = av;
+      sm[i * 32 + c] = mv;
+#pragma unroll
+      for (int r = 0; r < NS; ++r) so[(i * NS + r) * 32 + c] = tr4[(size_t)(l + 1) * state4 + st_off + (size_t)r * d4];
+    }
+  }
+  __syncthreads();
+  if (ll != 0) return;
+  const bool native = (NS == 1) ? (p.mode != 2) : (p.mode == 1);
+  float4 oldp[NS], newp[NS];
+  if (active) {
+#pragma unroll
+    for (int s = 0; s < NS; ++s) oldp[s] = newp[s] = tr4[(size_t)p.l0 * state4 + st_off + (size_t)s * d4];
+  }
+  for (int i = 0; i < p.nl; ++i) {
+    const int l = p.l0 + i;
+    float rs = 0.f, hs = 0.f;
+    if (active) {
+      const float4 av = sa[i * 32 + c], mv = sm[i * 32 + c];
+      const HcCoef &cf = p.coef[l];
+      float4 oldn[NS], newn[NS], tilde[NS];
+#pragma unroll
+      for (int r = 0; r < NS; ++r) {
+        oldn[r] = so[(i * NS + r) * 32 + c];
+        if (NS == 1) {
+          tilde[r] = f4_add(f4_add(oldp[0], av), mv);
+        } else {
+          float4 t = f4_scale(cf.A[r * NS], oldp[0]);
+#pragma unroll
+          for (int s = 1; s < NS; ++s) t = f4_fma(cf.A[r * NS + s], oldp[s], t);
+          tilde[r] = f4_fma(cf.cm[r], mv, f4_fma(cf.ca[r], av, t));
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < NS; ++r) {
+        if (p.mode == 2) {
+          newn[r] = tilde[r];
+        } else if (native) {
+          if (NS == 1) {
+            newn[r] = f4_add(f4_add(newp[0], av), mv);
+          } else {
+            float4 t = f4_scale(cf.A[r * NS], newp[0]);
+#pragma unroll
+            for (int s = 1; s < NS; ++s) t = f4_fma(cf.A[r * NS + s], newp[s], t);
+            newn[r] = f4_fma(cf.cm[r], mv, f4_fma(cf.ca[r], av, t));
+          }
+        } else {
+          newn[r] = f4_add(tilde[r], f4_sub(newp[r], oldp[r]));
+        }
+        const float4 rr = f4_sub(tilde[r], oldn[r]);
+        rs += f4_sq(rr);
+        hs += f4_sq(oldn[r]);
+        tr4[(size_t)(l + 1) * state4 + st_off + (size_t)r * d4] = newn[r];
+      }
+      if (NS > 1 && l + 1 < p.L) {
+        const HcCoef &cn = p.coef[l + 1];
+        float4 xa = f4_scale(cn.pa[0], newn[0]), xm = f4_scale(cn.pmra[0], newn[0]);
+#pragma unroll
+        for (int s = 1; s < NS; ++s) {
+          xa = f4_fma(cn.pa[s], newn[s], xa);
+          xm = f4_fma(cn.pmra[s], newn[s], xm);
+        }
+        reinterpret_cast<float4 *>(p.xa)[(size_t)(l + 1) * Md4 + bm_off] = xa;
+        reinterpret_cast<float4 *>(p.xm)[(size_t)(l + 1) * Md4 + bm_off] = xm;
+      }
+#pragma unroll
+      for (int r = 0; r < NS; ++r) { oldp[r] = oldn[r]; newp[r] = newn[r]; }
+    }
+    if (want_norm) {
+      rs = warp_sum(rs);
+      hs = warp_sum(hs);
+      if (c == 0) { snorm[i * 2] = rs; snorm[i * 2 + 1] = hs; }
+    }
+  }
+  if (!want_norm) return;
+  // warp 0 only from here on
+  __syncwarp();
+  const unsigned nblk = gridDim.x * gridDim.y, blk = blockIdx.y * gridDim.x + blockIdx.x;
+  for (int i = c; i < p.nl * 2; i += 32) p.partial[(size_t)blk * p.nl * 2 + i] = snorm[i];
+  __threadfence();
+  __syncwarp();
+  unsigned ticket = 0;
+  if (c == 0) ticket = atomicAdd(p.counter, 1u);
+  ticket = __shfl_sync(0xffffffffu, ticket, 0);
+  if (ticket != nblk - 1) return;
+  __threadfence();
+  for (int i = c; i < p.nl * 2; i += 32) {
+    double s = 0.0;
+    for (unsigned b = 0; b < nblk; ++b) s += (double)__ldcg(&p.partial[(size_t)b * p.nl * 2 + i]);
+    p.resnorm[(size_t)p.l0 * 2 + i] = (float)s;
+  }
+  __syncwarp();
+  if (c == 0) *p.counter = 0u;
+}
+
 }  // namespace snlp

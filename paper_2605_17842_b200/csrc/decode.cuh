@@ -254,24 +254,30 @@ __global__ void k_argmax_tiles(const float *__restrict__ pm_val, const int *__re
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Split-KV causal attention for <= 16 query rows per sequence.  A CTA owns one chunk of C consecutive
-// key positions of one (layer, sequence, head); its 8 half-warps take interleaved keys, every lane
-// holds 8 of the 128 head features (one 16-byte load per key row).  The chunk boundaries are fixed
-// multiples of C and a query's result never depends on the other queries in the call.
+// Split-KV causal attention for <= 16 query rows per sequence.  A CTA owns one chunk of `csub` x 64
+// consecutive key positions of one (layer, sequence, head) and walks it in 64-key sub-blocks with an
+// online softmax; its 8 half-warps take interleaved keys and every lane holds 8 of the 128 head
+// features (one 16-byte load per key row, K and V of a sub-block issued together).  The last CTA of a
+// (layer, sequence, head) to finish merges the chunk partials in chunk order and writes the bf16
+// output, so no second launch is needed; arrival order does not change the result.  Chunk boundaries
+// are fixed multiples of the chunk length and a query's result never depends on the other queries in
+// the call (batch invariance: a T = 1 decode step and a T = 9 verify block give identical rows).
 // part: [(l*BH + bh)*Tq + t][nchunk][132] = 128 un-normalised outputs, running max, denominator.
 constexpr int kAttnPartStride = 132;
+constexpr int kAttnSub = 64;
 
-template <int C>
-__global__ void __launch_bounds__(128) k_attn_decode(const __nv_bfloat16 *__restrict__ q, size_t q_ls,
-                                                     const __nv_bfloat16 *__restrict__ kc, const __nv_bfloat16 *__restrict__ vc,
-                                                     size_t kv_ls, size_t kv_bs, float *__restrict__ part, int Tq, int H,
-                                                     const int *__restrict__ pos_base) {
+__global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat16 *__restrict__ q, size_t q_ls,
+                                                        const __nv_bfloat16 *__restrict__ kc, const __nv_bfloat16 *__restrict__ vc,
+                                                        size_t kv_ls, size_t kv_bs, float *__restrict__ part,
+                                                        unsigned *__restrict__ counters, __nv_bfloat16 *__restrict__ out,
+                                                        size_t o_ls, int Tq, int H, const int *__restrict__ pos_base, int csub) {
   __shared__ float qs[16][128];
   __shared__ float hacc[8][128];
   __shared__ float hm[8], hl[8];
+  __shared__ bool s_last;
   const int chunk = blockIdx.x, nchunk = gridDim.x, bh = blockIdx.y, l = blockIdx.z;
   const int b = bh / H, h = bh % H, d = H * 128;
-  const int pos0 = *pos_base, key0 = chunk * C;
+  const int pos0 = *pos_base, kbeg = chunk * csub * kAttnSub;
   const int tid = threadIdx.x, hw = tid >> 4, li = tid & 15;
   const float scale = 0.08838834764831845f;  // 1/sqrt(128)
   for (int i = tid; i < Tq * 128; i += 128) {
@@ -281,11 +287,12 @@ __global__ void __launch_bounds__(128) k_attn_decode(const __nv_bfloat16 *__rest
   __syncthreads();
   const __nv_bfloat16 *kp = kc + (size_t)l * kv_ls + (size_t)b * kv_bs + h * 128 + li * 8;
   const __nv_bfloat16 *vp = vc + (size_t)l * kv_ls + (size_t)b * kv_bs + h * 128 + li * 8;
-  constexpr int J = C / 8;
+  float *pbase = part + (size_t)((size_t)l * gridDim.y + bh) * Tq * nchunk * kAttnPartStride;
+  constexpr int J = kAttnSub / 8;
   for (int t = 0; t < Tq; ++t) {
     const int pos_q = pos0 + t;
-    float *dst = part + ((size_t)((size_t)l * gridDim.y + bh) * Tq + t) * nchunk * kAttnPartStride + (size_t)chunk * kAttnPartStride;
-    if (key0 > pos_q) {  // whole chunk is in this query's future
+    float *dst = pbase + ((size_t)t * nchunk + chunk) * kAttnPartStride;
+    if (kbeg > pos_q) {  // whole chunk is in this query's future
       dst[tid] = 0.f;
       if (tid == 0) { dst[128] = -INFINITY; dst[129] = 0.f; }
       continue;
@@ -293,55 +300,62 @@ __global__ void __launch_bounds__(128) k_attn_decode(const __nv_bfloat16 *__rest
     float qv[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) qv[i] = qs[t][li * 8 + i];
-    uint4 kr[J];
-#pragma unroll
-    for (int j = 0; j < J; ++j) {
-      const int key = key0 + hw + 8 * j;
-      kr[j] = key <= pos_q ? ldg_stream(kp + (size_t)key * d) : make_uint4(0, 0, 0, 0);
-    }
-    float s[J];
-    float mloc = -INFINITY;
-#pragma unroll
-    for (int j = 0; j < J; ++j) {
-      const int key = key0 + hw + 8 * j;
-      const __nv_bfloat162 *k2 = reinterpret_cast<const __nv_bfloat162 *>(&kr[j]);
-      float dot = 0.f;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float2 f = __bfloat1622float2(k2[i]);
-        dot = fmaf(qv[2 * i], f.x, dot);
-        dot = fmaf(qv[2 * i + 1], f.y, dot);
-      }
-      dot += __shfl_xor_sync(0xffffffffu, dot, 8);
-      dot += __shfl_xor_sync(0xffffffffu, dot, 4);
-      dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-      dot += __shfl_xor_sync(0xffffffffu, dot, 1);
-      s[j] = key <= pos_q ? dot : -INFINITY;
-      mloc = fmaxf(mloc, s[j]);
-    }
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    float lsum = 0.f;
-    uint4 vr[J];
+    float mrun = -INFINITY, lrun = 0.f;
+    for (int sb = 0; sb < csub; ++sb) {
+      const int base = kbeg + sb * kAttnSub;
+      if (base > pos_q) break;
+      uint4 kr[J], vr[J];
 #pragma unroll
-    for (int j = 0; j < J; ++j) {
-      const int key = key0 + hw + 8 * j;
-      vr[j] = key <= pos_q ? ldg_stream(vp + (size_t)key * d) : make_uint4(0, 0, 0, 0);
-    }
-#pragma unroll
-    for (int j = 0; j < J; ++j) {
-      const float pj = s[j] == -INFINITY ? 0.f : __expf(s[j] - mloc);
-      lsum += pj;
-      const __nv_bfloat162 *v2 = reinterpret_cast<const __nv_bfloat162 *>(&vr[j]);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float2 f = __bfloat1622float2(v2[i]);
-        acc[2 * i] = fmaf(pj, f.x, acc[2 * i]);
-        acc[2 * i + 1] = fmaf(pj, f.y, acc[2 * i + 1]);
+      for (int j = 0; j < J; ++j) {
+        const int key = base + hw + 8 * j;
+        const bool ok = key <= pos_q;
+        kr[j] = ok ? ldg_stream(kp + (size_t)key * d) : make_uint4(0, 0, 0, 0);
+        vr[j] = ok ? ldg_stream(vp + (size_t)key * d) : make_uint4(0, 0, 0, 0);
       }
+      float s[J];
+      float mloc = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < J; ++j) {
+        const int key = base + hw + 8 * j;
+        const __nv_bfloat162 *k2 = reinterpret_cast<const __nv_bfloat162 *>(&kr[j]);
+        float dot = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 f = __bfloat1622float2(k2[i]);
+          dot = fmaf(qv[2 * i], f.x, dot);
+          dot = fmaf(qv[2 * i + 1], f.y, dot);
+        }
+        dot += __shfl_xor_sync(0xffffffffu, dot, 8);
+        dot += __shfl_xor_sync(0xffffffffu, dot, 4);
+        dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+        dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+        s[j] = key <= pos_q ? dot : -INFINITY;
+        mloc = fmaxf(mloc, s[j]);
+      }
+      if (mloc == -INFINITY) continue;  // none of this half-warp's keys of the sub-block is visible
+      const float mnew = fmaxf(mrun, mloc);
+      const float resc = mrun == -INFINITY ? 0.f : __expf(mrun - mnew);
+      lrun *= resc;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] *= resc;
+#pragma unroll
+      for (int j = 0; j < J; ++j) {
+        const float pj = s[j] == -INFINITY ? 0.f : __expf(s[j] - mnew);
+        lrun += pj;
+        const __nv_bfloat162 *v2 = reinterpret_cast<const __nv_bfloat162 *>(&vr[j]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 f = __bfloat1622float2(v2[i]);
+          acc[2 * i] = fmaf(pj, f.x, acc[2 * i]);
+          acc[2 * i + 1] = fmaf(pj, f.y, acc[2 * i + 1]);
+        }
+      }
+      mrun = mnew;
     }
 #pragma unroll
     for (int i = 0; i < 8; ++i) hacc[hw][li * 8 + i] = acc[i];
-    if (li == 0) { hm[hw] = mloc; hl[hw] = lsum; }
+    if (li == 0) { hm[hw] = mrun; hl[hw] = lrun; }
     __syncthreads();
     {  // merge the 8 half-warps in index order
       float M = hm[0];
@@ -359,25 +373,27 @@ __global__ void __launch_bounds__(128) k_attn_decode(const __nv_bfloat16 *__rest
     }
     __syncthreads();
   }
-}
-
-// Merge the chunk partials of one (layer, row, head) in chunk order.  grid (rows*H, nl), 128 threads.
-__global__ void __launch_bounds__(128) k_attn_combine(const float *__restrict__ part, int nchunk, int Tq, int H,
-                                                      __nv_bfloat16 *__restrict__ out, size_t o_ls) {
-  const int rh = blockIdx.x, l = blockIdx.y;
-  const int row = rh / H, h = rh % H, b = row / Tq, t = row % Tq, BH = (gridDim.x / (H * Tq)) * H;
-  const float *src = part + ((size_t)((size_t)l * BH + b * H + h) * Tq + t) * nchunk * kAttnPartStride;
-  float M = -INFINITY;
-  for (int c = 0; c < nchunk; ++c) M = fmaxf(M, src[(size_t)c * kAttnPartStride + 128]);
-  float o = 0.f, den = 0.f;
-  for (int c = 0; c < nchunk; ++c) {
-    const float mc = src[(size_t)c * kAttnPartStride + 128];
-    if (mc == -INFINITY) continue;
-    const float w = __expf(mc - M);
-    o = fmaf(w, src[(size_t)c * kAttnPartStride + threadIdx.x], o);
-    den = fmaf(w, src[(size_t)c * kAttnPartStride + 129], den);
+  // ---- last CTA of this (layer, sequence, head) merges the chunks in chunk order --------------------
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = atomicAdd(&counters[(size_t)l * gridDim.y + bh], 1u) == (unsigned)nchunk - 1;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  for (int t = 0; t < Tq; ++t) {
+    const float *src = pbase + (size_t)t * nchunk * kAttnPartStride;
+    float M = -INFINITY;
+    for (int c = 0; c < nchunk; ++c) M = fmaxf(M, __ldcg(src + (size_t)c * kAttnPartStride + 128));
+    float o = 0.f, den = 0.f;
+    for (int c = 0; c < nchunk; ++c) {
+      const float mc = __ldcg(src + (size_t)c * kAttnPartStride + 128);
+      const float w = mc == -INFINITY ? 0.f : __expf(mc - M);
+      o = fmaf(w, __ldcg(src + (size_t)c * kAttnPartStride + tid), o);
+      den = fmaf(w, __ldcg(src + (size_t)c * kAttnPartStride + 129), den);
+    }
+    out[(size_t)l * o_ls + (size_t)(b * Tq + t) * d + h * 128 + tid] = __float2bfloat16_rn(o / den);
   }
-  out[(size_t)l * o_ls + (size_t)row * (H * 128) + h * 128 + threadIdx.x] = __float2bfloat16_rn(o / den);
+  if (tid == 0) counters[(size_t)l * gridDim.y + bh] = 0u;
 }
 
 }  // namespace snlp

@@ -49,10 +49,10 @@ extern "C" const char *snlp_last_error(void) { return g_err.c_str(); }
 
 // ------------------------------------------------------------------------------------------------
 // handles
-constexpr int kAttnChunk = 64;   // key positions per split-KV chunk
 constexpr int kMaxSplits = 4;    // K-splits of the partial-sum GEMV outputs
 constexpr int kDecodeRows = 16;  // largest row count served by the decode-regime kernels
 constexpr size_t kGemvMaxSmem = 200 * 1024;
+constexpr size_t kCorrSmallSmem = 160 * 1024;
 
 struct GraphKey {
   int B, K, mode, nchunk;
@@ -63,6 +63,9 @@ struct GraphKey {
   }
 };
 struct GraphEntry { cudaGraphExec_t exec; int64_t nodes; };
+struct PendingTime { int cls; cudaEvent_t e0, e1; };
+enum { KC_QKV = 0, KC_ATTN, KC_OPROJ, KC_UP, KC_DOWN, KC_CORRECT, KC_LMHEAD, KC_OTHER, KC_COUNT };
+static_assert(KC_COUNT == SNLP_NUM_KERNEL_CLASSES, "kernel class count");
 
 struct snlp_model {
   snlp_config cfg{};
@@ -78,13 +81,17 @@ struct snlp_model {
   void *xn = nullptr, *q = nullptr, *att = nullptr, *z = nullptr, *sk = nullptr, *sv = nullptr, *xlm = nullptr;
   float *attn_part = nullptr, *corr_part = nullptr, *logits = nullptr, *pm_val = nullptr;
   int *pm_idx = nullptr;
-  unsigned *counter = nullptr;
+  unsigned *counter = nullptr, *attn_counters = nullptr;
   int *zero = nullptr;
   int32_t *spec = nullptr;  // [2 * (max_rows + 1)] ids / verifier tokens for draft-and-verify
   int logit_rows = 0;
   std::vector<void *> allocs;
   // flags / stats
-  int use_graphs = 1, force_generic = 0;
+  int use_graphs = 1, force_generic = 0, timing = 0;
+  std::vector<PendingTime> pending;
+  std::vector<cudaEvent_t> free_events;
+  double class_ms[KC_COUNT] = {};
+  int64_t class_launches[KC_COUNT] = {};
   int64_t launches = 0;
   bool capturing = false;
   int64_t cap_nodes = 0;
@@ -114,6 +121,41 @@ static inline void count(snlp_model *m, int n = 1) {
   else m->launches += n;
 }
 
+// Optional device timing of every launch, by kernel class (CUDA events on the launching stream).
+struct TimedLaunch {
+  snlp_model *m;
+  cudaStream_t st;
+  int cls;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  TimedLaunch(snlp_model *m_, cudaStream_t st_, int cls_) : m(m_), st(st_), cls(cls_) {
+    if (!m->timing || m->capturing || m->pending.size() >= 200000) return;
+    if (m->free_events.size() >= 2) {
+      e0 = m->free_events.back(); m->free_events.pop_back();
+      e1 = m->free_events.back(); m->free_events.pop_back();
+    } else if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) {
+      e0 = e1 = nullptr;
+      return;
+    }
+    cudaEventRecord(e0, st);
+  }
+  ~TimedLaunch() {
+    if (e0) {
+      cudaEventRecord(e1, st);
+      m->pending.push_back({cls, e0, e1});
+    }
+    count(m);
+  }
+};
+
+#define KLAUNCH(m, st, cls, ...)     \
+  do {                               \
+    {                                \
+      TimedLaunch tl_(m, st, cls);   \
+      __VA_ARGS__;                   \
+    }                                \
+    LAUNCH_CHECK();                  \
+  } while (0)
+
 #define LAUNCH_CHECK()                                                                              \
   do {                                                                                              \
     cudaError_t e_ = cudaGetLastError();                                                            \
@@ -135,6 +177,16 @@ static int dalloc(snlp_model *m, P **p, size_t bytes) {
 }
 
 static int init_kernel_attributes();
+
+// 64-key sub-blocks per split-KV chunk.  It depends only on how many (layer, sequence, head) triples one
+// launch covers (not on the context length or the number of query rows), so that calls of the same
+// geometry -- a decode step and the verifier block of self-speculative decoding -- merge their keys in the
+// same order.  Few triples (sequential execution, batch 1) get short chunks so the launch still fills the GPU.
+static int attn_csub(int triples) {
+  int c = 1;
+  while (c < 8 && triples >= 16 * c) c *= 2;
+  return c;
+}
 
 static bool fast_decode_ok(const snlp_model *m, int M) {
   const snlp_config &c = m->cfg;
@@ -192,7 +244,7 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
   A(&m->sk, L * R * d * es);
   A(&m->sv, L * R * d * es);
   A(&m->xlm, R * d * es);
-  const size_t nchunk_max = ((size_t)c.max_ctx + kAttnChunk - 1) / kAttnChunk;
+  const size_t nchunk_max = ((size_t)c.max_ctx + kAttnSub - 1) / kAttnSub;
   A(&m->attn_part, L * (size_t)kDecodeRows * c.n_head * nchunk_max * kAttnPartStride * 4);
   const size_t corr_blocks = (R * (d / 4) + 255) / 256;
   A(&m->corr_part, corr_blocks * L * 2 * 4);
@@ -201,10 +253,11 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
   A(&m->pm_val, (size_t)kDecodeRows * ((V + 127) / 128) * 4);
   A(&m->pm_idx, (size_t)kDecodeRows * ((V + 127) / 128) * 4);
   A(&m->counter, 16);
+  A(&m->attn_counters, L * (size_t)kDecodeRows * c.n_head * 4);
   A(&m->zero, 16);
   A(&m->spec, 2 * (R + 1) * 4);
   if (rc == SNLP_OK) {
-    if (cudaMemset(m->counter, 0, 16) != cudaSuccess || cudaMemset(m->zero, 0, 16) != cudaSuccess)
+    if (cudaMemset(m->attn_counters, 0, L * (size_t)kDecodeRows * c.n_head * 4) != cudaSuccess || cudaMemset(m->counter, 0, 16) != cudaSuccess || cudaMemset(m->zero, 0, 16) != cudaSuccess)
       rc = fail(SNLP_ERR_CUDA, "cudaMemset failed");
   }
   if (rc == SNLP_OK) {
@@ -236,6 +289,8 @@ extern "C" int snlp_destroy(snlp_model *m) {
   cudaDeviceSynchronize();
   for (auto &g : m->graphs) cudaGraphExecDestroy(g.second.exec);
   if (m->cap_stream) cudaStreamDestroy(m->cap_stream);
+  for (const PendingTime &t : m->pending) { cudaEventDestroy(t.e0); cudaEventDestroy(t.e1); }
+  for (cudaEvent_t e : m->free_events) cudaEventDestroy(e);
   for (void *p : m->allocs) cudaFree(p);
   delete m;
   return SNLP_OK;
@@ -295,7 +350,33 @@ extern "C" int snlp_set_flag(snlp_model *m, int flag, int value) {
   if (!m) return fail(SNLP_ERR_ARG, "snlp_set_flag: NULL handle");
   if (flag == 0) m->use_graphs = value != 0;
   else if (flag == 1) m->force_generic = value != 0;
+  else if (flag == 2) m->timing = value != 0;
   else return fail(SNLP_ERR_ARG, "snlp_set_flag: unknown flag %d", flag);
+  return SNLP_OK;
+}
+
+static int drain_times(snlp_model *m) {
+  for (const PendingTime &t : m->pending) {
+    CU(cudaEventSynchronize(t.e1));
+    float ms = 0.f;
+    CU(cudaEventElapsedTime(&ms, t.e0, t.e1));
+    m->class_ms[t.cls] += ms;
+    m->class_launches[t.cls] += 1;
+    m->free_events.push_back(t.e0);
+    m->free_events.push_back(t.e1);
+  }
+  m->pending.clear();
+  return SNLP_OK;
+}
+
+extern "C" int snlp_kernel_times(snlp_model *m, double *ms, int64_t *launches, int reset) {
+  if (!m || !ms || !launches) return fail(SNLP_ERR_ARG, "snlp_kernel_times: NULL argument");
+  TRY(drain_times(m));
+  for (int i = 0; i < KC_COUNT; ++i) {
+    ms[i] = m->class_ms[i];
+    launches[i] = m->class_launches[i];
+    if (reset) { m->class_ms[i] = 0.0; m->class_launches[i] = 0; }
+  }
   return SNLP_OK;
 }
 
@@ -308,12 +389,10 @@ extern "C" int snlp_launch_count(const snlp_model *m, int64_t *count_out) {
 // ------------------------------------------------------------------------------------------------
 // launch sequences
 template <typename T>
-static int gemm(snlp_model *m, cudaStream_t st, const T *A, size_t a_ls, const T *W, size_t w_ls, float *C, size_t c_ls, int M, int N,
-                int K, int nl) {
+static int gemm(snlp_model *m, cudaStream_t st, int cls, const T *A, size_t a_ls, const T *W, size_t w_ls, float *C, size_t c_ls, int M,
+                int N, int K, int nl) {
   dim3 grid((N + 63) / 64, (M + 63) / 64, nl);
-  k_gemm_nt<T><<<grid, 256, 0, st>>>(A, a_ls, W, w_ls, C, c_ls, M, N, K);
-  count(m);
-  LAUNCH_CHECK();
+  KLAUNCH(m, st, cls, k_gemm_nt<T><<<grid, 256, 0, st>>>(A, a_ls, W, w_ls, C, c_ls, M, N, K));
   return SNLP_OK;
 }
 
@@ -342,12 +421,23 @@ static int correct(snlp_model *m, const Fwd &f, int l0, int nl, int mode, int a_
   const int threads = 256;
   const unsigned blocks = (unsigned)((total + threads - 1) / threads);
   const size_t sm = resnorm ? (size_t)(threads / 32) * nl * 2 * sizeof(float) : 0;
-  switch (c.n_streams) {
-#define CASE(NS) case NS: k_correct<NS><<<blocks, threads, sm, f.st>>>(p); break;
-    CASE(1) CASE(2) CASE(3) CASE(4) CASE(5) CASE(6) CASE(7) CASE(8)
+  const size_t sm_small = (size_t)nl * 32 * (2 + c.n_streams) * sizeof(float4) + (size_t)nl * 2 * sizeof(float);
+  if (f.M <= kDecodeRows && c.n_streams <= 4 && sm_small <= kCorrSmallSmem) {
+    dim3 grid((c.d_model / 4 + 31) / 32, f.M);
+    TimedLaunch tl_(m, f.st, KC_CORRECT);
+    switch (c.n_streams) {
+#define CASE(NS) case NS: k_correct_small<NS><<<grid, 256, sm_small, f.st>>>(p); break;
+      CASE(1) CASE(2) CASE(3) CASE(4)
 #undef CASE
+    }
+  } else {
+    TimedLaunch tl_(m, f.st, KC_CORRECT);
+    switch (c.n_streams) {
+#define CASE(NS) case NS: k_correct<NS><<<blocks, threads, sm, f.st>>>(p); break;
+      CASE(1) CASE(2) CASE(3) CASE(4) CASE(5) CASE(6) CASE(7) CASE(8)
+#undef CASE
+    }
   }
-  count(m);
   LAUNCH_CHECK();
   return SNLP_OK;
 }
@@ -366,43 +456,31 @@ static int run_generic(snlp_model *m, const Fwd &f, int l0, int nl, int mode, fl
   float *qkv = m->qkv_raw + (size_t)l0 * M * 3 * d, *a = m->a + l0 * Md, *y = m->y_raw + (size_t)l0 * M * ff, *mb = m->mb + l0 * Md;
   T *kc = (T *)f.kc + (size_t)l0 * f.kv_ls, *vc = (T *)f.vc + (size_t)l0 * f.kv_ls;
 
-  k_rmsnorm_cast<T><<<dim3(M, nl), 256, 0, st>>>(xa_src, Md, (size_t)d, 1, xn, Md, d, c.rms_eps);
-  count(m);
-  LAUNCH_CHECK();
-  TRY(gemm<T>(m, st, xn, Md, (const T *)m->wqkv + (size_t)l0 * 3 * d * d, (size_t)3 * d * d, qkv, (size_t)M * 3 * d, M, 3 * d, d, nl));
-  k_rope_qknorm_store<T><<<dim3(M, 3 * H, nl), 128, 0, st>>>(qkv, (size_t)M * 3 * d, q, Md, kc, vc, f.kv_ls, f.kv_bs, f.T, H, hd, f.pos,
-                                                             m->rope, c.rms_eps);
-  count(m);
-  LAUNCH_CHECK();
-  k_attn_generic<T><<<dim3((M * H + 3) / 4, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, att, Md, M, f.T, H, hd, f.pos);
-  count(m);
-  LAUNCH_CHECK();
-  TRY(gemm<T>(m, st, att, Md, (const T *)m->wo + (size_t)l0 * d * d, (size_t)d * d, a, Md, M, d, d, nl));
-  k_resid_rmsnorm_cast<T><<<dim3(M, nl), 256, 0, st>>>(xm_src, Md, (size_t)d, a, Md, 1, 0, m->coef, l0, xn, Md, d, c.rms_eps);
-  count(m);
-  LAUNCH_CHECK();
-  TRY(gemm<T>(m, st, xn, Md, (const T *)m->wup + (size_t)l0 * ff * d, (size_t)ff * d, y, (size_t)M * ff, M, ff, d, nl));
+  KLAUNCH(m, st, KC_OTHER, k_rmsnorm_cast<T><<<dim3(M, nl), 256, 0, st>>>(xa_src, Md, (size_t)d, 1, xn, Md, d, c.rms_eps));
+  TRY(gemm<T>(m, st, KC_QKV, xn, Md, (const T *)m->wqkv + (size_t)l0 * 3 * d * d, (size_t)3 * d * d, qkv, (size_t)M * 3 * d, M, 3 * d, d, nl));
+  KLAUNCH(m, st, KC_OTHER, k_rope_qknorm_store<T><<<dim3(M, 3 * H, nl), 128, 0, st>>>(qkv, (size_t)M * 3 * d, q, Md, kc, vc, f.kv_ls, f.kv_bs, f.T, H, hd, f.pos,
+                                                             m->rope, c.rms_eps));
+  KLAUNCH(m, st, KC_ATTN, k_attn_generic<T><<<dim3((M * H + 3) / 4, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, att, Md, M, f.T, H, hd, f.pos));
+  TRY(gemm<T>(m, st, KC_OPROJ, att, Md, (const T *)m->wo + (size_t)l0 * d * d, (size_t)d * d, a, Md, M, d, d, nl));
+  KLAUNCH(m, st, KC_OTHER, k_resid_rmsnorm_cast<T><<<dim3(M, nl), 256, 0, st>>>(xm_src, Md, (size_t)d, a, Md, 1, 0, m->coef, l0, xn, Md, d, c.rms_eps));
+  TRY(gemm<T>(m, st, KC_UP, xn, Md, (const T *)m->wup + (size_t)l0 * ff * d, (size_t)ff * d, y, (size_t)M * ff, M, ff, d, nl));
   {
     const size_t tot = (size_t)nl * M * ff;
-    k_relu2_cast<T><<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(y, z, tot);
-    count(m);
-    LAUNCH_CHECK();
+    KLAUNCH(m, st, KC_OTHER, k_relu2_cast<T><<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(y, z, tot));
   }
-  TRY(gemm<T>(m, st, z, (size_t)M * ff, (const T *)m->wdn + (size_t)l0 * d * ff, (size_t)d * ff, mb, Md, M, d, ff, nl));
+  TRY(gemm<T>(m, st, KC_DOWN, z, (size_t)M * ff, (const T *)m->wdn + (size_t)l0 * d * ff, (size_t)d * ff, mb, Md, M, d, ff, nl));
   return correct(m, f, l0, nl, mode, 1, 1, resnorm);
 }
 
 template <int PRO, int EPI>
-static int launch_gemv(snlp_model *m, cudaStream_t st, GemvParams &p, int ksplit, int nl) {
+static int launch_gemv(snlp_model *m, cudaStream_t st, int cls, GemvParams &p, int ksplit, int nl) {
   const int NT = p.M <= 8 ? 1 : 2;
   p.kslice = p.Kd / ksplit;
   const size_t sm = (size_t)NT * 8 * (p.kslice + kGemvPad) * 2 + (size_t)NT * 8 * (kGemvRows + 1) * 4 + 16 * 4;
   if (sm > kGemvMaxSmem) return fail(SNLP_ERR_UNSUPPORTED, "gemv: K slice of %d needs %zu bytes of shared memory", p.kslice, sm);
   dim3 grid(p.N / kGemvRows, ksplit, nl);
-  if (NT == 1) k_gemv_mma<1, PRO, EPI><<<grid, kGemvThreads, sm, st>>>(p);
-  else k_gemv_mma<2, PRO, EPI><<<grid, kGemvThreads, sm, st>>>(p);
-  count(m);
-  LAUNCH_CHECK();
+  KLAUNCH(m, st, cls, if (NT == 1) k_gemv_mma<1, PRO, EPI><<<grid, kGemvThreads, sm, st>>>(p);
+  else k_gemv_mma<2, PRO, EPI><<<grid, kGemvThreads, sm, st>>>(p));
   return SNLP_OK;
 }
 
@@ -418,6 +496,10 @@ static int init_kernel_attributes() {
   CU((gemv_attr<PRO_BF16, EPI_PARTIAL>()));
   CU((gemv_attr<PRO_RESID_NORM, EPI_RELU2>()));
   CU((gemv_attr<PRO_NORM, EPI_LMHEAD>()));
+  CU(cudaFuncSetAttribute(k_correct_small<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
+  CU(cudaFuncSetAttribute(k_correct_small<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
+  CU(cudaFuncSetAttribute(k_correct_small<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
+  CU(cudaFuncSetAttribute(k_correct_small<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
   return SNLP_OK;
 }
 
@@ -441,22 +523,19 @@ static int run_decode(snlp_model *m, const Fwd &f, int l0, int nl, int mode, flo
     p.xf = xa_src; p.xf_ls = Md; p.xf_rs = d; p.nsum = 1; p.eps = c.rms_eps;
     p.q = q; p.q_ls = Md; p.kc = kc; p.vc = vc; p.kv_ls = f.kv_ls; p.kv_bs = f.kv_bs;
     p.T = f.T; p.H = H; p.pos_base = f.pos; p.rope = m->rope; p.qk_eps = c.rms_eps;
-    TRY((launch_gemv<PRO_NORM, EPI_QKV>(m, st, p, 1, nl)));
+    TRY((launch_gemv<PRO_NORM, EPI_QKV>(m, st, KC_QKV, p, 1, nl)));
   }
-  const int nchunk = (f.pos_hi + f.T - 1) / kAttnChunk + 1;
-  k_attn_decode<kAttnChunk><<<dim3(nchunk, f.B * H, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, m->attn_part, f.T, H, f.pos);
-  count(m);
-  LAUNCH_CHECK();
-  k_attn_combine<<<dim3(M * H, nl), 128, 0, st>>>(m->attn_part, nchunk, f.T, H, att, Md);
-  count(m);
-  LAUNCH_CHECK();
+  const int csub = attn_csub(nl * f.B * H);
+  const int nchunk = (f.pos_hi + f.T - 1) / (csub * kAttnSub) + 1;
+  KLAUNCH(m, st, KC_ATTN, k_attn_decode<<<dim3(nchunk, f.B * H, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, m->attn_part, m->attn_counters, att, Md,
+                                                                          f.T, H, f.pos, csub));
   {
     GemvParams p{};
     p.W = (const bf *)m->wo + (size_t)l0 * d * d; p.w_ls = (size_t)d * d;
     p.N = d; p.Kd = d; p.M = M;
     p.xb = att; p.xb_ls = Md;
     p.out = m->a + l0 * Md; p.out_ls = Md; p.out_ss = (size_t)L * Md;
-    TRY((launch_gemv<PRO_BF16, EPI_PARTIAL>(m, st, p, so, nl)));
+    TRY((launch_gemv<PRO_BF16, EPI_PARTIAL>(m, st, KC_OPROJ, p, so, nl)));
   }
   {
     GemvParams p{};
@@ -465,7 +544,7 @@ static int run_decode(snlp_model *m, const Fwd &f, int l0, int nl, int mode, flo
     p.xf = xm_src; p.xf_ls = Md; p.xf_rs = d; p.nsum = 1; p.eps = c.rms_eps;
     p.ap = m->a + l0 * Md; p.ap_ls = Md; p.ap_ss = (size_t)L * Md; p.ap_splits = so; p.coef = m->coef + l0;
     p.zout = z; p.z_ls = (size_t)M * ff;
-    TRY((launch_gemv<PRO_RESID_NORM, EPI_RELU2>(m, st, p, 1, nl)));
+    TRY((launch_gemv<PRO_RESID_NORM, EPI_RELU2>(m, st, KC_UP, p, 1, nl)));
   }
   {
     GemvParams p{};
@@ -473,7 +552,7 @@ static int run_decode(snlp_model *m, const Fwd &f, int l0, int nl, int mode, flo
     p.N = d; p.Kd = ff; p.M = M;
     p.xb = z; p.xb_ls = (size_t)M * ff;
     p.out = m->mb + l0 * Md; p.out_ls = Md; p.out_ss = (size_t)L * Md;
-    TRY((launch_gemv<PRO_BF16, EPI_PARTIAL>(m, st, p, sd, nl)));
+    TRY((launch_gemv<PRO_BF16, EPI_PARTIAL>(m, st, KC_DOWN, p, sd, nl)));
   }
   return correct(m, f, l0, nl, mode, so, sd, resnorm);
 }
@@ -490,10 +569,8 @@ static int premix(snlp_model *m, const Fwd &f, int l0, int nl) {
   const snlp_config &c = m->cfg;
   if (c.n_streams == 1) return SNLP_OK;
   const size_t Md = (size_t)f.M * c.d_model;
-  k_premix<<<dim3((unsigned)((Md + 255) / 256), nl), 256, 0, f.st>>>(m->trace, Md * c.n_streams, c.n_streams, c.d_model, Md, m->coef, l0,
-                                                                    m->xa, m->xm, Md);
-  count(m);
-  LAUNCH_CHECK();
+  KLAUNCH(m, f.st, KC_OTHER, k_premix<<<dim3((unsigned)((Md + 255) / 256), nl), 256, 0, f.st>>>(m->trace, Md * c.n_streams, c.n_streams, c.d_model, Md, m->coef, l0,
+                                                                    m->xa, m->xm, Md));
   return SNLP_OK;
 }
 
@@ -508,10 +585,8 @@ static int sequential(snlp_model *m, const Fwd &f) {
 static int parallel(snlp_model *m, const Fwd &f, int K, int mode, float *resnorm_out) {
   const snlp_config &c = m->cfg;
   const size_t n4 = (size_t)f.M * c.n_streams * c.d_model / 4;
-  k_bcast_trace<<<(unsigned)((n4 + 255) / 256), 256, 0, f.st>>>(reinterpret_cast<const float4 *>(m->trace),
-                                                               reinterpret_cast<float4 *>(m->trace) + n4, n4, c.n_layer);
-  count(m);
-  LAUNCH_CHECK();
+  KLAUNCH(m, f.st, KC_OTHER, k_bcast_trace<<<(unsigned)((n4 + 255) / 256), 256, 0, f.st>>>(reinterpret_cast<const float4 *>(m->trace),
+                                                               reinterpret_cast<float4 *>(m->trace) + n4, n4, c.n_layer));
   TRY(premix(m, f, 0, c.n_layer));
   for (int k = 0; k < K; ++k)
     TRY(run_layers(m, f, 0, c.n_layer, mode, resnorm_out ? resnorm_out + (size_t)k * c.n_layer * 2 : nullptr));
@@ -527,11 +602,9 @@ static int lm_head_impl(snlp_model *m, cudaStream_t st, const float *hL, size_t 
     p.N = V; p.Kd = d; p.M = rows;
     p.xf = hL; p.xf_ls = 0; p.xf_rs = row_stride; p.nsum = n; p.eps = c.rms_eps;
     p.logits = logits; p.pm_val = m->pm_val; p.pm_idx = m->pm_idx; p.ntile = V / 128;
-    TRY((launch_gemv<PRO_NORM, EPI_LMHEAD>(m, st, p, 1, 1)));
+    TRY((launch_gemv<PRO_NORM, EPI_LMHEAD>(m, st, KC_LMHEAD, p, 1, 1)));
     if (argmax) {
-      k_argmax_tiles<<<rows, 256, 0, st>>>(m->pm_val, m->pm_idx, V / 128, argmax);
-      count(m);
-      LAUNCH_CHECK();
+      KLAUNCH(m, st, KC_LMHEAD, k_argmax_tiles<<<rows, 256, 0, st>>>(m->pm_val, m->pm_idx, V / 128, argmax));
     }
     return SNLP_OK;
   }
@@ -541,21 +614,15 @@ static int lm_head_impl(snlp_model *m, cudaStream_t st, const float *hL, size_t 
     const float *src = hL + (size_t)r0 * row_stride;
     if (c.dtype == SNLP_DTYPE_BF16) {
       typedef __nv_bfloat16 T;
-      k_rmsnorm_cast<T><<<dim3(nr, 1), 256, 0, st>>>(src, 0, row_stride, n, (T *)m->xlm, 0, d, c.rms_eps);
-      count(m);
-      LAUNCH_CHECK();
-      TRY(gemm<T>(m, st, (const T *)m->xlm, 0, (const T *)m->lm_head, 0, lg, 0, nr, V, d, 1));
+      KLAUNCH(m, st, KC_OTHER, k_rmsnorm_cast<T><<<dim3(nr, 1), 256, 0, st>>>(src, 0, row_stride, n, (T *)m->xlm, 0, d, c.rms_eps));
+      TRY(gemm<T>(m, st, KC_LMHEAD, (const T *)m->xlm, 0, (const T *)m->lm_head, 0, lg, 0, nr, V, d, 1));
     } else {
       typedef float T;
-      k_rmsnorm_cast<T><<<dim3(nr, 1), 256, 0, st>>>(src, 0, row_stride, n, (T *)m->xlm, 0, d, c.rms_eps);
-      count(m);
-      LAUNCH_CHECK();
-      TRY(gemm<T>(m, st, (const T *)m->xlm, 0, (const T *)m->lm_head, 0, lg, 0, nr, V, d, 1));
+      KLAUNCH(m, st, KC_OTHER, k_rmsnorm_cast<T><<<dim3(nr, 1), 256, 0, st>>>(src, 0, row_stride, n, (T *)m->xlm, 0, d, c.rms_eps));
+      TRY(gemm<T>(m, st, KC_LMHEAD, (const T *)m->xlm, 0, (const T *)m->lm_head, 0, lg, 0, nr, V, d, 1));
     }
     if (argmax) {
-      k_argmax_rows<<<nr, 256, 0, st>>>(lg, V, argmax + r0);
-      count(m);
-      LAUNCH_CHECK();
+      KLAUNCH(m, st, KC_LMHEAD, k_argmax_rows<<<nr, 256, 0, st>>>(lg, V, argmax + r0));
     }
   }
   return SNLP_OK;
@@ -564,11 +631,9 @@ static int lm_head_impl(snlp_model *m, cudaStream_t st, const float *hL, size_t 
 static int embed_impl(snlp_model *m, cudaStream_t st, const int32_t *ids, int rows, float *h0) {
   const snlp_config &c = m->cfg;
   if (c.dtype == SNLP_DTYPE_BF16)
-    k_embed<__nv_bfloat16><<<rows, 128, 0, st>>>(ids, (const __nv_bfloat16 *)m->embed, h0, c.d_model, c.n_streams, c.vocab);
+    KLAUNCH(m, st, KC_OTHER, k_embed<__nv_bfloat16><<<rows, 128, 0, st>>>(ids, (const __nv_bfloat16 *)m->embed, h0, c.d_model, c.n_streams, c.vocab));
   else
-    k_embed<float><<<rows, 128, 0, st>>>(ids, (const float *)m->embed, h0, c.d_model, c.n_streams, c.vocab);
-  count(m);
-  LAUNCH_CHECK();
+    KLAUNCH(m, st, KC_OTHER, k_embed<float><<<rows, 128, 0, st>>>(ids, (const float *)m->embed, h0, c.d_model, c.n_streams, c.vocab));
   return SNLP_OK;
 }
 
@@ -694,9 +759,7 @@ extern "C" int snlp_kv_len(const snlp_kv *kv, int32_t *len) {
 extern "C" int snlp_kv_truncate(snlp_kv *kv, int new_len, void *stream) {
   if (!kv) return fail(SNLP_ERR_ARG, "snlp_kv_truncate: NULL handle");
   if (new_len < 0 || new_len > kv->len) return fail(SNLP_ERR_ARG, "snlp_kv_truncate: new_len = %d outside 0..%d", new_len, kv->len);
-  k_set_int<<<1, 1, 0, (cudaStream_t)stream>>>(kv->pos, new_len);
-  count(kv->m);
-  LAUNCH_CHECK();
+  KLAUNCH(kv->m, (cudaStream_t)stream, KC_OTHER, k_set_int<<<1, 1, 0, (cudaStream_t)stream>>>(kv->pos, new_len));
   kv->len = new_len;
   return SNLP_OK;
 }
@@ -731,15 +794,11 @@ extern "C" int snlp_prefill(snlp_model *m, snlp_kv *kv, const int32_t *ids, int 
   int Tc = 0;
   for (int t0 = 0; t0 < T; t0 += Tc) {
     Tc = T - t0 < tc_max ? T - t0 : tc_max;
-    k_gather_ids<<<(B * Tc + 255) / 256, 256, 0, st>>>(ids, m->spec, B, Tc, T, t0);
-    count(m);
-    LAUNCH_CHECK();
+    KLAUNCH(m, st, KC_OTHER, k_gather_ids<<<(B * Tc + 255) / 256, 256, 0, st>>>(ids, m->spec, B, Tc, T, t0));
     TRY(embed_impl(m, st, m->spec, B * Tc, m->trace));
     Fwd f = kv_fwd(m, kv, Tc, st);
     TRY(sequential(m, f));
-    k_add_int<<<1, 1, 0, st>>>(kv->pos, Tc);
-    count(m);
-    LAUNCH_CHECK();
+    KLAUNCH(m, st, KC_OTHER, k_add_int<<<1, 1, 0, st>>>(kv->pos, Tc));
     kv->len += Tc;
   }
   if (last_argmax) {
@@ -759,21 +818,20 @@ static int decode_launches(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, in
   else TRY(parallel(m, f, K, mode, resnorm_out));
   const size_t nd = (size_t)c.n_streams * c.d_model;
   TRY(lm_head_impl(m, st, m->trace + (size_t)c.n_layer * kv->B * nd, nd, kv->B, nullptr, tok_out));
-  k_add_int<<<1, 1, 0, st>>>(kv->pos, 1);
-  count(m);
-  LAUNCH_CHECK();
+  KLAUNCH(m, st, KC_OTHER, k_add_int<<<1, 1, 0, st>>>(kv->pos, 1));
   return SNLP_OK;
 }
 
 static int decode_step_impl(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, int K, int mode, int32_t *tok_out, float *resnorm_out,
                             cudaStream_t st) {
-  if (!m->use_graphs) {
+  if (!m->use_graphs || m->timing) {
     TRY(decode_launches(m, kv, tok_in, K, mode, tok_out, resnorm_out, st));
     kv->len += 1;
     return SNLP_OK;
   }
   const bool fast = fast_decode_ok(m, kv->B);
-  GraphKey key{kv->B, K, mode, fast ? kv->len / kAttnChunk + 1 : 0, tok_in, tok_out, resnorm_out, kv};
+  const int chunk_len = attn_csub((K == 0 ? 1 : m->cfg.n_layer) * kv->B * m->cfg.n_head) * kAttnSub;
+  GraphKey key{kv->B, K, mode, fast ? kv->len / chunk_len + 1 : 0, tok_in, tok_out, resnorm_out, kv};
   auto it = m->graphs.find(key);
   if (it == m->graphs.end()) {
     if (m->graphs.size() >= 256) {
@@ -834,18 +892,14 @@ extern "C" int snlp_draft_and_verify(snlp_model *m, snlp_kv *kv, int32_t *last_t
   int32_t *y = m->spec + (c.max_rows + 1);         // [block+1]: verifier tokens
   CU(cudaMemcpyAsync(ids, last_tok, 4, cudaMemcpyDeviceToDevice, st));
   for (int i = 0; i < block; ++i) TRY(decode_step_impl(m, kv, ids + i, K, mode, ids + i + 1, nullptr, st));
-  k_set_int<<<1, 1, 0, st>>>(kv->pos, len0);
-  count(m);
-  LAUNCH_CHECK();
+  KLAUNCH(m, st, KC_OTHER, k_set_int<<<1, 1, 0, st>>>(kv->pos, len0));
   kv->len = len0;
   TRY(embed_impl(m, st, ids, block + 1, m->trace));
   Fwd f = kv_fwd(m, kv, block + 1, st);
   TRY(sequential(m, f));
   const size_t nd = (size_t)c.n_streams * c.d_model;
   TRY(lm_head_impl(m, st, m->trace + (size_t)c.n_layer * (block + 1) * nd, nd, block + 1, nullptr, y));
-  k_accept<<<1, 32, 0, st>>>(ids + 1, y, block, emitted, n_emitted, n_accepted, last_tok, kv->pos, len0);
-  count(m);
-  LAUNCH_CHECK();
+  KLAUNCH(m, st, KC_OTHER, k_accept<<<1, 32, 0, st>>>(ids + 1, y, block, emitted, n_emitted, n_accepted, last_tok, kv->pos, len0));
   int32_t n = 0;
   CU(cudaMemcpyAsync(&n, n_accepted, 4, cudaMemcpyDeviceToHost, st));
   CU(cudaStreamSynchronize(st));

@@ -23,7 +23,7 @@ EXPORTS = [
     "snlp_create", "snlp_destroy", "snlp_load_weights", "snlp_embed", "snlp_forward_sequential",
     "snlp_forward_parallel", "snlp_lm_head", "snlp_kv_create", "snlp_kv_destroy", "snlp_kv_len",
     "snlp_kv_truncate", "snlp_prefill", "snlp_decode_step", "snlp_draft_and_verify", "snlp_set_flag",
-    "snlp_launch_count", "snlp_last_error",
+    "snlp_launch_count", "snlp_kernel_times", "snlp_last_error",
 ]
 
 
@@ -216,6 +216,15 @@ class Model:
         n = C.c_int64()
         _check(_lib.snlp_launch_count(self._h, C.byref(n)))
         return n.value
+
+    KERNEL_CLASSES = ("qkv", "attention", "out_proj", "mlp_up", "mlp_down", "correction", "lm_head", "other")
+
+    def kernel_times(self, reset: bool = True):
+        """{class: (milliseconds, launches)} of the launches timed since set_flag(2, 1)."""
+        ms = (C.c_double * 8)()
+        n = (C.c_int64 * 8)()
+        _check(_lib.snlp_kernel_times(self._h, ms, n, C.c_int(1 if reset else 0)))
+        return {k: (ms[i], n[i]) for i, k in enumerate(self.KERNEL_CLASSES)}
 
     def close(self):
         if self._h:
