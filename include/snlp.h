@@ -172,6 +172,32 @@ int snlp_kernel_times(snlp_model *m, double *ms, int64_t *launches, int reset);
 /* Number of kernel launches this handle has enqueued since creation (graph replays count their nodes). */
 int snlp_launch_count(const snlp_model *m, int64_t *count);
 
+/* Greedy LM head that allocates nothing (the paper has no counterpart: this entry point exists for
+ * callers that cannot obtain device memory at call time -- for example code running between the
+ * begin and end of a CUDA stream capture, a serving loop whose memory budget has been handed entirely to
+ * another allocator, or a latency-critical path where the implicit device synchronisation of an
+ * allocation is not acceptable).  Same computation as snlp_lm_head restricted to the argmax:
+ *     argmax[r] = argmax_v  lm_head[v] . RMSNorm(sum_s hL[r][s][:])        (ties -> lowest index)
+ * but without a model handle and without a cudaMalloc'd workspace: the per-tile argmax partials go to a
+ * fixed 256 KiB array inside the library image (each GPU that loads the library holds one copy until the
+ * process exits).
+ *   hL           device fp32 [rows][n_streams][d_model]
+ *   lm_head_bf16 device bf16 bit patterns [vocab][d_model], caller-owned (inputs and outputs are still yours)
+ *   argmax       device int32 [rows]
+ * Limits: rows <= 16, vocab <= SNLP_STATIC_LM_HEAD_MAX_VOCAB (multiple of 128), d_model <=
+ * SNLP_STATIC_LM_HEAD_MAX_D_MODEL (multiple of 32); larger sizes return SNLP_ERR_SHAPE before anything
+ * is launched.  Neither this call nor anything it uses calls cudaMalloc/cudaFree.
+ * The first call on a device looks up the array's device address and sets two kernel attributes; make
+ * that first call outside any stream capture, with the device current.
+ * All calls on a device share the one array, which keeps whatever the previous call left in it (nothing
+ * needs to start at zero: every slot a call reads, it has written first).  Two calls that overlap on the
+ * GPU -- different streams without ordering, or two host threads -- race on it: serialise them.
+ * Errors: ARG (NULL, non-positive sizes), SHAPE (beyond the limits), UNSUPPORTED (vocab % 128, d_model % 32), CUDA. */
+#define SNLP_STATIC_LM_HEAD_MAX_VOCAB 262144
+#define SNLP_STATIC_LM_HEAD_MAX_D_MODEL 4096
+int snlp_lm_head_greedy_static(const float *hL, const void *lm_head_bf16, int rows, int n_streams, int d_model, int vocab,
+                               float rms_eps, int32_t *argmax, void *stream);
+
 const char *snlp_last_error(void);
 
 #ifdef __cplusplus

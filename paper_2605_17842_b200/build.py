@@ -6,7 +6,7 @@ import subprocess
 import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-SRC = os.path.join(HERE, "csrc", "snlp.cu")
+SRCS = [os.path.join(HERE, "csrc", f) for f in ("snlp.cu", "lm_head_static.cu")]
 LIB = os.path.join(HERE, "libsnlp.so")
 
 
@@ -24,7 +24,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-Xcompiler", "-fPIC,-O2", "-shared",
-           "-o", LIB, SRC, "-lcudart", "-lcuda"]
+           "-o", LIB, *SRCS, "-lcudart", "-lcuda"]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

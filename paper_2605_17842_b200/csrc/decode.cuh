@@ -225,7 +225,7 @@ __global__ void __launch_bounds__(kGemvThreads) k_gemv_mma(GemvParams p) {
 }
 
 // Final argmax over the per-tile partials (ties -> lowest index).  One block per token.
-__global__ void k_argmax_tiles(const float *__restrict__ pm_val, const int *__restrict__ pm_idx, int ntile, int32_t *__restrict__ out) {
+static __global__ void k_argmax_tiles(const float *__restrict__ pm_val, const int *__restrict__ pm_idx, int ntile, int32_t *__restrict__ out) {
   __shared__ float sv[32];
   __shared__ int si[32];
   const int tok = blockIdx.x;
@@ -266,7 +266,7 @@ __global__ void k_argmax_tiles(const float *__restrict__ pm_val, const int *__re
 constexpr int kAttnPartStride = 132;
 constexpr int kAttnSub = 64;
 
-__global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat16 *__restrict__ q, size_t q_ls,
+static __global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat16 *__restrict__ q, size_t q_ls,
                                                         const __nv_bfloat16 *__restrict__ kc, const __nv_bfloat16 *__restrict__ vc,
                                                         size_t kv_ls, size_t kv_bs, float *__restrict__ part,
                                                         unsigned *__restrict__ counters, __nv_bfloat16 *__restrict__ out,

@@ -47,6 +47,10 @@ static int fail(int code, const char *fmt, ...) {
 
 extern "C" const char *snlp_last_error(void) { return g_err.c_str(); }
 
+namespace snlp {
+void set_last_error(const char *msg) { g_err = msg; }  // for the library's other translation units
+}
+
 // ------------------------------------------------------------------------------------------------
 // handles
 constexpr int kMaxSplits = 4;    // K-splits of the partial-sum GEMV outputs

@@ -23,7 +23,7 @@ EXPORTS = [
     "snlp_create", "snlp_destroy", "snlp_load_weights", "snlp_embed", "snlp_forward_sequential",
     "snlp_forward_parallel", "snlp_lm_head", "snlp_kv_create", "snlp_kv_destroy", "snlp_kv_len",
     "snlp_kv_truncate", "snlp_prefill", "snlp_decode_step", "snlp_draft_and_verify", "snlp_set_flag",
-    "snlp_launch_count", "snlp_kernel_times", "snlp_last_error",
+    "snlp_launch_count", "snlp_kernel_times", "snlp_lm_head_greedy_static", "snlp_last_error",
 ]
 
 
@@ -236,6 +236,21 @@ class Model:
             self.close()
         except Exception:
             pass
+
+
+def lm_head_greedy_static(hL: torch.Tensor, lm_head_bf16: torch.Tensor, n_streams: int, rms_eps: float,
+                          argmax: torch.Tensor | None = None) -> torch.Tensor:
+    """Greedy LM head through the entry point that allocates nothing inside the library.
+
+    hL: cuda fp32 [rows, n_streams, d]; lm_head_bf16: cuda bf16 (or int16/uint16 bit patterns) [vocab, d].
+    Pass a pre-allocated int32 `argmax` tensor to keep the whole call free of allocations."""
+    vocab, d = lm_head_bf16.shape
+    rows = hL.numel() // (n_streams * d)
+    if argmax is None:
+        argmax = torch.empty((rows,), dtype=torch.int32, device=hL.device)
+    _check(_lib.snlp_lm_head_greedy_static(_ptr(hL), _ptr(lm_head_bf16), C.c_int(rows), C.c_int(n_streams), C.c_int(d),
+                                           C.c_int(vocab), C.c_float(rms_eps), _ptr(argmax), _stream()))
+    return argmax
 
 
 def raw_library() -> C.CDLL:
