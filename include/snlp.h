@@ -169,6 +169,10 @@ int snlp_set_flag(snlp_model *m, int flag, int value);
 /* Waits for the timed launches recorded so far and returns, per class, the summed device time in
  * milliseconds (host double[8]) and the number of launches (host int64[8]); reset != 0 clears them. */
 int snlp_kernel_times(snlp_model *m, double *ms, int64_t *launches, int reset);
+/* Synchronises `stream` and reports whether any kernel of this handle gave up on one of its bounded
+ * device-side waits since the last check (SNLP_ERR_TIMEOUT, flag cleared) or not (SNLP_OK). */
+int snlp_device_status(snlp_model *m, void *stream);
+
 /* Number of kernel launches this handle has enqueued since creation (graph replays count their nodes). */
 int snlp_launch_count(const snlp_model *m, int64_t *count);
 

@@ -16,6 +16,7 @@
 #include "correct.cuh"
 #include "decode.cuh"
 #include "generic.cuh"
+#include "umma_gemm.cuh"
 
 using namespace snlp;
 
@@ -100,6 +101,8 @@ struct snlp_model {
   bool capturing = false;
   int64_t cap_nodes = 0;
   std::map<GraphKey, GraphEntry> graphs;
+  EncodeTiledFn encode_tiled = nullptr;  // cuTensorMapEncodeTiled, looked up through the runtime
+  int *dev_err = nullptr;                // raised by a kernel whose bounded wait expired
   cudaStream_t cap_stream = nullptr;  // capture target: graphs are recorded here and replayed on the caller's stream
 };
 
@@ -257,11 +260,12 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
   A(&m->pm_val, (size_t)kDecodeRows * ((V + 127) / 128) * 4);
   A(&m->pm_idx, (size_t)kDecodeRows * ((V + 127) / 128) * 4);
   A(&m->counter, 16);
+  A(&m->dev_err, 16);
   A(&m->attn_counters, L * (size_t)kDecodeRows * c.n_head * 4);
   A(&m->zero, 16);
   A(&m->spec, 2 * (R + 1) * 4);
   if (rc == SNLP_OK) {
-    if (cudaMemset(m->attn_counters, 0, L * (size_t)kDecodeRows * c.n_head * 4) != cudaSuccess || cudaMemset(m->counter, 0, 16) != cudaSuccess || cudaMemset(m->zero, 0, 16) != cudaSuccess)
+    if (cudaMemset(m->dev_err, 0, 16) != cudaSuccess || cudaMemset(m->attn_counters, 0, L * (size_t)kDecodeRows * c.n_head * 4) != cudaSuccess || cudaMemset(m->counter, 0, 16) != cudaSuccess || cudaMemset(m->zero, 0, 16) != cudaSuccess)
       rc = fail(SNLP_ERR_CUDA, "cudaMemset failed");
   }
   if (rc == SNLP_OK) {
@@ -277,6 +281,14 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
       rc = fail(SNLP_ERR_CUDA, "rotary table upload failed");
   }
   if (rc == SNLP_OK) rc = init_kernel_attributes();
+  if (rc == SNLP_OK) {
+    cudaDriverEntryPointQueryResult qres;
+    void *fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess && qres == cudaDriverEntryPointSuccess)
+      m->encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    else
+      cudaGetLastError();  // without it the tensor-core GEMM is not used
+  }
   if (rc == SNLP_OK && cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking) != cudaSuccess)
     rc = fail(SNLP_ERR_CUDA, "cudaStreamCreateWithFlags failed");
   if (rc != SNLP_OK) {
@@ -384,6 +396,18 @@ extern "C" int snlp_kernel_times(snlp_model *m, double *ms, int64_t *launches, i
   return SNLP_OK;
 }
 
+extern "C" int snlp_device_status(snlp_model *m, void *stream) {
+  if (!m) return fail(SNLP_ERR_ARG, "snlp_device_status: NULL handle");
+  int flag = 0;
+  CU(cudaStreamSynchronize((cudaStream_t)stream));
+  CU(cudaMemcpy(&flag, m->dev_err, sizeof flag, cudaMemcpyDeviceToHost));
+  if (flag) {
+    cudaMemset(m->dev_err, 0, sizeof flag);
+    return fail(SNLP_ERR_TIMEOUT, "a device-side bounded wait expired; results of the calls since the last check are invalid");
+  }
+  return SNLP_OK;
+}
+
 extern "C" int snlp_launch_count(const snlp_model *m, int64_t *count_out) {
   if (!m || !count_out) return fail(SNLP_ERR_ARG, "snlp_launch_count: NULL argument");
   *count_out = m->launches;
@@ -476,6 +500,57 @@ static int run_generic(snlp_model *m, const Fwd &f, int l0, int nl, int mode, fl
   return correct(m, f, l0, nl, mode, 1, 1, resnorm);
 }
 
+// Tensor-core GEMM of the prefill regime: C[l] = A[l] (M x K, bf16) * W[l]^T (N x K, bf16), nl layers per launch.
+static bool umma_ok(const snlp_model *m, int N, int K) {
+  return m->encode_tiled && !m->force_generic && m->cfg.dtype == SNLP_DTYPE_BF16 && N % 128 == 0 && K % kUmmaBK == 0;
+}
+
+template <int EPI>
+static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat16 *A, size_t a_ls, const __nv_bfloat16 *W, size_t w_ls,
+                     float *C, __nv_bfloat16 *Z, size_t out_ls, int M, int N, int K, int nl) {
+  CUtensorMap ta, tb;
+  const int BN = N % 256 == 0 ? 256 : 128;
+  if (!make_tmap_bf16(m->encode_tiled, &ta, A, K, M, nl, a_ls ? a_ls : (size_t)M * K, kUmmaBM) ||
+      !make_tmap_bf16(m->encode_tiled, &tb, W, K, N, nl, w_ls ? w_ls : (size_t)N * K, BN))
+    return fail(SNLP_ERR_CUDA, "cuTensorMapEncodeTiled failed (M=%d N=%d K=%d)", M, N, K);
+  UmmaParams p{};
+  p.M = M; p.N = N; p.K = K; p.c = C; p.z = Z; p.out_ls = out_ls; p.err = m->dev_err;
+  dim3 grid(N / BN, (M + kUmmaBM - 1) / kUmmaBM, nl);
+  if (BN == 256) KLAUNCH(m, st, cls, k_umma_gemm<256, EPI><<<grid, kUmmaThreads, UmmaCfg<256>::kSmem, st>>>(ta, tb, p));
+  else KLAUNCH(m, st, cls, k_umma_gemm<128, EPI><<<grid, kUmmaThreads, UmmaCfg<128>::kSmem, st>>>(ta, tb, p));
+  return SNLP_OK;
+}
+
+// Prefill-regime sweep over layers l0 .. l0+nl-1 (bf16, more than 16 rows): the four projections run on the
+// tcgen05 tensor-core GEMM; norms, rotary/QK-norm, attention and the correction are separate kernels.
+static int run_prefill(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float *resnorm) {
+  typedef __nv_bfloat16 T;
+  const snlp_config &c = m->cfg;
+  const int M = f.M, d = c.d_model, ff = c.d_ff, H = c.n_head, hd = c.head_dim, n = c.n_streams;
+  const size_t Md = (size_t)M * d;
+  cudaStream_t st = f.st;
+  const float *xa_src = n == 1 ? m->trace + l0 * Md : m->xa + l0 * Md;
+  const float *xm_src = n == 1 ? m->trace + l0 * Md : m->xm + l0 * Md;
+  T *xn = (T *)m->xn + l0 * Md, *q = (T *)m->q + l0 * Md, *att = (T *)m->att + l0 * Md;
+  T *z = (T *)m->z + (size_t)l0 * M * ff;
+  float *qkv = m->qkv_raw + (size_t)l0 * M * 3 * d, *a = m->a + l0 * Md, *mb = m->mb + l0 * Md;
+  T *kc = (T *)f.kc + (size_t)l0 * f.kv_ls, *vc = (T *)f.vc + (size_t)l0 * f.kv_ls;
+
+  KLAUNCH(m, st, KC_OTHER, k_rmsnorm_cast<T><<<dim3(M, nl), 256, 0, st>>>(xa_src, Md, (size_t)d, 1, xn, Md, d, c.rms_eps));
+  TRY(umma_gemm<UEPI_F32>(m, st, KC_QKV, xn, Md, (const T *)m->wqkv + (size_t)l0 * 3 * d * d, (size_t)3 * d * d, qkv, nullptr,
+                          (size_t)M * 3 * d, M, 3 * d, d, nl));
+  KLAUNCH(m, st, KC_OTHER, k_rope_qknorm_store<T><<<dim3(M, 3 * H, nl), 128, 0, st>>>(qkv, (size_t)M * 3 * d, q, Md, kc, vc, f.kv_ls, f.kv_bs, f.T, H, hd, f.pos,
+                                                             m->rope, c.rms_eps));
+  KLAUNCH(m, st, KC_ATTN, k_attn_generic<T><<<dim3((M * H + 3) / 4, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, att, Md, M, f.T, H, hd, f.pos));
+  TRY(umma_gemm<UEPI_F32>(m, st, KC_OPROJ, att, Md, (const T *)m->wo + (size_t)l0 * d * d, (size_t)d * d, a, nullptr, Md, M, d, d, nl));
+  KLAUNCH(m, st, KC_OTHER, k_resid_rmsnorm_cast<T><<<dim3(M, nl), 256, 0, st>>>(xm_src, Md, (size_t)d, a, Md, 1, 0, m->coef, l0, xn, Md, d, c.rms_eps));
+  TRY(umma_gemm<UEPI_RELU2_BF16>(m, st, KC_UP, xn, Md, (const T *)m->wup + (size_t)l0 * ff * d, (size_t)ff * d, nullptr, z, (size_t)M * ff,
+                                 M, ff, d, nl));
+  TRY(umma_gemm<UEPI_F32>(m, st, KC_DOWN, z, (size_t)M * ff, (const T *)m->wdn + (size_t)l0 * d * ff, (size_t)d * ff, mb, nullptr, Md, M, d,
+                          ff, nl));
+  return correct(m, f, l0, nl, mode, 1, 1, resnorm);
+}
+
 template <int PRO, int EPI>
 static int launch_gemv(snlp_model *m, cudaStream_t st, int cls, GemvParams &p, int ksplit, int nl) {
   const int NT = p.M <= 8 ? 1 : 2;
@@ -500,6 +575,10 @@ static int init_kernel_attributes() {
   CU((gemv_attr<PRO_BF16, EPI_PARTIAL>()));
   CU((gemv_attr<PRO_RESID_NORM, EPI_RELU2>()));
   CU((gemv_attr<PRO_NORM, EPI_LMHEAD>()));
+  CU(cudaFuncSetAttribute(k_umma_gemm<128, UEPI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<128>::kSmem));
+  CU(cudaFuncSetAttribute(k_umma_gemm<256, UEPI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<256>::kSmem));
+  CU(cudaFuncSetAttribute(k_umma_gemm<128, UEPI_RELU2_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<128>::kSmem));
+  CU(cudaFuncSetAttribute(k_umma_gemm<256, UEPI_RELU2_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<256>::kSmem));
   CU(cudaFuncSetAttribute(k_correct_small<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
   CU(cudaFuncSetAttribute(k_correct_small<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
   CU(cudaFuncSetAttribute(k_correct_small<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
@@ -563,6 +642,8 @@ static int run_decode(snlp_model *m, const Fwd &f, int l0, int nl, int mode, flo
 
 static int run_layers(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float *resnorm) {
   if (fast_decode_ok(m, f.M)) return run_decode(m, f, l0, nl, mode, resnorm);
+  if (umma_ok(m, m->cfg.d_model, m->cfg.d_model) && umma_ok(m, m->cfg.d_ff, m->cfg.d_ff) && f.M > kDecodeRows)
+    return run_prefill(m, f, l0, nl, mode, resnorm);
   if (m->cfg.dtype == SNLP_DTYPE_BF16) return run_generic<__nv_bfloat16>(m, f, l0, nl, mode, resnorm);
   return run_generic<float>(m, f, l0, nl, mode, resnorm);
 }

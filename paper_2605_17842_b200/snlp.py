@@ -23,7 +23,7 @@ EXPORTS = [
     "snlp_create", "snlp_destroy", "snlp_load_weights", "snlp_embed", "snlp_forward_sequential",
     "snlp_forward_parallel", "snlp_lm_head", "snlp_kv_create", "snlp_kv_destroy", "snlp_kv_len",
     "snlp_kv_truncate", "snlp_prefill", "snlp_decode_step", "snlp_draft_and_verify", "snlp_set_flag",
-    "snlp_launch_count", "snlp_kernel_times", "snlp_lm_head_greedy_static", "snlp_last_error",
+    "snlp_launch_count", "snlp_kernel_times", "snlp_device_status", "snlp_lm_head_greedy_static", "snlp_last_error",
 ]
 
 
@@ -211,6 +211,10 @@ class Model:
     # -- misc -------------------------------------------------------------------------------------
     def set_flag(self, flag: int, value: int):
         _check(_lib.snlp_set_flag(self._h, C.c_int(flag), C.c_int(value)))
+
+    def device_status(self):
+        """Synchronise and raise SnlpError(ERR_TIMEOUT) if a kernel gave up on a bounded device-side wait."""
+        _check(_lib.snlp_device_status(self._h, _stream()))
 
     def launch_count(self) -> int:
         n = C.c_int64()
