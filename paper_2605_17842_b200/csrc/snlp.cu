@@ -17,6 +17,7 @@
 #include "decode.cuh"
 #include "generic.cuh"
 #include "umma_gemm.cuh"
+#include "attn_prefill.cuh"
 
 using namespace snlp;
 
@@ -541,7 +542,11 @@ static int run_prefill(snlp_model *m, const Fwd &f, int l0, int nl, int mode, fl
                           (size_t)M * 3 * d, M, 3 * d, d, nl));
   KLAUNCH(m, st, KC_OTHER, k_rope_qknorm_store<T><<<dim3(M, 3 * H, nl), 128, 0, st>>>(qkv, (size_t)M * 3 * d, q, Md, kc, vc, f.kv_ls, f.kv_bs, f.T, H, hd, f.pos,
                                                              m->rope, c.rms_eps));
-  KLAUNCH(m, st, KC_ATTN, k_attn_generic<T><<<dim3((M * H + 3) / 4, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, att, Md, M, f.T, H, hd, f.pos));
+  if (hd == 128)
+    KLAUNCH(m, st, KC_ATTN, k_attn_prefill<<<dim3((f.T + kFaRows - 1) / kFaRows, f.B * H, nl), 128, kFaSmem, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, att, Md,
+                                                                                                    f.T, H, f.pos));
+  else
+    KLAUNCH(m, st, KC_ATTN, k_attn_generic<T><<<dim3((M * H + 3) / 4, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, att, Md, M, f.T, H, hd, f.pos));
   TRY(umma_gemm<UEPI_F32>(m, st, KC_OPROJ, att, Md, (const T *)m->wo + (size_t)l0 * d * d, (size_t)d * d, a, nullptr, Md, M, d, d, nl));
   KLAUNCH(m, st, KC_OTHER, k_resid_rmsnorm_cast<T><<<dim3(M, nl), 256, 0, st>>>(xm_src, Md, (size_t)d, a, Md, 1, 0, m->coef, l0, xn, Md, d, c.rms_eps));
   TRY(umma_gemm<UEPI_RELU2_BF16>(m, st, KC_UP, xn, Md, (const T *)m->wup + (size_t)l0 * ff * d, (size_t)ff * d, nullptr, z, (size_t)M * ff,
@@ -579,6 +584,7 @@ static int init_kernel_attributes() {
   CU(cudaFuncSetAttribute(k_umma_gemm<256, UEPI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<256>::kSmem));
   CU(cudaFuncSetAttribute(k_umma_gemm<128, UEPI_RELU2_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<128>::kSmem));
   CU(cudaFuncSetAttribute(k_umma_gemm<256, UEPI_RELU2_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<256>::kSmem));
+  CU(cudaFuncSetAttribute(k_attn_prefill, cudaFuncAttributeMaxDynamicSharedMemorySize, kFaSmem));
   CU(cudaFuncSetAttribute(k_correct_small<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
   CU(cudaFuncSetAttribute(k_correct_small<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
   CU(cudaFuncSetAttribute(k_correct_small<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
