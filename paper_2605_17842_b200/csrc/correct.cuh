@@ -18,6 +18,8 @@ struct CorrParams {
   int mode;          // SNLP_MODE_*
   const HcCoef *coef;
   float *xa, *xm;    // [L][M][d] pre-mapped inputs for the next sweep (n > 1 only)
+  __nv_bfloat16 *xb; // nullable: [L][M][d] bf16 copy of the next sweep's attention-branch input (h_l, or pa_l . x_l)
+  float *ssq_x;      //           [L][d/128][M] its row sums of squares, one partial per 128 columns
   float *partial;    // [gridDim.x][nl][2] scratch for the norms (nullable => no norms)
   float *resnorm;    // [L][2] (entries l0 .. l0+nl-1 written)
   unsigned *counter; // zero on entry, left zero on exit
@@ -59,7 +61,7 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
   }
   for (int i = 0; i < p.nl; ++i) {
     const int l = p.l0 + i;
-    float rs = 0.f, hs = 0.f;
+    float rs = 0.f, hs = 0.f, xs = 0.f;
     if (active) {
       float4 av = a4[(size_t)l * Md4 + bm_off];
       for (int q = 1; q < p.a_splits; ++q) av = f4_add(av, a4[(size_t)q * (p.a_ss >> 2) + (size_t)l * Md4 + bm_off]);
@@ -100,6 +102,7 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
         hs += f4_sq(oldn[r]);
         tr4[(size_t)(l + 1) * state4 + st_off + (size_t)r * d4] = newn[r];
       }
+      float4 nxt = newn[0];  // the next layer's attention-branch input
       if (NS > 1 && l + 1 < p.L) {
         const HcCoef &cn = p.coef[l + 1];
         float4 sa = f4_scale(cn.pa[0], newn[0]), sm = f4_scale(cn.pmra[0], newn[0]);
@@ -110,9 +113,21 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
         }
         reinterpret_cast<float4 *>(p.xa)[(size_t)(l + 1) * Md4 + bm_off] = sa;
         reinterpret_cast<float4 *>(p.xm)[(size_t)(l + 1) * Md4 + bm_off] = sm;
+        nxt = sa;
+      }
+      if (p.xb != nullptr && l + 1 < p.L) {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(nxt.x, nxt.y), hi = __floats2bfloat162_rn(nxt.z, nxt.w);
+        uint2 pk = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+        reinterpret_cast<uint2 *>(p.xb)[(size_t)(l + 1) * Md4 + bm_off] = pk;
+        xs = f4_sq(nxt);
       }
 #pragma unroll
       for (int r = 0; r < NS; ++r) { oldp[r] = oldn[r]; newp[r] = newn[r]; }
+    }
+    if (p.xb != nullptr && l + 1 < p.L) {
+      // d is a multiple of 128 here, so the 32 lanes of a warp hold 128 consecutive columns of one row
+      xs = warp_sum(xs);
+      if (lane == 0 && active) p.ssq_x[((size_t)(l + 1) * (d4 >> 5) + (c4 >> 5)) * p.M + row] = xs;
     }
     if (want_norm) {
       rs = warp_sum(rs);
@@ -142,6 +157,35 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
   if (threadIdx.x == 0) *p.counter = 0u;
 }
 
+
+// Branch inputs of layers l0 .. l0+nl-1 from the current trace, for the tensor-core path: xb = bf16 of the
+// attention-branch input (h_l, or pa_l . x_l for mHC), its per-128-column sums of squares, and for mHC the
+// fp32 MLP pre-map xm = pmra_l . x_l.  Used before the first sweep; afterwards k_correct keeps them current.
+// grid (M, nl), d/4 threads (d a multiple of 128).
+template <int NS>
+__global__ void k_prep_rows(const float *__restrict__ trace, int l0, int M, int d, const HcCoef *__restrict__ coef,
+                            __nv_bfloat16 *__restrict__ xb, float *__restrict__ ssq_x, float *__restrict__ xm) {
+  const int d4 = d >> 2, c4 = threadIdx.x, l = l0 + blockIdx.y;
+  const size_t row = blockIdx.x, Md4 = (size_t)M * d4;
+  const float4 *x = reinterpret_cast<const float4 *>(trace) + (size_t)l * Md4 * NS + row * NS * d4 + c4;
+  float4 v = x[0];
+  if (NS > 1) {
+    const HcCoef &c = coef[l];
+    float4 sa = f4_scale(c.pa[0], v), sm = f4_scale(c.pmra[0], v);
+#pragma unroll
+    for (int s = 1; s < NS; ++s) {
+      const float4 xv = x[(size_t)s * d4];
+      sa = f4_fma(c.pa[s], xv, sa);
+      sm = f4_fma(c.pmra[s], xv, sm);
+    }
+    reinterpret_cast<float4 *>(xm)[(size_t)l * Md4 + row * d4 + c4] = sm;
+    v = sa;
+  }
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+  reinterpret_cast<uint2 *>(xb)[(size_t)l * Md4 + row * d4 + c4] = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+  const float ss = warp_sum(f4_sq(v));
+  if ((threadIdx.x & 31) == 0) ssq_x[((size_t)l * (d4 >> 5) + (c4 >> 5)) * M + row] = ss;
+}
 
 // Latency-oriented variant for the decode regime (a handful of rows): the per-thread loop over
 // layers above serialises ~7 dependent-latency loads per layer, which dominates when there are too

@@ -84,6 +84,8 @@ struct snlp_model {
   float2 *rope = nullptr;
   // workspace (R = max_rows)
   float *trace = nullptr, *xa = nullptr, *xm = nullptr, *qkv_raw = nullptr, *a = nullptr, *y_raw = nullptr, *mb = nullptr;
+  void *ub = nullptr;
+  float *ssq_x = nullptr, *ssq_u = nullptr;
   void *xn = nullptr, *q = nullptr, *att = nullptr, *z = nullptr, *sk = nullptr, *sv = nullptr, *xlm = nullptr;
   float *attn_part = nullptr, *corr_part = nullptr, *logits = nullptr, *pm_val = nullptr;
   int *pm_idx = nullptr;
@@ -185,6 +187,7 @@ static int dalloc(snlp_model *m, P **p, size_t bytes) {
 }
 
 static int init_kernel_attributes();
+static bool fused_prefill_ok(const snlp_model *m, int M);
 
 // 64-key sub-blocks per split-KV chunk.  It depends only on how many (layer, sequence, head) triples one
 // launch covers (not on the context length or the number of query rows), so that calls of the same
@@ -246,6 +249,11 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
   A(&m->y_raw, L * R * ff * 4);
   A(&m->mb, L * split_rows * d * 4);
   A(&m->xn, L * R * d * es);
+  if (c.dtype == SNLP_DTYPE_BF16 && d % 128 == 0) {
+    A(&m->ub, L * R * d * es);
+    A(&m->ssq_x, L * (d / 128) * R * 4);
+    A(&m->ssq_u, L * (d / 128) * R * 4);
+  }
   A(&m->q, L * R * d * es);
   A(&m->att, L * R * d * es);
   A(&m->z, L * R * ff * es);
@@ -443,6 +451,8 @@ static int correct(snlp_model *m, const Fwd &f, int l0, int nl, int mode, int a_
   p.coef = m->coef;
   p.xa = m->xa;
   p.xm = m->xm;
+  p.xb = fused_prefill_ok(m, f.M) ? (__nv_bfloat16 *)m->xn : nullptr;
+  p.ssq_x = m->ssq_x;
   p.partial = resnorm ? m->corr_part : nullptr;
   p.resnorm = resnorm;
   p.counter = m->counter;
@@ -502,58 +512,83 @@ static int run_generic(snlp_model *m, const Fwd &f, int l0, int nl, int mode, fl
 }
 
 // Tensor-core GEMM of the prefill regime: C[l] = A[l] (M x K, bf16) * W[l]^T (N x K, bf16), nl layers per launch.
-static bool umma_ok(const snlp_model *m, int N, int K) {
-  return m->encode_tiled && !m->force_generic && m->cfg.dtype == SNLP_DTYPE_BF16 && N % 128 == 0 && K % kUmmaBK == 0;
+static bool fused_prefill_ok(const snlp_model *m, int M) {
+  const snlp_config &c = m->cfg;
+  return m->encode_tiled && !m->force_generic && c.dtype == SNLP_DTYPE_BF16 && c.head_dim == 128 && M > kDecodeRows &&
+         c.d_model % 128 == 0 && c.d_ff % 128 == 0 && c.d_model <= 4096;
 }
 
 template <int EPI>
 static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat16 *A, size_t a_ls, const __nv_bfloat16 *W, size_t w_ls,
-                     float *C, __nv_bfloat16 *Z, size_t out_ls, int M, int N, int K, int nl) {
+                     UmmaParams p, int M, int N, int K, int nl) {
   CUtensorMap ta, tb;
   const int BN = N % 256 == 0 ? 256 : 128;
   if (!make_tmap_bf16(m->encode_tiled, &ta, A, K, M, nl, a_ls ? a_ls : (size_t)M * K, kUmmaBM) ||
       !make_tmap_bf16(m->encode_tiled, &tb, W, K, N, nl, w_ls ? w_ls : (size_t)N * K, BN))
     return fail(SNLP_ERR_CUDA, "cuTensorMapEncodeTiled failed (M=%d N=%d K=%d)", M, N, K);
-  UmmaParams p{};
-  p.M = M; p.N = N; p.K = K; p.c = C; p.z = Z; p.out_ls = out_ls; p.err = m->dev_err;
+  p.M = M; p.N = N; p.K = K; p.err = m->dev_err;
   dim3 grid(N / BN, (M + kUmmaBM - 1) / kUmmaBM, nl);
   if (BN == 256) KLAUNCH(m, st, cls, k_umma_gemm<256, EPI><<<grid, kUmmaThreads, UmmaCfg<256>::kSmem, st>>>(ta, tb, p));
   else KLAUNCH(m, st, cls, k_umma_gemm<128, EPI><<<grid, kUmmaThreads, UmmaCfg<128>::kSmem, st>>>(ta, tb, p));
   return SNLP_OK;
 }
 
-// Prefill-regime sweep over layers l0 .. l0+nl-1 (bf16, more than 16 rows): the four projections run on the
-// tcgen05 tensor-core GEMM; norms, rotary/QK-norm, attention and the correction are separate kernels.
+// Prefill-regime sweep over layers l0 .. l0+nl-1 (bf16, head_dim 128, more than 16 rows): six launches.
+// The four projections run on the tcgen05 tensor-core GEMM with everything else of the block fused into
+// their epilogues (row RMSNorm as a scale, rotary + QK-norm + KV store, residual add + sum of squares,
+// ReLU^2); the bf16 branch inputs xb/ssq_x of the range must be current (k_prep_rows or the last correction).
 static int run_prefill(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float *resnorm) {
   typedef __nv_bfloat16 T;
   const snlp_config &c = m->cfg;
-  const int M = f.M, d = c.d_model, ff = c.d_ff, H = c.n_head, hd = c.head_dim, n = c.n_streams;
+  const int M = f.M, d = c.d_model, ff = c.d_ff, H = c.n_head, n = c.n_streams, P = d / 128;
   const size_t Md = (size_t)M * d;
   cudaStream_t st = f.st;
-  const float *xa_src = n == 1 ? m->trace + l0 * Md : m->xa + l0 * Md;
   const float *xm_src = n == 1 ? m->trace + l0 * Md : m->xm + l0 * Md;
-  T *xn = (T *)m->xn + l0 * Md, *q = (T *)m->q + l0 * Md, *att = (T *)m->att + l0 * Md;
+  T *xb = (T *)m->xn + l0 * Md, *ub = (T *)m->ub + l0 * Md, *q = (T *)m->q + l0 * Md, *att = (T *)m->att + l0 * Md;
   T *z = (T *)m->z + (size_t)l0 * M * ff;
-  float *qkv = m->qkv_raw + (size_t)l0 * M * 3 * d, *a = m->a + l0 * Md, *mb = m->mb + l0 * Md;
+  float *a = m->a + l0 * Md, *mb = m->mb + l0 * Md;
   T *kc = (T *)f.kc + (size_t)l0 * f.kv_ls, *vc = (T *)f.vc + (size_t)l0 * f.kv_ls;
-
-  KLAUNCH(m, st, KC_OTHER, k_rmsnorm_cast<T><<<dim3(M, nl), 256, 0, st>>>(xa_src, Md, (size_t)d, 1, xn, Md, d, c.rms_eps));
-  TRY(umma_gemm<UEPI_F32>(m, st, KC_QKV, xn, Md, (const T *)m->wqkv + (size_t)l0 * 3 * d * d, (size_t)3 * d * d, qkv, nullptr,
-                          (size_t)M * 3 * d, M, 3 * d, d, nl));
-  KLAUNCH(m, st, KC_OTHER, k_rope_qknorm_store<T><<<dim3(M, 3 * H, nl), 128, 0, st>>>(qkv, (size_t)M * 3 * d, q, Md, kc, vc, f.kv_ls, f.kv_bs, f.T, H, hd, f.pos,
-                                                             m->rope, c.rms_eps));
-  if (hd == 128)
-    KLAUNCH(m, st, KC_ATTN, k_attn_prefill<<<dim3((f.T + kFaRows - 1) / kFaRows, f.B * H, nl), 128, kFaSmem, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, att, Md,
-                                                                                                    f.T, H, f.pos));
-  else
-    KLAUNCH(m, st, KC_ATTN, k_attn_generic<T><<<dim3((M * H + 3) / 4, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, att, Md, M, f.T, H, hd, f.pos));
-  TRY(umma_gemm<UEPI_F32>(m, st, KC_OPROJ, att, Md, (const T *)m->wo + (size_t)l0 * d * d, (size_t)d * d, a, nullptr, Md, M, d, d, nl));
-  KLAUNCH(m, st, KC_OTHER, k_resid_rmsnorm_cast<T><<<dim3(M, nl), 256, 0, st>>>(xm_src, Md, (size_t)d, a, Md, 1, 0, m->coef, l0, xn, Md, d, c.rms_eps));
-  TRY(umma_gemm<UEPI_RELU2_BF16>(m, st, KC_UP, xn, Md, (const T *)m->wup + (size_t)l0 * ff * d, (size_t)ff * d, nullptr, z, (size_t)M * ff,
-                                 M, ff, d, nl));
-  TRY(umma_gemm<UEPI_F32>(m, st, KC_DOWN, z, (size_t)M * ff, (const T *)m->wdn + (size_t)l0 * d * ff, (size_t)d * ff, mb, nullptr, Md, M, d,
-                          ff, nl));
+  const int Pu = d / (d % 256 == 0 ? 256 : 128);  // column tiles of the out-projection = partials of sum u^2
+  {
+    UmmaParams p{};
+    p.ssq = m->ssq_x + (size_t)l0 * P * M; p.nparts = P; p.eps = c.rms_eps;
+    p.q = q; p.q_ls = Md; p.kc = kc; p.vc = vc; p.kv_ls = f.kv_ls; p.kv_bs = f.kv_bs;
+    p.T = f.T; p.d = d; p.pos_base = f.pos; p.rope = m->rope; p.qk_eps = c.rms_eps;
+    TRY(umma_gemm<UEPI_QKV>(m, st, KC_QKV, xb, Md, (const T *)m->wqkv + (size_t)l0 * 3 * d * d, (size_t)3 * d * d, p, M, 3 * d, d, nl));
+  }
+  KLAUNCH(m, st, KC_ATTN, k_attn_prefill<<<dim3((f.T + kFaRows - 1) / kFaRows, f.B * H, nl), 128, kFaSmem, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, att, Md,
+                                                                                                  f.T, H, f.pos));
+  {
+    UmmaParams p{};
+    p.c = a; p.z = ub; p.out_ls = Md;
+    p.xm = xm_src; p.xm_ls = Md; p.coef = m->coef + l0; p.ssq_out = m->ssq_u + (size_t)l0 * Pu * M;
+    TRY(umma_gemm<UEPI_RESID>(m, st, KC_OPROJ, att, Md, (const T *)m->wo + (size_t)l0 * d * d, (size_t)d * d, p, M, d, d, nl));
+  }
+  {
+    UmmaParams p{};
+    p.z = z; p.out_ls = (size_t)M * ff;
+    p.ssq = m->ssq_u + (size_t)l0 * Pu * M; p.nparts = Pu; p.eps = c.rms_eps;
+    TRY(umma_gemm<UEPI_RELU2_BF16>(m, st, KC_UP, ub, Md, (const T *)m->wup + (size_t)l0 * ff * d, (size_t)ff * d, p, M, ff, d, nl));
+  }
+  {
+    UmmaParams p{};
+    p.c = mb; p.out_ls = Md;
+    TRY(umma_gemm<UEPI_F32>(m, st, KC_DOWN, z, (size_t)M * ff, (const T *)m->wdn + (size_t)l0 * d * ff, (size_t)d * ff, p, M, d, ff, nl));
+  }
   return correct(m, f, l0, nl, mode, 1, 1, resnorm);
+}
+
+// bf16 branch inputs of layers l0 .. l0+nl-1 for run_prefill (and the fp32 MLP pre-map of mHC models)
+static int prep_rows(snlp_model *m, const Fwd &f, int l0, int nl) {
+  const snlp_config &c = m->cfg;
+  dim3 grid(f.M, nl);
+  const int threads = c.d_model / 4;
+  switch (c.n_streams) {
+#define CASE(NS) case NS: KLAUNCH(m, f.st, KC_OTHER, k_prep_rows<NS><<<grid, threads, 0, f.st>>>(m->trace, l0, f.M, c.d_model, m->coef, (__nv_bfloat16 *)m->xn, m->ssq_x, m->xm)); break;
+    CASE(1) CASE(2) CASE(3) CASE(4) CASE(5) CASE(6) CASE(7) CASE(8)
+#undef CASE
+  }
+  return SNLP_OK;
 }
 
 template <int PRO, int EPI>
@@ -582,6 +617,10 @@ static int init_kernel_attributes() {
   CU((gemv_attr<PRO_NORM, EPI_LMHEAD>()));
   CU(cudaFuncSetAttribute(k_umma_gemm<128, UEPI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<128>::kSmem));
   CU(cudaFuncSetAttribute(k_umma_gemm<256, UEPI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<256>::kSmem));
+  CU(cudaFuncSetAttribute(k_umma_gemm<128, UEPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<128>::kSmem));
+  CU(cudaFuncSetAttribute(k_umma_gemm<256, UEPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<256>::kSmem));
+  CU(cudaFuncSetAttribute(k_umma_gemm<128, UEPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<128>::kSmem));
+  CU(cudaFuncSetAttribute(k_umma_gemm<256, UEPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<256>::kSmem));
   CU(cudaFuncSetAttribute(k_umma_gemm<128, UEPI_RELU2_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<128>::kSmem));
   CU(cudaFuncSetAttribute(k_umma_gemm<256, UEPI_RELU2_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<256>::kSmem));
   CU(cudaFuncSetAttribute(k_attn_prefill, cudaFuncAttributeMaxDynamicSharedMemorySize, kFaSmem));
@@ -648,8 +687,7 @@ static int run_decode(snlp_model *m, const Fwd &f, int l0, int nl, int mode, flo
 
 static int run_layers(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float *resnorm) {
   if (fast_decode_ok(m, f.M)) return run_decode(m, f, l0, nl, mode, resnorm);
-  if (umma_ok(m, m->cfg.d_model, m->cfg.d_model) && umma_ok(m, m->cfg.d_ff, m->cfg.d_ff) && f.M > kDecodeRows)
-    return run_prefill(m, f, l0, nl, mode, resnorm);
+  if (fused_prefill_ok(m, f.M)) return run_prefill(m, f, l0, nl, mode, resnorm);
   if (m->cfg.dtype == SNLP_DTYPE_BF16) return run_generic<__nv_bfloat16>(m, f, l0, nl, mode, resnorm);
   return run_generic<float>(m, f, l0, nl, mode, resnorm);
 }
@@ -667,7 +705,8 @@ static int premix(snlp_model *m, const Fwd &f, int l0, int nl) {
 
 // Alg. 1 over the internal trace (trace[0] must hold h_0).
 static int sequential(snlp_model *m, const Fwd &f) {
-  TRY(premix(m, f, 0, 1));
+  if (fused_prefill_ok(m, f.M)) TRY(prep_rows(m, f, 0, 1));
+  else TRY(premix(m, f, 0, 1));
   for (int l = 0; l < m->cfg.n_layer; ++l) TRY(run_layers(m, f, l, 1, native_mode(m), nullptr));
   return SNLP_OK;
 }
@@ -678,7 +717,8 @@ static int parallel(snlp_model *m, const Fwd &f, int K, int mode, float *resnorm
   const size_t n4 = (size_t)f.M * c.n_streams * c.d_model / 4;
   KLAUNCH(m, f.st, KC_OTHER, k_bcast_trace<<<(unsigned)((n4 + 255) / 256), 256, 0, f.st>>>(reinterpret_cast<const float4 *>(m->trace),
                                                                reinterpret_cast<float4 *>(m->trace) + n4, n4, c.n_layer));
-  TRY(premix(m, f, 0, c.n_layer));
+  if (fused_prefill_ok(m, f.M)) TRY(prep_rows(m, f, 0, c.n_layer));
+  else TRY(premix(m, f, 0, c.n_layer));
   for (int k = 0; k < K; ++k)
     TRY(run_layers(m, f, 0, c.n_layer, mode, resnorm_out ? resnorm_out + (size_t)k * c.n_layer * 2 : nullptr));
   return SNLP_OK;

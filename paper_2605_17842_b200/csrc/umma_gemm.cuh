@@ -13,14 +13,31 @@
 
 namespace snlp {
 
-enum { UEPI_F32 = 0, UEPI_RELU2_BF16 = 1 };
+// Epilogues.  The A operand of the QKV and MLP-up products is the *un-normalised* bf16 branch input; its
+// RMSNorm is a per-row scalar, so it is applied to the accumulator row here (sum of squares of the row =
+// sum of `nparts` partials written by the producing kernel, in fixed order).
+//   UEPI_F32         c = acc
+//   UEPI_RELU2_BF16  z = bf16(relu(rstd_row * acc)^2)                      (rstd_row = 1 if ssq == nullptr)
+//   UEPI_QKV         per 128-wide head: y = rstd_row * acc; q,k: rotary + RMSNorm over the head; q -> q buffer,
+//                    k,v -> the layer's key/value store at the row's position
+//   UEPI_RESID       u = xm + kappa_l * acc;  a = acc (fp32, for the correction), ub = bf16(u), and the partial
+//                    sum of u^2 over this CTA's BN columns -> ssq_out[l][n_tile][row]
+enum { UEPI_F32 = 0, UEPI_RELU2_BF16 = 1, UEPI_QKV = 2, UEPI_RESID = 3 };
 
 struct UmmaParams {
   int M, N, K;             // rows, columns, reduction length of one layer's product
-  float *c;                // UEPI_F32:        [nl][M][N] fp32
-  __nv_bfloat16 *z;        // UEPI_RELU2_BF16: [nl][M][N] bf16 = relu(acc)^2
-  size_t out_ls;           // layer stride of the output (elements)
+  float *c;                // UEPI_F32 / UEPI_RESID: [nl][M][N] fp32
+  __nv_bfloat16 *z;        // UEPI_RELU2_BF16: [nl][M][N] bf16;  UEPI_RESID: ub [nl][M][N] bf16
+  size_t out_ls;           // layer stride of the outputs above (elements)
   int *err;                // device flag set to 1 when a bounded wait expires
+  // row scale (UEPI_QKV, UEPI_RELU2_BF16)
+  const float *ssq; int nparts; float eps;   // [nl][nparts][M] partial sums of squares of the A rows
+  // UEPI_QKV
+  __nv_bfloat16 *q; size_t q_ls;
+  __nv_bfloat16 *kc, *vc; size_t kv_ls, kv_bs;
+  int T, d; const int *pos_base; const float2 *rope; float qk_eps;
+  // UEPI_RESID
+  const float *xm; size_t xm_ls; const HcCoef *coef; float *ssq_out;   // ssq_out [nl][N/BN][M]
 };
 
 constexpr int kUmmaThreads = 192;   // warp 0: TMA, warp 1: MMA + TMEM allocation, warps 2-5: epilogue
@@ -223,31 +240,144 @@ __global__ void __launch_bounds__(kUmmaThreads) k_umma_gemm(const __grid_constan
     if (ok) {
       const int quarter = warp & 3;  // tensor-memory lanes this warp may read: 32*quarter .. +31
       const int row = m_tile * kUmmaBM + quarter * 32 + lane;
+      const bool live = row < p.M;
       const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16);
+      float rstd = 1.f;
+      if ((EPI == UEPI_QKV || EPI == UEPI_RELU2_BF16) && p.ssq != nullptr && live) {
+        float ss = 0.f;
+        for (int i = 0; i < p.nparts; ++i) ss += p.ssq[((size_t)l * p.nparts + i) * p.M + row];
+        rstd = rsqrtf(ss / (float)p.K + p.eps);
+      }
+      if (EPI == UEPI_F32 || EPI == UEPI_RELU2_BF16) {
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(tbase + c * 32, r);
-        if (row < p.M) {
-          const size_t off = (size_t)l * p.out_ls + (size_t)row * p.N + (size_t)n_tile * BN + c * 32;
-          if (EPI == UEPI_F32) {
-            float4 *dst = reinterpret_cast<float4 *>(p.c + off);
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(tbase + c * 32, r);
+          if (live) {
+            const size_t off = (size_t)l * p.out_ls + (size_t)row * p.N + (size_t)n_tile * BN + c * 32;
+            if (EPI == UEPI_F32) {
+              float4 *dst = reinterpret_cast<float4 *>(p.c + off);
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-              dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
-                                   __uint_as_float(r[4 * j + 3]));
-          } else {
-            uint4 *dst = reinterpret_cast<uint4 *>(p.z + off);
+              for (int j = 0; j < 8; ++j)
+                dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                                     __uint_as_float(r[4 * j + 3]));
+            } else {
+              uint4 *dst = reinterpret_cast<uint4 *>(p.z + off);
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                uint32_t w[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  const float a = fmaxf(__uint_as_float(r[8 * j + 2 * q]) * rstd, 0.f);
+                  const float b = fmaxf(__uint_as_float(r[8 * j + 2 * q + 1]) * rstd, 0.f);
+                  __nv_bfloat162 v = __floats2bfloat162_rn(a * a, b * b);
+                  w[q] = *reinterpret_cast<uint32_t *>(&v);
+                }
+                dst[j] = make_uint4(w[0], w[1], w[2], w[3]);
+              }
+            }
+          }
+        }
+      } else if (EPI == UEPI_RESID) {
+        const float kappa = p.coef[l].kappa;
+        float ss = 0.f;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(tbase + c * 32, r);
+          if (live) {
+            const size_t col = (size_t)n_tile * BN + c * 32;
+            const size_t off = (size_t)l * p.out_ls + (size_t)row * p.N + col;
+            const float4 *xs = reinterpret_cast<const float4 *>(p.xm + (size_t)l * p.xm_ls + (size_t)row * p.N + col);
+            float4 *adst = reinterpret_cast<float4 *>(p.c + off);
+            uint4 *udst = reinterpret_cast<uint4 *>(p.z + off);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               uint32_t w[4];
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                const float a = fmaxf(__uint_as_float(r[8 * j + 2 * q]), 0.f), b = fmaxf(__uint_as_float(r[8 * j + 2 * q + 1]), 0.f);
-                __nv_bfloat162 v = __floats2bfloat162_rn(a * a, b * b);
-                w[q] = *reinterpret_cast<uint32_t *>(&v);
+              for (int q = 0; q < 2; ++q) {
+                const float4 x = xs[2 * j + q];
+                const float a0 = __uint_as_float(r[8 * j + 4 * q]), a1 = __uint_as_float(r[8 * j + 4 * q + 1]);
+                const float a2 = __uint_as_float(r[8 * j + 4 * q + 2]), a3 = __uint_as_float(r[8 * j + 4 * q + 3]);
+                adst[2 * j + q] = make_float4(a0, a1, a2, a3);
+                const float u0 = fmaf(kappa, a0, x.x), u1 = fmaf(kappa, a1, x.y), u2 = fmaf(kappa, a2, x.z), u3 = fmaf(kappa, a3, x.w);
+                ss += u0 * u0 + u1 * u1 + u2 * u2 + u3 * u3;
+                __nv_bfloat162 v0 = __floats2bfloat162_rn(u0, u1), v1 = __floats2bfloat162_rn(u2, u3);
+                w[2 * q] = *reinterpret_cast<uint32_t *>(&v0);
+                w[2 * q + 1] = *reinterpret_cast<uint32_t *>(&v1);
               }
-              dst[j] = make_uint4(w[0], w[1], w[2], w[3]);
+              udst[j] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+        if (live) p.ssq_out[((size_t)l * gridDim.x + n_tile) * p.M + row] = ss;
+      } else {  // UEPI_QKV
+        const int Tn = p.T, b = live ? row / Tn : 0, pos = *p.pos_base + (live ? row % Tn : 0);
+#pragma unroll 1
+        for (int hh = 0; hh < BN / 128; ++hh) {
+          const int n = n_tile * BN + hh * 128, kind = n / p.d, hcol = n % p.d;
+          const uint32_t tcol = tbase + hh * 128;
+          __nv_bfloat16 *dst;
+          if (kind == 0) dst = p.q + (size_t)l * p.q_ls + (size_t)row * p.d + hcol;
+          else dst = (kind == 1 ? p.kc : p.vc) + (size_t)l * p.kv_ls + (size_t)b * p.kv_bs + (size_t)pos * p.d + hcol;
+          if (kind == 2) {
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+              uint32_t r[32];
+              tmem_ld32(tcol + c * 32, r);
+              if (live) {
+                uint4 *o = reinterpret_cast<uint4 *>(dst + c * 32);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  uint32_t w[4];
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[8 * j + 2 * q]) * rstd, __uint_as_float(r[8 * j + 2 * q + 1]) * rstd);
+                    w[q] = *reinterpret_cast<uint32_t *>(&v);
+                  }
+                  o[j] = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+              }
+            }
+          } else {
+            float ss = 0.f;  // rotation preserves the norm, so the head's sum of squares can be taken before it
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+              uint32_t r[32];
+              tmem_ld32(tcol + c * 32, r);
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const float v = __uint_as_float(r[j]) * rstd;
+                ss = fmaf(v, v, ss);
+              }
+            }
+            const float rn = rsqrtf(ss * (1.f / 128.f) + p.qk_eps) * rstd;
+            const float2 *cs = p.rope + (size_t)pos * 64;
+#pragma unroll 1
+            for (int c = 0; c < 2; ++c) {
+              uint32_t lo[32], hi[32];
+              tmem_ld32(tcol + c * 32, lo);
+              tmem_ld32(tcol + 64 + c * 32, hi);
+              if (live) {
+                uint4 *o1 = reinterpret_cast<uint4 *>(dst + c * 32), *o2 = reinterpret_cast<uint4 *>(dst + 64 + c * 32);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  uint32_t w1[4], w2[4];
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    const int i0 = 8 * j + 2 * q;
+                    const float2 ca = cs[c * 32 + i0], cb = cs[c * 32 + i0 + 1];
+                    const float xa1 = __uint_as_float(lo[i0]) * rn, xa2 = __uint_as_float(hi[i0]) * rn;
+                    const float xb1 = __uint_as_float(lo[i0 + 1]) * rn, xb2 = __uint_as_float(hi[i0 + 1]) * rn;
+                    __nv_bfloat162 y1 = __floats2bfloat162_rn(xa1 * ca.x - xa2 * ca.y, xb1 * cb.x - xb2 * cb.y);
+                    __nv_bfloat162 y2 = __floats2bfloat162_rn(xa1 * ca.y + xa2 * ca.x, xb1 * cb.y + xb2 * cb.x);
+                    w1[q] = *reinterpret_cast<uint32_t *>(&y1);
+                    w2[q] = *reinterpret_cast<uint32_t *>(&y2);
+                  }
+                  o1[j] = make_uint4(w1[0], w1[1], w1[2], w1[3]);
+                  o2[j] = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+                }
+              }
             }
           }
         }
