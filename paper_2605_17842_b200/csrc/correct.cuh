@@ -18,8 +18,9 @@ struct CorrParams {
   int mode;          // SNLP_MODE_*
   const HcCoef *coef;
   float *xa, *xm;    // [L][M][d] pre-mapped inputs for the next sweep (n > 1 only)
-  __nv_bfloat16 *xb; // nullable: [L][M][d] bf16 copy of the next sweep's attention-branch input (h_l, or pa_l . x_l)
-  float *ssq_x;      //           [L][d/128][M] its row sums of squares, one partial per 128 columns
+  __nv_bfloat16 *xb; // nullable: [L+1][M][d] bf16 copy of the next sweep's attention-branch input (h_l, or pa_l . x_l);
+                     //           slot L = the LM-head input (sum of the streams of the last state)
+  float *ssq_x;      //           [L+1][d/128][M] its row sums of squares, one partial per 128 columns
   float *partial;    // [gridDim.x][nl][2] scratch for the norms (nullable => no norms)
   float *resnorm;    // [L][2] (entries l0 .. l0+nl-1 written)
   unsigned *counter; // zero on entry, left zero on exit
@@ -115,7 +116,11 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
         reinterpret_cast<float4 *>(p.xm)[(size_t)(l + 1) * Md4 + bm_off] = sm;
         nxt = sa;
       }
-      if (p.xb != nullptr && l + 1 < p.L) {
+      if (NS > 1 && l + 1 == p.L) {  // after the last block: the LM head reads the sum of the streams
+#pragma unroll
+        for (int s = 1; s < NS; ++s) nxt = f4_add(nxt, newn[s]);
+      }
+      if (p.xb != nullptr) {
         __nv_bfloat162 lo = __floats2bfloat162_rn(nxt.x, nxt.y), hi = __floats2bfloat162_rn(nxt.z, nxt.w);
         uint2 pk = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
         reinterpret_cast<uint2 *>(p.xb)[(size_t)(l + 1) * Md4 + bm_off] = pk;
@@ -124,7 +129,7 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
 #pragma unroll
       for (int r = 0; r < NS; ++r) { oldp[r] = oldn[r]; newp[r] = newn[r]; }
     }
-    if (p.xb != nullptr && l + 1 < p.L) {
+    if (p.xb != nullptr) {
       // d is a multiple of 128 here, so the 32 lanes of a warp hold 128 consecutive columns of one row
       xs = warp_sum(xs);
       if (lane == 0 && active) p.ssq_x[((size_t)(l + 1) * (d4 >> 5) + (c4 >> 5)) * p.M + row] = xs;
@@ -187,6 +192,21 @@ __global__ void k_prep_rows(const float *__restrict__ trace, int l0, int M, int 
   if ((threadIdx.x & 31) == 0) ssq_x[((size_t)l * (d4 >> 5) + (c4 >> 5)) * M + row] = ss;
 }
 
+// LM-head input from arbitrary hidden-state rows: xb = bf16(sum of the NS streams), per-128-column sums of squares.
+// grid (rows), d/4 threads.
+__global__ void k_prep_lm(const float *__restrict__ h, size_t row_stride, int nsum, int rows, int d, __nv_bfloat16 *__restrict__ xb,
+                          float *__restrict__ ssq) {
+  const int d4 = d >> 2, c4 = threadIdx.x;
+  const size_t row = blockIdx.x;
+  const float4 *x = reinterpret_cast<const float4 *>(h + row * row_stride) + c4;
+  float4 v = x[0];
+  for (int s = 1; s < nsum; ++s) v = f4_add(v, x[(size_t)s * d4]);
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+  reinterpret_cast<uint2 *>(xb)[row * d4 + c4] = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+  const float ss = warp_sum(f4_sq(v));
+  if ((threadIdx.x & 31) == 0) ssq[(size_t)(c4 >> 5) * rows + row] = ss;
+}
+
 // Latency-oriented variant for the decode regime (a handful of rows): the per-thread loop over
 // layers above serialises ~7 dependent-latency loads per layer, which dominates when there are too
 // few threads to hide it.  Here a block owns 32 float4 columns of one row; its 8 warps first fetch
@@ -232,7 +252,7 @@ __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
   }
   for (int i = 0; i < p.nl; ++i) {
     const int l = p.l0 + i;
-    float rs = 0.f, hs = 0.f;
+    float rs = 0.f, hs = 0.f, xs = 0.f;
     if (active) {
       const float4 av = sa[i * 32 + c], mv = sm[i * 32 + c];
       const HcCoef &cf = p.coef[l];
@@ -270,6 +290,7 @@ __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
         hs += f4_sq(oldn[r]);
         tr4[(size_t)(l + 1) * state4 + st_off + (size_t)r * d4] = newn[r];
       }
+      float4 nxt = newn[0];
       if (NS > 1 && l + 1 < p.L) {
         const HcCoef &cn = p.coef[l + 1];
         float4 xa = f4_scale(cn.pa[0], newn[0]), xm = f4_scale(cn.pmra[0], newn[0]);
@@ -280,9 +301,23 @@ __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
         }
         reinterpret_cast<float4 *>(p.xa)[(size_t)(l + 1) * Md4 + bm_off] = xa;
         reinterpret_cast<float4 *>(p.xm)[(size_t)(l + 1) * Md4 + bm_off] = xm;
+        nxt = xa;
+      }
+      if (NS > 1 && l + 1 == p.L) {
+#pragma unroll
+        for (int s = 1; s < NS; ++s) nxt = f4_add(nxt, newn[s]);
+      }
+      if (p.xb != nullptr) {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(nxt.x, nxt.y), hi = __floats2bfloat162_rn(nxt.z, nxt.w);
+        reinterpret_cast<uint2 *>(p.xb)[(size_t)(l + 1) * Md4 + bm_off] = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+        xs = f4_sq(nxt);
       }
 #pragma unroll
       for (int r = 0; r < NS; ++r) { oldp[r] = oldn[r]; newp[r] = newn[r]; }
+    }
+    if (p.xb != nullptr) {  // this warp holds 128 consecutive columns of the row: partial blockIdx.x
+      xs = warp_sum(xs);
+      if (c == 0) p.ssq_x[((size_t)(l + 1) * gridDim.x + blockIdx.x) * p.M + row] = xs;
     }
     if (want_norm) {
       rs = warp_sum(rs);

@@ -57,7 +57,6 @@ void set_last_error(const char *msg) { g_err = msg; }  // for the library's othe
 // handles
 constexpr int kMaxSplits = 4;    // K-splits of the partial-sum GEMV outputs
 constexpr int kDecodeRows = 16;  // largest row count served by the decode-regime kernels
-constexpr size_t kGemvMaxSmem = 200 * 1024;
 constexpr size_t kCorrSmallSmem = 160 * 1024;
 
 struct GraphKey {
@@ -70,6 +69,7 @@ struct GraphKey {
 };
 struct GraphEntry { cudaGraphExec_t exec; int64_t nodes; };
 struct PendingTime { int cls; cudaEvent_t e0, e1; };
+struct WMap { CUtensorMap tm; int BN; };  // TMA map over one stacked weight array, box {64, BN, 1}
 enum { KC_QKV = 0, KC_ATTN, KC_OPROJ, KC_UP, KC_DOWN, KC_CORRECT, KC_LMHEAD, KC_OTHER, KC_COUNT };
 static_assert(KC_COUNT == SNLP_NUM_KERNEL_CLASSES, "kernel class count");
 
@@ -85,7 +85,7 @@ struct snlp_model {
   // workspace (R = max_rows)
   float *trace = nullptr, *xa = nullptr, *xm = nullptr, *qkv_raw = nullptr, *a = nullptr, *y_raw = nullptr, *mb = nullptr;
   void *ub = nullptr;
-  float *ssq_x = nullptr, *ssq_u = nullptr;
+  float *ssq_x = nullptr, *ssq_u = nullptr, *ssq_lm = nullptr;
   void *xn = nullptr, *q = nullptr, *att = nullptr, *z = nullptr, *sk = nullptr, *sv = nullptr, *xlm = nullptr;
   float *attn_part = nullptr, *corr_part = nullptr, *logits = nullptr, *pm_val = nullptr;
   int *pm_idx = nullptr;
@@ -104,6 +104,9 @@ struct snlp_model {
   bool capturing = false;
   int64_t cap_nodes = 0;
   std::map<GraphKey, GraphEntry> graphs;
+  WMap w_qkv, w_o, w_up, w_dn, w_lm;
+  bool have_wmaps = false;
+  int n_sm = 148;
   EncodeTiledFn encode_tiled = nullptr;  // cuTensorMapEncodeTiled, looked up through the runtime
   int *dev_err = nullptr;                // raised by a kernel whose bounded wait expired
   cudaStream_t cap_stream = nullptr;  // capture target: graphs are recorded here and replayed on the caller's stream
@@ -188,6 +191,8 @@ static int dalloc(snlp_model *m, P **p, size_t bytes) {
 
 static int init_kernel_attributes();
 static bool fused_prefill_ok(const snlp_model *m, int M);
+static bool fast_decode_ok(const snlp_model *m, int M);
+static bool umma_path_ok(const snlp_model *m);
 
 // 64-key sub-blocks per split-KV chunk.  It depends only on how many (layer, sequence, head) triples one
 // launch covers (not on the context length or the number of query rows), so that calls of the same
@@ -197,12 +202,6 @@ static int attn_csub(int triples) {
   int c = 1;
   while (c < 8 && triples >= 16 * c) c *= 2;
   return c;
-}
-
-static bool fast_decode_ok(const snlp_model *m, int M) {
-  const snlp_config &c = m->cfg;
-  return !m->force_generic && c.dtype == SNLP_DTYPE_BF16 && c.head_dim == 128 && M <= kDecodeRows && c.d_model % 128 == 0 &&
-         c.d_ff % 128 == 0 && (c.d_ff / kMaxSplits) % 32 == 0 && (c.d_model / kMaxSplits) % 32 == 0;
 }
 
 extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
@@ -248,11 +247,12 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
   A(&m->a, L * split_rows * d * 4);
   A(&m->y_raw, L * R * ff * 4);
   A(&m->mb, L * split_rows * d * 4);
-  A(&m->xn, L * R * d * es);
+  A(&m->xn, (L + 1) * R * d * es);
   if (c.dtype == SNLP_DTYPE_BF16 && d % 128 == 0) {
     A(&m->ub, L * R * d * es);
-    A(&m->ssq_x, L * (d / 128) * R * 4);
+    A(&m->ssq_x, (L + 1) * (d / 128) * R * 4);
     A(&m->ssq_u, L * (d / 128) * R * 4);
+    A(&m->ssq_lm, (size_t)(d / 128) * kDecodeRows * 4);
   }
   A(&m->q, L * R * d * es);
   A(&m->att, L * R * d * es);
@@ -290,6 +290,10 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
       rc = fail(SNLP_ERR_CUDA, "rotary table upload failed");
   }
   if (rc == SNLP_OK) rc = init_kernel_attributes();
+  if (rc == SNLP_OK) {
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, m->device) == cudaSuccess) m->n_sm = prop.multiProcessorCount;
+  }
   if (rc == SNLP_OK) {
     cudaDriverEntryPointQueryResult qres;
     void *fn = nullptr;
@@ -367,6 +371,15 @@ extern "C" int snlp_load_weights(snlp_model *m, const snlp_weights *w) {
     h.kappa = (float)kappa;
   }
   CU(cudaMemcpy(m->coef, co.data(), L * sizeof(HcCoef), cudaMemcpyHostToDevice));
+  m->have_wmaps = false;
+  if (m->encode_tiled && c.dtype == SNLP_DTYPE_BF16 && d % 128 == 0 && ff % 128 == 0 && V % 128 == 0) {
+    auto mk = [&](WMap &w, const void *base, uint64_t K, uint64_t N, uint64_t layers) {
+      w.BN = N % 256 == 0 ? 256 : 128;
+      return make_tmap_bf16(m->encode_tiled, &w.tm, base, K, N, layers, N * K, w.BN);
+    };
+    m->have_wmaps = mk(m->w_qkv, m->wqkv, d, 3 * d, L) && mk(m->w_o, m->wo, d, d, L) && mk(m->w_up, m->wup, d, ff, L) &&
+                    mk(m->w_dn, m->wdn, ff, d, L) && mk(m->w_lm, m->lm_head, d, V, 1);
+  }
   m->loaded = true;
   return SNLP_OK;
 }
@@ -451,7 +464,7 @@ static int correct(snlp_model *m, const Fwd &f, int l0, int nl, int mode, int a_
   p.coef = m->coef;
   p.xa = m->xa;
   p.xm = m->xm;
-  p.xb = fused_prefill_ok(m, f.M) ? (__nv_bfloat16 *)m->xn : nullptr;
+  p.xb = umma_path_ok(m) ? (__nv_bfloat16 *)m->xn : nullptr;
   p.ssq_x = m->ssq_x;
   p.partial = resnorm ? m->corr_part : nullptr;
   p.resnorm = resnorm;
@@ -512,35 +525,73 @@ static int run_generic(snlp_model *m, const Fwd &f, int l0, int nl, int mode, fl
 }
 
 // Tensor-core GEMM of the prefill regime: C[l] = A[l] (M x K, bf16) * W[l]^T (N x K, bf16), nl layers per launch.
-static bool fused_prefill_ok(const snlp_model *m, int M) {
+// The tensor-core path (both regimes): bf16, head_dim 128, dims in whole 128-column tiles, weight maps built.
+static bool umma_path_ok(const snlp_model *m) {
   const snlp_config &c = m->cfg;
-  return m->encode_tiled && !m->force_generic && c.dtype == SNLP_DTYPE_BF16 && c.head_dim == 128 && M > kDecodeRows &&
-         c.d_model % 128 == 0 && c.d_ff % 128 == 0 && c.d_model <= 4096;
+  return m->have_wmaps && !m->force_generic && c.dtype == SNLP_DTYPE_BF16 && c.head_dim == 128 && c.d_model % 128 == 0 &&
+         c.d_ff % 128 == 0 && c.d_model <= 4096;
+}
+static bool fused_prefill_ok(const snlp_model *m, int M) { return umma_path_ok(m) && M > kDecodeRows; }
+static bool fast_decode_ok(const snlp_model *m, int M) { return umma_path_ok(m) && M <= kDecodeRows; }
+
+// Largest K split <= want whose slices are whole 64-element k-blocks.
+static int pick_ksplit(int K, int want) {
+  for (int s = want; s > 1; --s)
+    if (K % s == 0 && (K / s) % kUmmaBK == 0) return s;
+  return 1;
 }
 
+template <int BN, int AM, int EPI>
+static cudaError_t umma_attr() {
+  return cudaFuncSetAttribute(k_umma_gemm<BN, AM, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<BN, AM>::kSmem);
+}
 template <int EPI>
-static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat16 *A, size_t a_ls, const __nv_bfloat16 *W, size_t w_ls,
-                     UmmaParams p, int M, int N, int K, int nl) {
-  CUtensorMap ta, tb;
-  const int BN = N % 256 == 0 ? 256 : 128;
-  if (!make_tmap_bf16(m->encode_tiled, &ta, A, K, M, nl, a_ls ? a_ls : (size_t)M * K, kUmmaBM) ||
-      !make_tmap_bf16(m->encode_tiled, &tb, W, K, N, nl, w_ls ? w_ls : (size_t)N * K, BN))
-    return fail(SNLP_ERR_CUDA, "cuTensorMapEncodeTiled failed (M=%d N=%d K=%d)", M, N, K);
-  p.M = M; p.N = N; p.K = K; p.err = m->dev_err;
-  dim3 grid(N / BN, (M + kUmmaBM - 1) / kUmmaBM, nl);
-  if (BN == 256) KLAUNCH(m, st, cls, k_umma_gemm<256, EPI><<<grid, kUmmaThreads, UmmaCfg<256>::kSmem, st>>>(ta, tb, p));
-  else KLAUNCH(m, st, cls, k_umma_gemm<128, EPI><<<grid, kUmmaThreads, UmmaCfg<128>::kSmem, st>>>(ta, tb, p));
+static cudaError_t umma_attr_all() {
+  cudaError_t e = umma_attr<128, 128, EPI>();
+  if (e == cudaSuccess) e = umma_attr<256, 128, EPI>();
+  if (e == cudaSuccess) e = umma_attr<128, 16, EPI>();
+  if (e == cudaSuccess) e = umma_attr<256, 16, EPI>();
+  return e;
+}
+
+// C[l] = A[l] (M x K bf16, activations) * W[l0 + l]^T (N x K bf16, stacked weights), nl layers, `ksplit` K slices.
+template <int EPI>
+static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat16 *A, size_t a_ls, const WMap &w, int l0, UmmaParams p,
+                     int M, int N, int K, int ksplit, int nl) {
+  const bool small = M <= kDecodeRows;
+  if (EPI == UEPI_LMHEAD && !small) return fail(SNLP_ERR_UNSUPPORTED, "LM-head epilogue needs <= %d rows", kDecodeRows);
+  CUtensorMap ta;
+  if (!make_tmap_bf16(m->encode_tiled, &ta, A, K, M, nl, a_ls ? a_ls : (size_t)M * K, small ? 16 : kUmmaBM))
+    return fail(SNLP_ERR_CUDA, "cuTensorMapEncodeTiled failed (M=%d K=%d)", M, K);
+  p.M = M; p.N = N; p.K = K; p.ksplit = ksplit; p.kslice = K / ksplit;
+  p.Mt = small ? 1 : (M + kUmmaBM - 1) / kUmmaBM; p.Nt = N / w.BN; p.nl = nl; p.l0 = l0; p.err = m->dev_err;
+  const int items = p.Mt * p.Nt * ksplit * nl;
+  const int grid = items < m->n_sm ? items : m->n_sm;
+#define SNLP_UMMA_LAUNCH(BN_, AM_)                                                                                                   \
+  do {                                                                                                                               \
+    p.nstages = UmmaCfg<BN_, AM_>::kStages;                                                                                          \
+    KLAUNCH(m, st, cls, k_umma_gemm<BN_, AM_, EPI><<<grid, kUmmaThreads, UmmaCfg<BN_, AM_>::kSmem, st>>>(ta, w.tm, p));              \
+  } while (0)
+  if (w.BN == 256) {
+    if (small) SNLP_UMMA_LAUNCH(256, 16);
+    else if (EPI != UEPI_LMHEAD) SNLP_UMMA_LAUNCH(256, 128);
+  } else {
+    if (small) SNLP_UMMA_LAUNCH(128, 16);
+    else if (EPI != UEPI_LMHEAD) SNLP_UMMA_LAUNCH(128, 128);
+  }
+#undef SNLP_UMMA_LAUNCH
   return SNLP_OK;
 }
 
-// Prefill-regime sweep over layers l0 .. l0+nl-1 (bf16, head_dim 128, more than 16 rows): six launches.
-// The four projections run on the tcgen05 tensor-core GEMM with everything else of the block fused into
-// their epilogues (row RMSNorm as a scale, rotary + QK-norm + KV store, residual add + sum of squares,
-// ReLU^2); the bf16 branch inputs xb/ssq_x of the range must be current (k_prep_rows or the last correction).
-static int run_prefill(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float *resnorm) {
+// One sweep over layers l0 .. l0+nl-1 on the tensor-core path: six launches whatever nl.
+// The four projections run on k_umma_gemm with the rest of the block fused into their epilogues (row RMSNorm
+// as a scale, rotary + QK-norm + KV store, residual add + sum of squares, ReLU^2); the bf16 branch inputs
+// xb/ssq_x of the range must be current (prep_rows, or the previous correction).
+static int run_umma(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float *resnorm) {
   typedef __nv_bfloat16 T;
   const snlp_config &c = m->cfg;
-  const int M = f.M, d = c.d_model, ff = c.d_ff, H = c.n_head, n = c.n_streams, P = d / 128;
+  const int M = f.M, d = c.d_model, ff = c.d_ff, H = c.n_head, n = c.n_streams, P = d / 128, L = c.n_layer;
+  const bool small = M <= kDecodeRows;
   const size_t Md = (size_t)M * d;
   cudaStream_t st = f.st;
   const float *xm_src = n == 1 ? m->trace + l0 * Md : m->xm + l0 * Md;
@@ -548,37 +599,46 @@ static int run_prefill(snlp_model *m, const Fwd &f, int l0, int nl, int mode, fl
   T *z = (T *)m->z + (size_t)l0 * M * ff;
   float *a = m->a + l0 * Md, *mb = m->mb + l0 * Md;
   T *kc = (T *)f.kc + (size_t)l0 * f.kv_ls, *vc = (T *)f.vc + (size_t)l0 * f.kv_ls;
-  const int Pu = d / (d % 256 == 0 ? 256 : 128);  // column tiles of the out-projection = partials of sum u^2
+  const int Pu = d / m->w_o.BN;  // column tiles of the out-projection = partials of sum u^2
+  // K split of the down-projection: only worth it when a launch has too few items to occupy the GPU
+  const int sd = (small && nl * (d / m->w_dn.BN) < m->n_sm / 2) ? pick_ksplit(ff, kMaxSplits) : 1;
   {
     UmmaParams p{};
     p.ssq = m->ssq_x + (size_t)l0 * P * M; p.nparts = P; p.eps = c.rms_eps;
     p.q = q; p.q_ls = Md; p.kc = kc; p.vc = vc; p.kv_ls = f.kv_ls; p.kv_bs = f.kv_bs;
     p.T = f.T; p.d = d; p.pos_base = f.pos; p.rope = m->rope; p.qk_eps = c.rms_eps;
-    TRY(umma_gemm<UEPI_QKV>(m, st, KC_QKV, xb, Md, (const T *)m->wqkv + (size_t)l0 * 3 * d * d, (size_t)3 * d * d, p, M, 3 * d, d, nl));
+    TRY(umma_gemm<UEPI_QKV>(m, st, KC_QKV, xb, Md, m->w_qkv, l0, p, M, 3 * d, d, 1, nl));
   }
-  KLAUNCH(m, st, KC_ATTN, k_attn_prefill<<<dim3((f.T + kFaRows - 1) / kFaRows, f.B * H, nl), 128, kFaSmem, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, att, Md,
-                                                                                                  f.T, H, f.pos));
+  if (small) {
+    const int csub = attn_csub(nl * f.B * H);
+    const int nchunk = (f.pos_hi + f.T - 1) / (csub * kAttnSub) + 1;
+    KLAUNCH(m, st, KC_ATTN, k_attn_decode<<<dim3(nchunk, f.B * H, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, m->attn_part, m->attn_counters, att, Md,
+                                                                            f.T, H, f.pos, csub));
+  } else {
+    KLAUNCH(m, st, KC_ATTN, k_attn_prefill<<<dim3((f.T + kFaRows - 1) / kFaRows, f.B * H, nl), 128, kFaSmem, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, att, Md,
+                                                                                                    f.T, H, f.pos));
+  }
   {
     UmmaParams p{};
     p.c = a; p.z = ub; p.out_ls = Md;
     p.xm = xm_src; p.xm_ls = Md; p.coef = m->coef + l0; p.ssq_out = m->ssq_u + (size_t)l0 * Pu * M;
-    TRY(umma_gemm<UEPI_RESID>(m, st, KC_OPROJ, att, Md, (const T *)m->wo + (size_t)l0 * d * d, (size_t)d * d, p, M, d, d, nl));
+    TRY(umma_gemm<UEPI_RESID>(m, st, KC_OPROJ, att, Md, m->w_o, l0, p, M, d, d, 1, nl));
   }
   {
     UmmaParams p{};
     p.z = z; p.out_ls = (size_t)M * ff;
     p.ssq = m->ssq_u + (size_t)l0 * Pu * M; p.nparts = Pu; p.eps = c.rms_eps;
-    TRY(umma_gemm<UEPI_RELU2_BF16>(m, st, KC_UP, ub, Md, (const T *)m->wup + (size_t)l0 * ff * d, (size_t)ff * d, p, M, ff, d, nl));
+    TRY(umma_gemm<UEPI_RELU2_BF16>(m, st, KC_UP, ub, Md, m->w_up, l0, p, M, ff, d, 1, nl));
   }
   {
     UmmaParams p{};
-    p.c = mb; p.out_ls = Md;
-    TRY(umma_gemm<UEPI_F32>(m, st, KC_DOWN, z, (size_t)M * ff, (const T *)m->wdn + (size_t)l0 * d * ff, (size_t)d * ff, p, M, d, ff, nl));
+    p.c = mb; p.out_ls = Md; p.out_ss = (size_t)L * Md;
+    TRY(umma_gemm<UEPI_F32>(m, st, KC_DOWN, z, (size_t)M * ff, m->w_dn, l0, p, M, d, ff, sd, nl));
   }
-  return correct(m, f, l0, nl, mode, 1, 1, resnorm);
+  return correct(m, f, l0, nl, mode, 1, sd, resnorm);
 }
 
-// bf16 branch inputs of layers l0 .. l0+nl-1 for run_prefill (and the fp32 MLP pre-map of mHC models)
+// bf16 branch inputs of layers l0 .. l0+nl-1 for run_umma (and the fp32 MLP pre-map of mHC models)
 static int prep_rows(snlp_model *m, const Fwd &f, int l0, int nl) {
   const snlp_config &c = m->cfg;
   dim3 grid(f.M, nl);
@@ -591,38 +651,13 @@ static int prep_rows(snlp_model *m, const Fwd &f, int l0, int nl) {
   return SNLP_OK;
 }
 
-template <int PRO, int EPI>
-static int launch_gemv(snlp_model *m, cudaStream_t st, int cls, GemvParams &p, int ksplit, int nl) {
-  const int NT = p.M <= 8 ? 1 : 2;
-  p.kslice = p.Kd / ksplit;
-  const size_t sm = (size_t)NT * 8 * (p.kslice + kGemvPad) * 2 + (size_t)NT * 8 * (kGemvRows + 1) * 4 + 16 * 4;
-  if (sm > kGemvMaxSmem) return fail(SNLP_ERR_UNSUPPORTED, "gemv: K slice of %d needs %zu bytes of shared memory", p.kslice, sm);
-  dim3 grid(p.N / kGemvRows, ksplit, nl);
-  KLAUNCH(m, st, cls, if (NT == 1) k_gemv_mma<1, PRO, EPI><<<grid, kGemvThreads, sm, st>>>(p);
-  else k_gemv_mma<2, PRO, EPI><<<grid, kGemvThreads, sm, st>>>(p));
-  return SNLP_OK;
-}
-
-template <int PRO, int EPI>
-static cudaError_t gemv_attr() {
-  cudaError_t e = cudaFuncSetAttribute(k_gemv_mma<1, PRO, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemvMaxSmem);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_gemv_mma<2, PRO, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemvMaxSmem);
-}
-
 static int init_kernel_attributes() {
-  CU((gemv_attr<PRO_NORM, EPI_QKV>()));
-  CU((gemv_attr<PRO_BF16, EPI_PARTIAL>()));
-  CU((gemv_attr<PRO_RESID_NORM, EPI_RELU2>()));
-  CU((gemv_attr<PRO_NORM, EPI_LMHEAD>()));
-  CU(cudaFuncSetAttribute(k_umma_gemm<128, UEPI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<128>::kSmem));
-  CU(cudaFuncSetAttribute(k_umma_gemm<256, UEPI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<256>::kSmem));
-  CU(cudaFuncSetAttribute(k_umma_gemm<128, UEPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<128>::kSmem));
-  CU(cudaFuncSetAttribute(k_umma_gemm<256, UEPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<256>::kSmem));
-  CU(cudaFuncSetAttribute(k_umma_gemm<128, UEPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<128>::kSmem));
-  CU(cudaFuncSetAttribute(k_umma_gemm<256, UEPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<256>::kSmem));
-  CU(cudaFuncSetAttribute(k_umma_gemm<128, UEPI_RELU2_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<128>::kSmem));
-  CU(cudaFuncSetAttribute(k_umma_gemm<256, UEPI_RELU2_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<256>::kSmem));
+  CU(umma_attr_all<UEPI_F32>());
+  CU(umma_attr_all<UEPI_RELU2_BF16>());
+  CU(umma_attr_all<UEPI_QKV>());
+  CU(umma_attr_all<UEPI_RESID>());
+  CU((umma_attr<128, 16, UEPI_LMHEAD>()));
+  CU((umma_attr<256, 16, UEPI_LMHEAD>()));
   CU(cudaFuncSetAttribute(k_attn_prefill, cudaFuncAttributeMaxDynamicSharedMemorySize, kFaSmem));
   CU(cudaFuncSetAttribute(k_correct_small<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
   CU(cudaFuncSetAttribute(k_correct_small<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
@@ -631,63 +666,8 @@ static int init_kernel_attributes() {
   return SNLP_OK;
 }
 
-// Decode-regime sweep over layers l0 .. l0+nl-1 (bf16, <= 16 rows): 7 launches independent of nl.
-static int run_decode(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float *resnorm) {
-  typedef __nv_bfloat16 bf;
-  const snlp_config &c = m->cfg;
-  const int M = f.M, d = c.d_model, ff = c.d_ff, H = c.n_head, n = c.n_streams, L = c.n_layer;
-  const size_t Md = (size_t)M * d;
-  cudaStream_t st = f.st;
-  const float *xa_src = n == 1 ? m->trace + l0 * Md : m->xa + l0 * Md;
-  const float *xm_src = n == 1 ? m->trace + l0 * Md : m->xm + l0 * Md;
-  bf *q = (bf *)m->q + l0 * Md, *att = (bf *)m->att + l0 * Md, *z = (bf *)m->z + (size_t)l0 * M * ff;
-  bf *kc = (bf *)f.kc + (size_t)l0 * f.kv_ls, *vc = (bf *)f.vc + (size_t)l0 * f.kv_ls;
-  const int so = d >= 1024 ? 2 : 1;          // K-splits of the out-projection
-  const int sd = kMaxSplits;                 // K-splits of the down-projection
-  {
-    GemvParams p{};
-    p.W = (const bf *)m->wqkv + (size_t)l0 * 3 * d * d; p.w_ls = (size_t)3 * d * d;
-    p.N = 3 * d; p.Kd = d; p.M = M;
-    p.xf = xa_src; p.xf_ls = Md; p.xf_rs = d; p.nsum = 1; p.eps = c.rms_eps;
-    p.q = q; p.q_ls = Md; p.kc = kc; p.vc = vc; p.kv_ls = f.kv_ls; p.kv_bs = f.kv_bs;
-    p.T = f.T; p.H = H; p.pos_base = f.pos; p.rope = m->rope; p.qk_eps = c.rms_eps;
-    TRY((launch_gemv<PRO_NORM, EPI_QKV>(m, st, KC_QKV, p, 1, nl)));
-  }
-  const int csub = attn_csub(nl * f.B * H);
-  const int nchunk = (f.pos_hi + f.T - 1) / (csub * kAttnSub) + 1;
-  KLAUNCH(m, st, KC_ATTN, k_attn_decode<<<dim3(nchunk, f.B * H, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, m->attn_part, m->attn_counters, att, Md,
-                                                                          f.T, H, f.pos, csub));
-  {
-    GemvParams p{};
-    p.W = (const bf *)m->wo + (size_t)l0 * d * d; p.w_ls = (size_t)d * d;
-    p.N = d; p.Kd = d; p.M = M;
-    p.xb = att; p.xb_ls = Md;
-    p.out = m->a + l0 * Md; p.out_ls = Md; p.out_ss = (size_t)L * Md;
-    TRY((launch_gemv<PRO_BF16, EPI_PARTIAL>(m, st, KC_OPROJ, p, so, nl)));
-  }
-  {
-    GemvParams p{};
-    p.W = (const bf *)m->wup + (size_t)l0 * ff * d; p.w_ls = (size_t)ff * d;
-    p.N = ff; p.Kd = d; p.M = M;
-    p.xf = xm_src; p.xf_ls = Md; p.xf_rs = d; p.nsum = 1; p.eps = c.rms_eps;
-    p.ap = m->a + l0 * Md; p.ap_ls = Md; p.ap_ss = (size_t)L * Md; p.ap_splits = so; p.coef = m->coef + l0;
-    p.zout = z; p.z_ls = (size_t)M * ff;
-    TRY((launch_gemv<PRO_RESID_NORM, EPI_RELU2>(m, st, KC_UP, p, 1, nl)));
-  }
-  {
-    GemvParams p{};
-    p.W = (const bf *)m->wdn + (size_t)l0 * d * ff; p.w_ls = (size_t)d * ff;
-    p.N = d; p.Kd = ff; p.M = M;
-    p.xb = z; p.xb_ls = (size_t)M * ff;
-    p.out = m->mb + l0 * Md; p.out_ls = Md; p.out_ss = (size_t)L * Md;
-    TRY((launch_gemv<PRO_BF16, EPI_PARTIAL>(m, st, KC_DOWN, p, sd, nl)));
-  }
-  return correct(m, f, l0, nl, mode, so, sd, resnorm);
-}
-
 static int run_layers(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float *resnorm) {
-  if (fast_decode_ok(m, f.M)) return run_decode(m, f, l0, nl, mode, resnorm);
-  if (fused_prefill_ok(m, f.M)) return run_prefill(m, f, l0, nl, mode, resnorm);
+  if (umma_path_ok(m)) return run_umma(m, f, l0, nl, mode, resnorm);
   if (m->cfg.dtype == SNLP_DTYPE_BF16) return run_generic<__nv_bfloat16>(m, f, l0, nl, mode, resnorm);
   return run_generic<float>(m, f, l0, nl, mode, resnorm);
 }
@@ -705,7 +685,7 @@ static int premix(snlp_model *m, const Fwd &f, int l0, int nl) {
 
 // Alg. 1 over the internal trace (trace[0] must hold h_0).
 static int sequential(snlp_model *m, const Fwd &f) {
-  if (fused_prefill_ok(m, f.M)) TRY(prep_rows(m, f, 0, 1));
+  if (umma_path_ok(m)) TRY(prep_rows(m, f, 0, 1));
   else TRY(premix(m, f, 0, 1));
   for (int l = 0; l < m->cfg.n_layer; ++l) TRY(run_layers(m, f, l, 1, native_mode(m), nullptr));
   return SNLP_OK;
@@ -717,26 +697,31 @@ static int parallel(snlp_model *m, const Fwd &f, int K, int mode, float *resnorm
   const size_t n4 = (size_t)f.M * c.n_streams * c.d_model / 4;
   KLAUNCH(m, f.st, KC_OTHER, k_bcast_trace<<<(unsigned)((n4 + 255) / 256), 256, 0, f.st>>>(reinterpret_cast<const float4 *>(m->trace),
                                                                reinterpret_cast<float4 *>(m->trace) + n4, n4, c.n_layer));
-  if (fused_prefill_ok(m, f.M)) TRY(prep_rows(m, f, 0, c.n_layer));
+  if (umma_path_ok(m)) TRY(prep_rows(m, f, 0, c.n_layer));
   else TRY(premix(m, f, 0, c.n_layer));
   for (int k = 0; k < K; ++k)
     TRY(run_layers(m, f, 0, c.n_layer, mode, resnorm_out ? resnorm_out + (size_t)k * c.n_layer * 2 : nullptr));
   return SNLP_OK;
 }
 
-static int lm_head_impl(snlp_model *m, cudaStream_t st, const float *hL, size_t row_stride, int rows, float *logits, int32_t *argmax) {
+// LMHead on `rows` hidden states.  pre_xb / pre_ssq: the bf16 stream-summed rows and their sums of squares if the
+// caller already has them (slot L of the branch-input buffers after a decode-regime forward), else NULL.
+static int lm_head_impl(snlp_model *m, cudaStream_t st, const float *hL, size_t row_stride, int rows, float *logits, int32_t *argmax,
+                        const __nv_bfloat16 *pre_xb = nullptr, const float *pre_ssq = nullptr) {
   const snlp_config &c = m->cfg;
   const int d = c.d_model, V = c.vocab, n = c.n_streams;
-  if (!m->force_generic && c.dtype == SNLP_DTYPE_BF16 && rows <= kDecodeRows && d % 32 == 0 && V % 128 == 0) {
-    GemvParams p{};
-    p.W = (const __nv_bfloat16 *)m->lm_head; p.w_ls = 0;
-    p.N = V; p.Kd = d; p.M = rows;
-    p.xf = hL; p.xf_ls = 0; p.xf_rs = row_stride; p.nsum = n; p.eps = c.rms_eps;
-    p.logits = logits; p.pm_val = m->pm_val; p.pm_idx = m->pm_idx; p.ntile = V / 128;
-    TRY((launch_gemv<PRO_NORM, EPI_LMHEAD>(m, st, KC_LMHEAD, p, 1, 1)));
-    if (argmax) {
-      KLAUNCH(m, st, KC_LMHEAD, k_argmax_tiles<<<rows, 256, 0, st>>>(m->pm_val, m->pm_idx, V / 128, argmax));
+  if (umma_path_ok(m) && rows <= kDecodeRows) {
+    const int P = d / 128;
+    if (!pre_xb) {
+      KLAUNCH(m, st, KC_LMHEAD, k_prep_lm<<<rows, d / 4, 0, st>>>(hL, row_stride, n, rows, d, (__nv_bfloat16 *)m->xlm, m->ssq_lm));
+      pre_xb = (const __nv_bfloat16 *)m->xlm;
+      pre_ssq = m->ssq_lm;
     }
+    UmmaParams p{};
+    p.ssq = pre_ssq; p.nparts = P; p.eps = c.rms_eps;
+    p.logits = logits; p.pm_val = m->pm_val; p.pm_idx = m->pm_idx;
+    TRY(umma_gemm<UEPI_LMHEAD>(m, st, KC_LMHEAD, pre_xb, 0, m->w_lm, 0, p, rows, V, d, 1, 1));
+    if (argmax) KLAUNCH(m, st, KC_LMHEAD, k_argmax_tiles<<<rows, 256, 0, st>>>(m->pm_val, m->pm_idx, V / m->w_lm.BN, argmax));
     return SNLP_OK;
   }
   for (int r0 = 0; r0 < rows; r0 += m->logit_rows) {
@@ -939,6 +924,16 @@ extern "C" int snlp_prefill(snlp_model *m, snlp_kv *kv, const int32_t *ids, int 
   return SNLP_OK;
 }
 
+// greedy tokens of all `rows` rows of the forward that just ran (rows <= 16)
+static int lm_head_tail(snlp_model *m, cudaStream_t st, int rows, int32_t *argmax) {
+  const snlp_config &c = m->cfg;
+  const size_t nd = (size_t)c.n_streams * c.d_model, L = c.n_layer;
+  if (umma_path_ok(m) && rows <= kDecodeRows)  // the correction left the LM-head input in slot L of xb / ssq_x
+    return lm_head_impl(m, st, nullptr, 0, rows, nullptr, argmax, (const __nv_bfloat16 *)m->xn + L * rows * c.d_model,
+                        m->ssq_x + L * (c.d_model / 128) * rows);
+  return lm_head_impl(m, st, m->trace + L * rows * nd, nd, rows, nullptr, argmax);
+}
+
 // enqueue one decode step (no graph handling, no host-side length update)
 static int decode_launches(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, int K, int mode, int32_t *tok_out, float *resnorm_out,
                            cudaStream_t st) {
@@ -948,7 +943,7 @@ static int decode_launches(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, in
   if (K == 0) TRY(sequential(m, f));
   else TRY(parallel(m, f, K, mode, resnorm_out));
   const size_t nd = (size_t)c.n_streams * c.d_model;
-  TRY(lm_head_impl(m, st, m->trace + (size_t)c.n_layer * kv->B * nd, nd, kv->B, nullptr, tok_out));
+  TRY(lm_head_tail(m, st, kv->B, tok_out));
   KLAUNCH(m, st, KC_OTHER, k_add_int<<<1, 1, 0, st>>>(kv->pos, 1));
   return SNLP_OK;
 }
@@ -1029,7 +1024,7 @@ extern "C" int snlp_draft_and_verify(snlp_model *m, snlp_kv *kv, int32_t *last_t
   Fwd f = kv_fwd(m, kv, block + 1, st);
   TRY(sequential(m, f));
   const size_t nd = (size_t)c.n_streams * c.d_model;
-  TRY(lm_head_impl(m, st, m->trace + (size_t)c.n_layer * (block + 1) * nd, nd, block + 1, nullptr, y));
+  TRY(lm_head_tail(m, st, block + 1, y));
   KLAUNCH(m, st, KC_OTHER, k_accept<<<1, 32, 0, st>>>(ids + 1, y, block, emitted, n_emitted, n_accepted, last_tok, kv->pos, len0));
   int32_t n = 0;
   CU(cudaMemcpyAsync(&n, n_accepted, 4, cudaMemcpyDeviceToHost, st));

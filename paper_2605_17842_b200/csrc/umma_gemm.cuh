@@ -1,11 +1,19 @@
-// Prefill-regime layer-batched GEMM on the 5th-generation tensor cores (sm_100a):
-//   D[l][m][n] = sum_k A[l][m][k] * B[l][n][k]     A = activations [L][M][K] bf16, B = weights [L][N][K] bf16
-// One CTA computes a 128 x BN tile of one layer.  Operand tiles (128 x 64 and BN x 64 bf16, 128-byte
-// swizzle) are brought into a shared-memory ring by TMA (one elected thread), a second elected thread
-// issues tcgen05.mma (UMMA 128 x BN x 16, fp32 accumulator in tensor memory) and releases ring slots with
-// tcgen05.commit; four epilogue warps read the accumulator back with tcgen05.ld and apply the fused
-// epilogue.  Every wait on an mbarrier is bounded: on expiry the kernel raises a flag in global memory,
-// lets its copies in flight land, frees its tensor memory and returns.
+// Layer-batched grouped GEMM on the 5th-generation tensor cores (sm_100a), used by both regimes:
+//   D[l][m][n] = sum_k A[l][m][k] * W[l][n][k]     A = activations [nl][M][K] bf16, W = stacked weights [L][N][K] bf16
+// Persistent CTAs (one per SM) walk (row tile, column tile, K split, layer) items.  Operand tiles -- AM x 64
+// activations and BN x 64 weights, 128-byte swizzle -- are brought into a shared-memory ring by TMA (one
+// elected thread) that keeps running across item boundaries; a second elected thread issues tcgen05.mma
+// (UMMA 128 x BN x 16, fp32 accumulators in tensor memory, two accumulators so the epilogue of one item
+// overlaps the main loop of the next) and releases ring slots with tcgen05.commit; four epilogue warps read
+// the accumulator back with tcgen05.ld and apply the fused epilogue.
+//   AM = 128: prefill regime, one accumulator row per epilogue thread.
+//   AM = 16 : decode regime (<= 16 rows).  The weights stay the 256-wide operand -- a tcgen05.mma costs the
+//             same ~155 cycles whatever its shape, so streaming needs 8 KB of weights per instruction -- and
+//             the token box is only 16 rows high (rows 16..127 of the A operand are whatever follows in shared
+//             memory and land in accumulator rows nobody reads).  The kernel is then bound by the weight stream
+//             from HBM; the accumulator is transposed through shared memory so all 128 epilogue threads work.
+// Every wait on an mbarrier is bounded: on expiry the kernel raises a flag in global memory, lets its
+// copies in flight land, frees its tensor memory and returns.
 #pragma once
 #include <cuda.h>
 
@@ -13,36 +21,39 @@
 
 namespace snlp {
 
-// Epilogues.  The A operand of the QKV and MLP-up products is the *un-normalised* bf16 branch input; its
-// RMSNorm is a per-row scalar, so it is applied to the accumulator row here (sum of squares of the row =
+// Epilogues.  The A operand of the QKV, MLP-up and LM-head products is the *un-normalised* bf16 branch input;
+// its RMSNorm is a per-row scalar, so it is applied to the accumulator row here (sum of squares of the row =
 // sum of `nparts` partials written by the producing kernel, in fixed order).
-//   UEPI_F32         c = acc
-//   UEPI_RELU2_BF16  z = bf16(relu(rstd_row * acc)^2)                      (rstd_row = 1 if ssq == nullptr)
+//   UEPI_F32         c[ks] = acc                                           (K-split partial sums)
+//   UEPI_RELU2_BF16  z = bf16(relu(rstd_row * acc)^2)
 //   UEPI_QKV         per 128-wide head: y = rstd_row * acc; q,k: rotary + RMSNorm over the head; q -> q buffer,
 //                    k,v -> the layer's key/value store at the row's position
-//   UEPI_RESID       u = xm + kappa_l * acc;  a = acc (fp32, for the correction), ub = bf16(u), and the partial
-//                    sum of u^2 over this CTA's BN columns -> ssq_out[l][n_tile][row]
-enum { UEPI_F32 = 0, UEPI_RELU2_BF16 = 1, UEPI_QKV = 2, UEPI_RESID = 3 };
+//   UEPI_RESID       u = xm + kappa_l * acc;  c = acc (fp32, for the correction), z = bf16(u), and the partial
+//                    sum of u^2 over this tile's BN columns -> ssq_out[l][n_tile][row]
+//   UEPI_LMHEAD      v = rstd_row * acc; optional logits; per-tile argmax -> pm_val/pm_idx[row][n_tile]   (AM = 16 only)
+enum { UEPI_F32 = 0, UEPI_RELU2_BF16 = 1, UEPI_QKV = 2, UEPI_RESID = 3, UEPI_LMHEAD = 4 };
 
 struct UmmaParams {
   int M, N, K;             // rows, columns, reduction length of one layer's product
-  float *c;                // UEPI_F32 / UEPI_RESID: [nl][M][N] fp32
-  __nv_bfloat16 *z;        // UEPI_RELU2_BF16: [nl][M][N] bf16;  UEPI_RESID: ub [nl][M][N] bf16
-  size_t out_ls;           // layer stride of the outputs above (elements)
+  int kslice, ksplit;      // K split: kslice = K / ksplit (a multiple of 64)
+  int Mt, Nt, nl, l0;      // row tiles, column tiles, layers of the launch; l0 = first layer's coordinate in the weight map
+  int nstages;             // ring depth
+  float *c;                // UEPI_F32 / UEPI_RESID: [ksplit][nl][M][N] fp32
+  __nv_bfloat16 *z;        // UEPI_RELU2_BF16: [nl][M][N] bf16;  UEPI_RESID: bf16(u) [nl][M][N]
+  size_t out_ls, out_ss;   // layer / split stride of the outputs above (elements)
   int *err;                // device flag set to 1 when a bounded wait expires
-  // row scale (UEPI_QKV, UEPI_RELU2_BF16)
-  const float *ssq; int nparts; float eps;   // [nl][nparts][M] partial sums of squares of the A rows
-  // UEPI_QKV
-  __nv_bfloat16 *q; size_t q_ls;
+  const float *ssq; int nparts; float eps;   // row scale: [nl][nparts][M] partial sums of squares of the A rows
+  __nv_bfloat16 *q; size_t q_ls;             // UEPI_QKV
   __nv_bfloat16 *kc, *vc; size_t kv_ls, kv_bs;
   int T, d; const int *pos_base; const float2 *rope; float qk_eps;
-  // UEPI_RESID
-  const float *xm; size_t xm_ls; const HcCoef *coef; float *ssq_out;   // ssq_out [nl][N/BN][M]
+  const float *xm; size_t xm_ls; const HcCoef *coef; float *ssq_out;   // UEPI_RESID; ssq_out [nl][Nt][M]
+  float *logits; float *pm_val; int *pm_idx;                            // UEPI_LMHEAD
 };
 
 constexpr int kUmmaThreads = 192;   // warp 0: TMA, warp 1: MMA + TMEM allocation, warps 2-5: epilogue
 constexpr int kUmmaBM = 128;
 constexpr int kUmmaBK = 64;         // 64 bf16 = one 128-byte swizzle row
+constexpr int kUmmaSmemBudget = 222 * 1024;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -58,6 +69,9 @@ __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
   uint32_t ok;
@@ -130,6 +144,18 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// Barrier over the 128 epilogue threads (named barrier 1), plain and with an AND-reduced predicate: after a
+// bounded wait every thread learns whether all of them got through, so they leave the item loop together.
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ bool epi_all(bool v) {
+  uint32_t out;
+  asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 q, %1, 0;\n bar.red.and.pred p, 1, 128, q;\n selp.b32 %0, 1, 0, p;\n}"
+               : "=r"(out)
+               : "r"((uint32_t)v)
+               : "memory");
+  return out != 0;
+}
+
 // Shared-memory matrix descriptor for a K-major operand tile stored as rows of 128 bytes with the
 // 128-byte swizzle (what TMA writes): 8-row groups are 1024 bytes apart.
 __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
@@ -147,46 +173,286 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-template <int BN>
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+
+template <int BN, int AM>
 struct UmmaCfg {
-  static constexpr int kStages = BN == 256 ? 4 : 6;
-  static constexpr int kABytes = kUmmaBM * kUmmaBK * 2;
+  static constexpr int kABytes = AM * kUmmaBK * 2;
   static constexpr int kBBytes = BN * kUmmaBK * 2;
-  static constexpr int kSmem = kStages * (kABytes + kBBytes) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int kOuts = AM == 16 ? 16 * (BN + 1) * 4 : 0;   // transposed accumulator of the decode regime
+  static constexpr int kFixed = kOuts + 1024 /*alignment slack*/ + 512 /*barriers*/;
+  static constexpr int kStagesMax = (kUmmaSmemBudget - kFixed) / (kABytes + kBBytes);
+  static constexpr int kStages = kStagesMax > 10 ? 10 : kStagesMax;
+  static constexpr int kSmem = kStages * (kABytes + kBBytes) + kFixed;
 };
 
-// grid (N/BN, ceil(M/128), nl), 192 threads, dynamic shared memory UmmaCfg<BN>::kSmem.
-// tmA: 3-D map over A {K, M, nl}, box {64, 128, 1}; tmB: 3-D map over B {K, N, nl}, box {64, BN, 1}; both
-// bf16, 128-byte swizzle, out-of-range rows read as zero.
+// ---- epilogue of the prefill regime: thread = accumulator row ----------------------------------------
 template <int BN, int EPI>
-__global__ void __launch_bounds__(kUmmaThreads) k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                                                           UmmaParams p) {
-  using Cfg = UmmaCfg<BN>;
+__device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t tbase, int row, int n_tile, int ks, int l) {
+  const bool live = row < p.M;
+  float rstd = 1.f;
+  if ((EPI == UEPI_QKV || EPI == UEPI_RELU2_BF16) && p.ssq != nullptr && live) {
+    float ss = 0.f;
+    for (int i = 0; i < p.nparts; ++i) ss += p.ssq[((size_t)l * p.nparts + i) * p.M + row];
+    rstd = rsqrtf(ss / (float)p.K + p.eps);
+  }
+  if (EPI == UEPI_F32 || EPI == UEPI_RELU2_BF16) {
+#pragma unroll 1
+    for (int c = 0; c < BN / 32; ++c) {
+      uint32_t r[32];
+      tmem_ld32(tbase + c * 32, r);
+      if (live) {
+        const size_t off = (size_t)l * p.out_ls + (size_t)row * p.N + (size_t)n_tile * BN + c * 32;
+        if (EPI == UEPI_F32) {
+          float4 *dst = reinterpret_cast<float4 *>(p.c + (size_t)ks * p.out_ss + off);
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                                 __uint_as_float(r[4 * j + 3]));
+        } else {
+          uint4 *dst = reinterpret_cast<uint4 *>(p.z + off);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint32_t w[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float a = fmaxf(__uint_as_float(r[8 * j + 2 * q]) * rstd, 0.f);
+              const float b = fmaxf(__uint_as_float(r[8 * j + 2 * q + 1]) * rstd, 0.f);
+              w[q] = pack_bf16x2(a * a, b * b);
+            }
+            dst[j] = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+    }
+  } else if (EPI == UEPI_RESID) {
+    const float kappa = p.coef[l].kappa;
+    float ss = 0.f;
+#pragma unroll 1
+    for (int c = 0; c < BN / 32; ++c) {
+      uint32_t r[32];
+      tmem_ld32(tbase + c * 32, r);
+      if (live) {
+        const size_t col = (size_t)n_tile * BN + c * 32;
+        const size_t off = (size_t)l * p.out_ls + (size_t)row * p.N + col;
+        const float4 *xs = reinterpret_cast<const float4 *>(p.xm + (size_t)l * p.xm_ls + (size_t)row * p.N + col);
+        float4 *adst = reinterpret_cast<float4 *>(p.c + off);
+        uint4 *udst = reinterpret_cast<uint4 *>(p.z + off);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          uint32_t w[4];
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            const float4 x = xs[2 * j + q];
+            const float a0 = __uint_as_float(r[8 * j + 4 * q]), a1 = __uint_as_float(r[8 * j + 4 * q + 1]);
+            const float a2 = __uint_as_float(r[8 * j + 4 * q + 2]), a3 = __uint_as_float(r[8 * j + 4 * q + 3]);
+            adst[2 * j + q] = make_float4(a0, a1, a2, a3);
+            const float u0 = fmaf(kappa, a0, x.x), u1 = fmaf(kappa, a1, x.y), u2 = fmaf(kappa, a2, x.z), u3 = fmaf(kappa, a3, x.w);
+            ss += u0 * u0 + u1 * u1 + u2 * u2 + u3 * u3;
+            w[2 * q] = pack_bf16x2(u0, u1);
+            w[2 * q + 1] = pack_bf16x2(u2, u3);
+          }
+          udst[j] = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+    }
+    if (live) p.ssq_out[((size_t)l * p.Nt + n_tile) * p.M + row] = ss;
+  } else if (EPI == UEPI_QKV) {
+    const int Tn = p.T, b = live ? row / Tn : 0, pos = *p.pos_base + (live ? row % Tn : 0);
+#pragma unroll 1
+    for (int hh = 0; hh < BN / 128; ++hh) {
+      const int n = n_tile * BN + hh * 128, kind = n / p.d, hcol = n % p.d;
+      const uint32_t tcol = tbase + hh * 128;
+      __nv_bfloat16 *dst;
+      if (kind == 0) dst = p.q + (size_t)l * p.q_ls + (size_t)row * p.d + hcol;
+      else dst = (kind == 1 ? p.kc : p.vc) + (size_t)l * p.kv_ls + (size_t)b * p.kv_bs + (size_t)pos * p.d + hcol;
+      if (kind == 2) {
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
+          tmem_ld32(tcol + c * 32, r);
+          if (live) {
+            uint4 *o = reinterpret_cast<uint4 *>(dst + c * 32);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint32_t w[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) w[q] = pack_bf16x2(__uint_as_float(r[8 * j + 2 * q]) * rstd, __uint_as_float(r[8 * j + 2 * q + 1]) * rstd);
+              o[j] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+      } else {
+        float ss = 0.f;  // rotation preserves the norm, so the head's sum of squares can be taken before it
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
+          tmem_ld32(tcol + c * 32, r);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float v = __uint_as_float(r[j]) * rstd;
+            ss = fmaf(v, v, ss);
+          }
+        }
+        const float rn = rsqrtf(ss * (1.f / 128.f) + p.qk_eps) * rstd;
+        const float2 *cs = p.rope + (size_t)pos * 64;
+#pragma unroll 1
+        for (int c = 0; c < 2; ++c) {
+          uint32_t lo[32], hi[32];
+          tmem_ld32(tcol + c * 32, lo);
+          tmem_ld32(tcol + 64 + c * 32, hi);
+          if (live) {
+            uint4 *o1 = reinterpret_cast<uint4 *>(dst + c * 32), *o2 = reinterpret_cast<uint4 *>(dst + 64 + c * 32);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint32_t w1[4], w2[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const int i0 = 8 * j + 2 * q;
+                const float2 ca = cs[c * 32 + i0], cb = cs[c * 32 + i0 + 1];
+                const float xa1 = __uint_as_float(lo[i0]) * rn, xa2 = __uint_as_float(hi[i0]) * rn;
+                const float xb1 = __uint_as_float(lo[i0 + 1]) * rn, xb2 = __uint_as_float(hi[i0 + 1]) * rn;
+                w1[q] = pack_bf16x2(xa1 * ca.x - xa2 * ca.y, xb1 * cb.x - xb2 * cb.y);
+                w2[q] = pack_bf16x2(xa1 * ca.y + xa2 * ca.x, xb1 * cb.y + xb2 * cb.x);
+              }
+              o1[j] = make_uint4(w1[0], w1[1], w1[2], w1[3]);
+              o2[j] = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+            }
+          }
+        }
+      }
+    }
+  }
+}
+
+// ---- epilogue of the decode regime: accumulator rows (tokens) already transposed into outs[16][BN+1] ----
+// ew = epilogue warp 0..3, lane; one warp per token, lanes across the tile's columns.
+template <int BN, int EPI>
+__device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const float *outs, int ew, int lane, int n_tile, int ks, int l) {
+  for (int tok = ew; tok < p.M; tok += 4) {
+    const float *y = outs + tok * (BN + 1);
+    float rstd = 1.f;
+    if ((EPI == UEPI_QKV || EPI == UEPI_RELU2_BF16 || EPI == UEPI_LMHEAD) && p.ssq != nullptr) {
+      float ss = 0.f;
+      for (int i = 0; i < p.nparts; ++i) ss += p.ssq[((size_t)l * p.nparts + i) * p.M + tok];
+      rstd = rsqrtf(ss / (float)p.K + p.eps);
+    }
+    const size_t n0 = (size_t)n_tile * BN;
+    if (EPI == UEPI_F32) {
+      float *dst = p.c + (size_t)ks * p.out_ss + (size_t)l * p.out_ls + (size_t)tok * p.N + n0;
+#pragma unroll
+      for (int j = 0; j < BN / 32; ++j) dst[lane + 32 * j] = y[lane + 32 * j];
+    } else if (EPI == UEPI_RELU2_BF16) {
+      __nv_bfloat16 *dst = p.z + (size_t)l * p.out_ls + (size_t)tok * p.N + n0;
+#pragma unroll
+      for (int j = 0; j < BN / 32; ++j) {
+        const float v = fmaxf(y[lane + 32 * j] * rstd, 0.f);
+        dst[lane + 32 * j] = __float2bfloat16_rn(v * v);
+      }
+    } else if (EPI == UEPI_RESID) {
+      const float kappa = p.coef[l].kappa;
+      const float *xs = p.xm + (size_t)l * p.xm_ls + (size_t)tok * p.N + n0;
+      float *adst = p.c + (size_t)l * p.out_ls + (size_t)tok * p.N + n0;
+      __nv_bfloat16 *udst = p.z + (size_t)l * p.out_ls + (size_t)tok * p.N + n0;
+      float ss = 0.f;
+#pragma unroll
+      for (int j = 0; j < BN / 32; ++j) {
+        const float a = y[lane + 32 * j];
+        const float u = fmaf(kappa, a, xs[lane + 32 * j]);
+        adst[lane + 32 * j] = a;
+        udst[lane + 32 * j] = __float2bfloat16_rn(u);
+        ss = fmaf(u, u, ss);
+      }
+      ss = warp_sum(ss);
+      if (lane == 0) p.ssq_out[((size_t)l * p.Nt + n_tile) * p.M + tok] = ss;
+    } else if (EPI == UEPI_QKV) {
+      const int b = tok / p.T, pos = *p.pos_base + (tok % p.T);
+#pragma unroll 1
+      for (int hh = 0; hh < BN / 128; ++hh) {
+        const int n = (int)n0 + hh * 128, kind = n / p.d, hcol = n % p.d;
+        const float *yh = y + hh * 128;
+        __nv_bfloat16 *dst;
+        if (kind == 0) dst = p.q + (size_t)l * p.q_ls + (size_t)tok * p.d + hcol;
+        else dst = (kind == 1 ? p.kc : p.vc) + (size_t)l * p.kv_ls + (size_t)b * p.kv_bs + (size_t)pos * p.d + hcol;
+        if (kind == 2) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) dst[lane + 32 * j] = __float2bfloat16_rn(yh[lane + 32 * j] * rstd);
+        } else {
+          const float2 c0 = p.rope[(size_t)pos * 64 + lane], c1 = p.rope[(size_t)pos * 64 + lane + 32];
+          const float a1 = yh[lane] * rstd, a2 = yh[lane + 64] * rstd, b1 = yh[lane + 32] * rstd, b2 = yh[lane + 96] * rstd;
+          const float ya1 = a1 * c0.x - a2 * c0.y, ya2 = a1 * c0.y + a2 * c0.x;
+          const float yb1 = b1 * c1.x - b2 * c1.y, yb2 = b1 * c1.y + b2 * c1.x;
+          const float ss = warp_sum(ya1 * ya1 + ya2 * ya2 + yb1 * yb1 + yb2 * yb2);
+          const float rn = rsqrtf(ss * (1.f / 128.f) + p.qk_eps);
+          dst[lane] = __float2bfloat16_rn(ya1 * rn);
+          dst[lane + 64] = __float2bfloat16_rn(ya2 * rn);
+          dst[lane + 32] = __float2bfloat16_rn(yb1 * rn);
+          dst[lane + 96] = __float2bfloat16_rn(yb2 * rn);
+        }
+      }
+    } else {  // UEPI_LMHEAD
+      float bv = -INFINITY;
+      int bi = 0x7fffffff;
+#pragma unroll
+      for (int j = 0; j < BN / 32; ++j) {
+        const int cidx = lane + 32 * j;
+        const float v = y[cidx] * rstd;
+        if (p.logits) p.logits[(size_t)tok * p.N + n0 + cidx] = v;
+        if (v > bv) { bv = v; bi = (int)n0 + cidx; }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+      }
+      if (lane == 0) { p.pm_val[(size_t)tok * p.Nt + n_tile] = bv; p.pm_idx[(size_t)tok * p.Nt + n_tile] = bi; }
+    }
+  }
+}
+
+// grid = min(items, #SMs), 192 threads, dynamic shared memory UmmaCfg<BN, AM>::kSmem.
+// tmA: 3-D map over A {K, M, nl}, box {64, AM, 1}; tmB: 3-D map over the stacked weights {K, N, L}, box {64, BN, 1};
+// both bf16, 128-byte swizzle, rows outside the tensor read as zero.
+template <int BN, int AM, int EPI>
+__global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                                                              UmmaParams p) {
+  using Cfg = UmmaCfg<BN, AM>;
   extern __shared__ unsigned char umma_smem_raw[];
   unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)umma_smem_raw + 1023) & ~(uintptr_t)1023);
-  unsigned char *sA = smem;
-  unsigned char *sB = smem + Cfg::kStages * Cfg::kABytes;
-  uint64_t *full = reinterpret_cast<uint64_t *>(sB + Cfg::kStages * Cfg::kBBytes);
-  uint64_t *empty = full + Cfg::kStages;
-  uint64_t *accbar = empty + Cfg::kStages;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(accbar + 1);
+  const int S = p.nstages;
+  unsigned char *sA = smem;                                   // [S][AM x 128 B]; the A descriptor reads 128 rows from a slot
+  unsigned char *sB = smem + (size_t)S * Cfg::kABytes;        // [S][BN x 128 B]   (>= 14 KB, so those reads stay in bounds)
+  float *outs = reinterpret_cast<float *>(sB + (size_t)S * Cfg::kBBytes);
+  uint64_t *full = reinterpret_cast<uint64_t *>(reinterpret_cast<unsigned char *>(outs) + Cfg::kOuts);
+  uint64_t *empty = full + S;
+  uint64_t *accfull = empty + S, *accempty = accfull + 2;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(accempty + 2);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_tile = blockIdx.x, m_tile = blockIdx.y, l = blockIdx.z;
-  const int nkb = p.K / kUmmaBK;
+  const int nkb = p.kslice / kUmmaBK;
+  const int n_items = p.Mt * p.Nt * p.ksplit * p.nl;
+  const int my_items = (int)blockIdx.x < n_items ? (n_items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+  constexpr uint32_t kTmemCols = 2 * BN;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < Cfg::kStages; ++s) {
+    for (int s = 0; s < S; ++s) {
       mbar_init(&full[s], 1);
       mbar_init(&empty[s], 1);
     }
-    mbar_init(accbar, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&accfull[i], 1);
+      mbar_init(&accempty[i], 1);
+    }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, BN);
+    tmem_alloc(tmem_slot, kTmemCols);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -194,199 +460,104 @@ __global__ void __launch_bounds__(kUmmaThreads) k_umma_gemm(const __grid_constan
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // item -> (row tile, column tile, K split, layer); row tiles fastest so that concurrent CTAs share a weight tile
+#define SNLP_DECODE_ITEM(i)                                       \
+  const int it_ = (int)blockIdx.x + (i) * (int)gridDim.x;         \
+  const int m_tile = it_ % p.Mt;                                  \
+  const int n_tile = (it_ / p.Mt) % p.Nt;                         \
+  const int ks = (it_ / (p.Mt * p.Nt)) % p.ksplit;                \
+  const int l = it_ / (p.Mt * p.Nt * p.ksplit);
+
   if (warp == 0) {
     if (lane == 0) {
-      int issued = 0;
-      for (int kb = 0; kb < nkb; ++kb) {
-        const int s = kb % Cfg::kStages;
-        const uint32_t ph = (kb / Cfg::kStages) & 1;
-        if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag, p.err)) break;
-        mbar_expect_tx(&full[s], Cfg::kABytes + Cfg::kBBytes);
-        tma_load_3d(sA + s * Cfg::kABytes, &tmA, &full[s], kb * kUmmaBK, m_tile * kUmmaBM, l);
-        tma_load_3d(sB + s * Cfg::kBBytes, &tmB, &full[s], kb * kUmmaBK, n_tile * BN, l);
-        issued = kb + 1;
+      int g = 0, issued = 0;
+      bool ok = true;
+      for (int i = 0; i < my_items && ok; ++i) {
+        SNLP_DECODE_ITEM(i)
+        for (int kb = 0; kb < nkb; ++kb, ++g) {
+          const int s = g % S;
+          ok = mbar_wait(&empty[s], ((g / S) & 1) ^ 1u, abort_flag, p.err);
+          if (!ok) break;
+          mbar_expect_tx(&full[s], Cfg::kABytes + Cfg::kBBytes);
+          const int k0 = ks * p.kslice + kb * kUmmaBK;
+          tma_load_3d(sA + (size_t)s * Cfg::kABytes, &tmA, &full[s], k0, m_tile * kUmmaBM, l);
+          tma_load_3d(sB + (size_t)s * Cfg::kBBytes, &tmB, &full[s], k0, n_tile * BN, p.l0 + l);
+          issued = g + 1;
+        }
       }
       if (*abort_flag) {
         // let the copies still in flight land before the CTA's shared memory is handed on
-        const int first = issued > Cfg::kStages ? issued - Cfg::kStages : 0;
-        for (int kb = first; kb < issued; ++kb) {
+        const int first = issued > S ? issued - S : 0;
+        for (int q = first; q < issued; ++q) {
           const unsigned long long t0 = global_ns();
-          while (!mbar_try_wait(&full[kb % Cfg::kStages], (kb / Cfg::kStages) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+          while (!mbar_try_wait(&full[q % S], (q / S) & 1) && global_ns() - t0 < kWaitLimitNs) {}
         }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16(kUmmaBM, BN);
+      int g = 0;
       bool ok = true;
-      for (int kb = 0; kb < nkb && ok; ++kb) {
-        const int s = kb % Cfg::kStages;
-        const uint32_t ph = (kb / Cfg::kStages) & 1;
-        ok = mbar_wait(&full[s], ph, abort_flag, p.err);
+      for (int i = 0; i < my_items && ok; ++i) {
+        const int b = i & 1;
+        ok = mbar_wait(&accempty[b], ((i >> 1) & 1) ^ 1u, abort_flag, p.err);
         if (!ok) break;
         tc_fence_after();
-        const uint64_t da = umma_desc_sw128(smem_u32(sA + s * Cfg::kABytes));
-        const uint64_t db = umma_desc_sw128(smem_u32(sB + s * Cfg::kBBytes));
+        const uint32_t dcol = tmem_base + b * BN;
+        for (int kb = 0; kb < nkb; ++kb, ++g) {
+          const int s = g % S;
+          ok = mbar_wait(&full[s], (g / S) & 1, abort_flag, p.err);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t da = umma_desc_sw128(smem_u32(sA + (size_t)s * Cfg::kABytes));
+          const uint64_t db = umma_desc_sw128(smem_u32(sB + (size_t)s * Cfg::kBBytes));
 #pragma unroll
-        for (int k = 0; k < kUmmaBK / 16; ++k)  // 16 bf16 = 32 bytes = 2 descriptor address units per step
-          umma_bf16(tmem_base, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
-        umma_commit(&empty[s]);
+          for (int k = 0; k < kUmmaBK / 16; ++k)  // 16 bf16 = 32 bytes = 2 descriptor address units per step
+            umma_bf16(dcol, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+          umma_commit(&empty[s]);
+        }
+        if (ok) umma_commit(&accfull[b]);
       }
-      if (ok) umma_commit(accbar);
     }
   } else {
-    const bool ok = mbar_wait(accbar, 0, abort_flag, p.err);
-    tc_fence_after();
-    if (ok) {
-      const int quarter = warp & 3;  // tensor-memory lanes this warp may read: 32*quarter .. +31
-      const int row = m_tile * kUmmaBM + quarter * 32 + lane;
-      const bool live = row < p.M;
-      const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16);
-      float rstd = 1.f;
-      if ((EPI == UEPI_QKV || EPI == UEPI_RELU2_BF16) && p.ssq != nullptr && live) {
-        float ss = 0.f;
-        for (int i = 0; i < p.nparts; ++i) ss += p.ssq[((size_t)l * p.nparts + i) * p.M + row];
-        rstd = rsqrtf(ss / (float)p.K + p.eps);
-      }
-      if (EPI == UEPI_F32 || EPI == UEPI_RELU2_BF16) {
+    const int et = threadIdx.x - 64, ew = et >> 5;
+    const int quarter = warp & 3;  // tensor-memory lanes this warp may read: 32*quarter .. +31
+    for (int i = 0; i < my_items; ++i) {
+      SNLP_DECODE_ITEM(i)
+      const int b = i & 1;
+      if (!epi_all(mbar_wait(&accfull[b], (i >> 1) & 1, abort_flag, p.err))) break;
+      tc_fence_after();
+      const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * BN;
+      if (AM == kUmmaBM) {
+        umma_epilogue_rows<BN, EPI>(p, tbase, m_tile * kUmmaBM + quarter * 32 + lane, n_tile, ks, l);
+        tc_fence_before();
+        epi_bar_sync();
+        if (et == 0) mbar_arrive(&accempty[b]);
+      } else {
+        if (quarter == 0) {  // the token rows live in lanes 0..15
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(tbase + c * 32, r);
-          if (live) {
-            const size_t off = (size_t)l * p.out_ls + (size_t)row * p.N + (size_t)n_tile * BN + c * 32;
-            if (EPI == UEPI_F32) {
-              float4 *dst = reinterpret_cast<float4 *>(p.c + off);
+          for (int c = 0; c < BN / 32; ++c) {
+            uint32_t r[32];
+            tmem_ld32(tbase + c * 32, r);
+            if (lane < 16) {
 #pragma unroll
-              for (int j = 0; j < 8; ++j)
-                dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
-                                     __uint_as_float(r[4 * j + 3]));
-            } else {
-              uint4 *dst = reinterpret_cast<uint4 *>(p.z + off);
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                uint32_t w[4];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                  const float a = fmaxf(__uint_as_float(r[8 * j + 2 * q]) * rstd, 0.f);
-                  const float b = fmaxf(__uint_as_float(r[8 * j + 2 * q + 1]) * rstd, 0.f);
-                  __nv_bfloat162 v = __floats2bfloat162_rn(a * a, b * b);
-                  w[q] = *reinterpret_cast<uint32_t *>(&v);
-                }
-                dst[j] = make_uint4(w[0], w[1], w[2], w[3]);
-              }
+              for (int j = 0; j < 32; ++j) outs[lane * (BN + 1) + c * 32 + j] = __uint_as_float(r[j]);
             }
           }
         }
-      } else if (EPI == UEPI_RESID) {
-        const float kappa = p.coef[l].kappa;
-        float ss = 0.f;
-#pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(tbase + c * 32, r);
-          if (live) {
-            const size_t col = (size_t)n_tile * BN + c * 32;
-            const size_t off = (size_t)l * p.out_ls + (size_t)row * p.N + col;
-            const float4 *xs = reinterpret_cast<const float4 *>(p.xm + (size_t)l * p.xm_ls + (size_t)row * p.N + col);
-            float4 *adst = reinterpret_cast<float4 *>(p.c + off);
-            uint4 *udst = reinterpret_cast<uint4 *>(p.z + off);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              uint32_t w[4];
-#pragma unroll
-              for (int q = 0; q < 2; ++q) {
-                const float4 x = xs[2 * j + q];
-                const float a0 = __uint_as_float(r[8 * j + 4 * q]), a1 = __uint_as_float(r[8 * j + 4 * q + 1]);
-                const float a2 = __uint_as_float(r[8 * j + 4 * q + 2]), a3 = __uint_as_float(r[8 * j + 4 * q + 3]);
-                adst[2 * j + q] = make_float4(a0, a1, a2, a3);
-                const float u0 = fmaf(kappa, a0, x.x), u1 = fmaf(kappa, a1, x.y), u2 = fmaf(kappa, a2, x.z), u3 = fmaf(kappa, a3, x.w);
-                ss += u0 * u0 + u1 * u1 + u2 * u2 + u3 * u3;
-                __nv_bfloat162 v0 = __floats2bfloat162_rn(u0, u1), v1 = __floats2bfloat162_rn(u2, u3);
-                w[2 * q] = *reinterpret_cast<uint32_t *>(&v0);
-                w[2 * q + 1] = *reinterpret_cast<uint32_t *>(&v1);
-              }
-              udst[j] = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-          }
-        }
-        if (live) p.ssq_out[((size_t)l * gridDim.x + n_tile) * p.M + row] = ss;
-      } else {  // UEPI_QKV
-        const int Tn = p.T, b = live ? row / Tn : 0, pos = *p.pos_base + (live ? row % Tn : 0);
-#pragma unroll 1
-        for (int hh = 0; hh < BN / 128; ++hh) {
-          const int n = n_tile * BN + hh * 128, kind = n / p.d, hcol = n % p.d;
-          const uint32_t tcol = tbase + hh * 128;
-          __nv_bfloat16 *dst;
-          if (kind == 0) dst = p.q + (size_t)l * p.q_ls + (size_t)row * p.d + hcol;
-          else dst = (kind == 1 ? p.kc : p.vc) + (size_t)l * p.kv_ls + (size_t)b * p.kv_bs + (size_t)pos * p.d + hcol;
-          if (kind == 2) {
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-              uint32_t r[32];
-              tmem_ld32(tcol + c * 32, r);
-              if (live) {
-                uint4 *o = reinterpret_cast<uint4 *>(dst + c * 32);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  uint32_t w[4];
-#pragma unroll
-                  for (int q = 0; q < 4; ++q) {
-                    __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[8 * j + 2 * q]) * rstd, __uint_as_float(r[8 * j + 2 * q + 1]) * rstd);
-                    w[q] = *reinterpret_cast<uint32_t *>(&v);
-                  }
-                  o[j] = make_uint4(w[0], w[1], w[2], w[3]);
-                }
-              }
-            }
-          } else {
-            float ss = 0.f;  // rotation preserves the norm, so the head's sum of squares can be taken before it
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-              uint32_t r[32];
-              tmem_ld32(tcol + c * 32, r);
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const float v = __uint_as_float(r[j]) * rstd;
-                ss = fmaf(v, v, ss);
-              }
-            }
-            const float rn = rsqrtf(ss * (1.f / 128.f) + p.qk_eps) * rstd;
-            const float2 *cs = p.rope + (size_t)pos * 64;
-#pragma unroll 1
-            for (int c = 0; c < 2; ++c) {
-              uint32_t lo[32], hi[32];
-              tmem_ld32(tcol + c * 32, lo);
-              tmem_ld32(tcol + 64 + c * 32, hi);
-              if (live) {
-                uint4 *o1 = reinterpret_cast<uint4 *>(dst + c * 32), *o2 = reinterpret_cast<uint4 *>(dst + 64 + c * 32);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  uint32_t w1[4], w2[4];
-#pragma unroll
-                  for (int q = 0; q < 4; ++q) {
-                    const int i0 = 8 * j + 2 * q;
-                    const float2 ca = cs[c * 32 + i0], cb = cs[c * 32 + i0 + 1];
-                    const float xa1 = __uint_as_float(lo[i0]) * rn, xa2 = __uint_as_float(hi[i0]) * rn;
-                    const float xb1 = __uint_as_float(lo[i0 + 1]) * rn, xb2 = __uint_as_float(hi[i0 + 1]) * rn;
-                    __nv_bfloat162 y1 = __floats2bfloat162_rn(xa1 * ca.x - xa2 * ca.y, xb1 * cb.x - xb2 * cb.y);
-                    __nv_bfloat162 y2 = __floats2bfloat162_rn(xa1 * ca.y + xa2 * ca.x, xb1 * cb.y + xb2 * cb.x);
-                    w1[q] = *reinterpret_cast<uint32_t *>(&y1);
-                    w2[q] = *reinterpret_cast<uint32_t *>(&y2);
-                  }
-                  o1[j] = make_uint4(w1[0], w1[1], w1[2], w1[3]);
-                  o2[j] = make_uint4(w2[0], w2[1], w2[2], w2[3]);
-                }
-              }
-            }
-          }
-        }
+        tc_fence_before();
+        epi_bar_sync();
+        if (et == 0) mbar_arrive(&accempty[b]);
+        umma_epilogue_small<BN, EPI>(p, outs, ew, lane, n_tile, ks, l);
+        epi_bar_sync();  // outs is reused by the next item
       }
     }
   }
+#undef SNLP_DECODE_ITEM
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_base, BN);
+  if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
 }
 
 // ---- host side: tensor maps -----------------------------------------------------------------------
