@@ -286,10 +286,12 @@ def run_ours(args):
         "e2e": {"value": world * 1e3 / ms_e2e, "unit": "tokens/s", "h2d_bytes_per_step": 4, "d2h_bytes_per_step": 4,
                 "steps": e2e_steps, "note": "host token in pinned memory -> H2D, snlp_decode_step, D2H, stream sync, every step"},
         "gpu_launches": launches_timed,
-        "roofline": {"bound": "hbm", "kernel": f"k_gemv_mma ({dom}, all 20 layers in one launch)", "achieved": achieved,
+        "roofline": {"bound": "hbm", "kernel": f"k_umma_gemm<BN=256, AM=16> ({dom} projection, all 20 layers in one launch)", "achieved": achieved,
                      "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak, "peak_source": peak_src,
                      "traffic": NCU_TRAFFIC_BYTES.get(dom), "alg_bytes_per_launch": cls_bytes[dom],
-                     "ms_per_launch": dom_ms},
+                     "ms_per_launch": dom_ms,
+                     "note": "duration = CUDA events recorded by the library around every launch of the class (graphs off), "
+                             "which adds a few microseconds per launch; the whole-step figure under `sweep` has no such overhead"},
         "sweep": {"alg_bytes_per_step": step_bytes, "achieved_GBs": step_gbs, "frac_of_hbm_peak": step_gbs / hbm_peak,
                   "target_frac": 0.70, "note": "whole decode step (K sweeps + lm head) under CUDA-graph replay"},
         "kernels": per_class,

@@ -194,15 +194,12 @@ static bool fused_prefill_ok(const snlp_model *m, int M);
 static bool fast_decode_ok(const snlp_model *m, int M);
 static bool umma_path_ok(const snlp_model *m);
 
-// 64-key sub-blocks per split-KV chunk.  It depends only on how many (layer, sequence, head) triples one
-// launch covers (not on the context length or the number of query rows), so that calls of the same
-// geometry -- a decode step and the verifier block of self-speculative decoding -- merge their keys in the
-// same order.  Few triples (sequential execution, batch 1) get short chunks so the launch still fills the GPU.
-static int attn_csub(int triples) {
-  int c = 1;
-  while (c < 8 && triples >= 16 * c) c *= 2;
-  return c;
-}
+// 64-key sub-blocks per split-KV chunk of the decode-regime attention.  It depends only on the number of
+// (sequence, head) pairs -- not on the context length, the number of query rows or how many layers one
+// launch covers -- so a decode step, the verifier block of self-speculative decoding, a sequential pass and
+// a layer-parallel sweep all merge their keys in the same order (K = L sweeps then reproduce the
+// sequential result bit for bit).
+static int attn_csub(int pairs) { return pairs < 32 ? 4 : 8; }
 
 extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
   if (!cfg || !out) return fail(SNLP_ERR_ARG, "snlp_create: NULL argument");
@@ -600,8 +597,9 @@ static int run_umma(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float
   float *a = m->a + l0 * Md, *mb = m->mb + l0 * Md;
   T *kc = (T *)f.kc + (size_t)l0 * f.kv_ls, *vc = (T *)f.vc + (size_t)l0 * f.kv_ls;
   const int Pu = d / m->w_o.BN;  // column tiles of the out-projection = partials of sum u^2
-  // K split of the down-projection: only worth it when a launch has too few items to occupy the GPU
-  const int sd = (small && nl * (d / m->w_dn.BN) < m->n_sm / 2) ? pick_ksplit(ff, kMaxSplits) : 1;
+  // K split of the decode-regime down-projection (its reduction is the longest); it does not depend on nl, so
+  // sequential execution and layer-parallel sweeps add the partial sums in the same order
+  const int sd = small ? pick_ksplit(ff, kMaxSplits) : 1;
   {
     UmmaParams p{};
     p.ssq = m->ssq_x + (size_t)l0 * P * M; p.nparts = P; p.eps = c.rms_eps;
@@ -610,7 +608,7 @@ static int run_umma(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float
     TRY(umma_gemm<UEPI_QKV>(m, st, KC_QKV, xb, Md, m->w_qkv, l0, p, M, 3 * d, d, 1, nl));
   }
   if (small) {
-    const int csub = attn_csub(nl * f.B * H);
+    const int csub = attn_csub(f.B * H);
     const int nchunk = (f.pos_hi + f.T - 1) / (csub * kAttnSub) + 1;
     KLAUNCH(m, st, KC_ATTN, k_attn_decode<<<dim3(nchunk, f.B * H, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, m->attn_part, m->attn_counters, att, Md,
                                                                             f.T, H, f.pos, csub));
@@ -956,7 +954,7 @@ static int decode_step_impl(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, i
     return SNLP_OK;
   }
   const bool fast = fast_decode_ok(m, kv->B);
-  const int chunk_len = attn_csub((K == 0 ? 1 : m->cfg.n_layer) * kv->B * m->cfg.n_head) * kAttnSub;
+  const int chunk_len = attn_csub(kv->B * m->cfg.n_head) * kAttnSub;
   GraphKey key{kv->B, K, mode, fast ? kv->len / chunk_len + 1 : 0, tok_in, tok_out, resnorm_out, kv};
   auto it = m->graphs.find(key);
   if (it == m->graphs.end()) {
