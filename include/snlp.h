@@ -110,6 +110,9 @@ int snlp_forward_sequential(snlp_model *m, const float *h0, int B, int T, float 
  *               (sum |F_l(h_l) - h_{l+1}|^2, sum |h_{l+1}|^2) over all rows, streams and features,
  *               i.e. the squared residual of Eq. (2) and the normaliser for a relative residual.
  * K > L is allowed (the trace no longer changes after L sweeps).
+ * Sweep k evaluates only blocks k .. L-1: by finite-step exactness the states 0..k already equal the sequential
+ * trace, so blocks 0..k-1 would reproduce the branch outputs of the previous sweep bit for bit; the correction
+ * and the residual norms still cover every layer.  The result is identical to evaluating all L blocks.
  * Errors: ARG (K < 1, unknown mode, NULL h0, B,T < 1), SHAPE, STATE. */
 int snlp_forward_parallel(snlp_model *m, const float *h0, int B, int T, int K, int mode,
                           float *trace_out, float *resnorm_out, void *stream);

@@ -491,9 +491,9 @@ static int correct(snlp_model *m, const Fwd &f, int l0, int nl, int mode, int a_
   return SNLP_OK;
 }
 
-// Blocks l0 .. l0+nl-1, each on its own current input state, then the correction over that range.
+// Blocks l0 .. l0+nl-1, each on its own current input state (branch outputs a, m; the correction is separate).
 template <typename T>
-static int run_generic(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float *resnorm) {
+static int blocks_generic(snlp_model *m, const Fwd &f, int l0, int nl) {
   const snlp_config &c = m->cfg;
   const int M = f.M, d = c.d_model, ff = c.d_ff, H = c.n_head, hd = c.head_dim, n = c.n_streams;
   const size_t Md = (size_t)M * d;
@@ -517,8 +517,7 @@ static int run_generic(snlp_model *m, const Fwd &f, int l0, int nl, int mode, fl
     const size_t tot = (size_t)nl * M * ff;
     KLAUNCH(m, st, KC_OTHER, k_relu2_cast<T><<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(y, z, tot));
   }
-  TRY(gemm<T>(m, st, KC_DOWN, z, (size_t)M * ff, (const T *)m->wdn + (size_t)l0 * d * ff, (size_t)d * ff, mb, Md, M, d, ff, nl));
-  return correct(m, f, l0, nl, mode, 1, 1, resnorm);
+  return gemm<T>(m, st, KC_DOWN, z, (size_t)M * ff, (const T *)m->wdn + (size_t)l0 * d * ff, (size_t)d * ff, mb, Md, M, d, ff, nl);
 }
 
 // Tensor-core GEMM of the prefill regime: C[l] = A[l] (M x K, bf16) * W[l]^T (N x K, bf16), nl layers per launch.
@@ -580,11 +579,13 @@ static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat1
   return SNLP_OK;
 }
 
-// One sweep over layers l0 .. l0+nl-1 on the tensor-core path: six launches whatever nl.
+// The blocks of layers l0 .. l0+nl-1 on the tensor-core path: five launches whatever nl (the correction is the sixth).
 // The four projections run on k_umma_gemm with the rest of the block fused into their epilogues (row RMSNorm
 // as a scale, rotary + QK-norm + KV store, residual add + sum of squares, ReLU^2); the bf16 branch inputs
 // xb/ssq_x of the range must be current (prep_rows, or the previous correction).
-static int run_umma(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float *resnorm) {
+static int down_splits(const snlp_model *m, int M);
+
+static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl) {
   typedef __nv_bfloat16 T;
   const snlp_config &c = m->cfg;
   const int M = f.M, d = c.d_model, ff = c.d_ff, H = c.n_head, n = c.n_streams, P = d / 128, L = c.n_layer;
@@ -597,9 +598,7 @@ static int run_umma(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float
   float *a = m->a + l0 * Md, *mb = m->mb + l0 * Md;
   T *kc = (T *)f.kc + (size_t)l0 * f.kv_ls, *vc = (T *)f.vc + (size_t)l0 * f.kv_ls;
   const int Pu = d / m->w_o.BN;  // column tiles of the out-projection = partials of sum u^2
-  // K split of the decode-regime down-projection (its reduction is the longest); it does not depend on nl, so
-  // sequential execution and layer-parallel sweeps add the partial sums in the same order
-  const int sd = small ? pick_ksplit(ff, kMaxSplits) : 1;
+  const int sd = down_splits(m, M);
   {
     UmmaParams p{};
     p.ssq = m->ssq_x + (size_t)l0 * P * M; p.nparts = P; p.eps = c.rms_eps;
@@ -633,10 +632,16 @@ static int run_umma(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float
     p.c = mb; p.out_ls = Md; p.out_ss = (size_t)L * Md;
     TRY(umma_gemm<UEPI_F32>(m, st, KC_DOWN, z, (size_t)M * ff, m->w_dn, l0, p, M, d, ff, sd, nl));
   }
-  return correct(m, f, l0, nl, mode, 1, sd, resnorm);
+  return SNLP_OK;
 }
 
-// bf16 branch inputs of layers l0 .. l0+nl-1 for run_umma (and the fp32 MLP pre-map of mHC models)
+// K split of the decode-regime down-projection (its reduction is the longest); it does not depend on how many
+// layers a launch covers, so sequential execution and layer-parallel sweeps add the partial sums in the same order.
+static int down_splits(const snlp_model *m, int M) {
+  return (umma_path_ok(m) && M <= kDecodeRows) ? pick_ksplit(m->cfg.d_ff, kMaxSplits) : 1;
+}
+
+// bf16 branch inputs of layers l0 .. l0+nl-1 for blocks_umma (and the fp32 MLP pre-map of mHC models)
 static int prep_rows(snlp_model *m, const Fwd &f, int l0, int nl) {
   const snlp_config &c = m->cfg;
   dim3 grid(f.M, nl);
@@ -664,10 +669,10 @@ static int init_kernel_attributes() {
   return SNLP_OK;
 }
 
-static int run_layers(snlp_model *m, const Fwd &f, int l0, int nl, int mode, float *resnorm) {
-  if (umma_path_ok(m)) return run_umma(m, f, l0, nl, mode, resnorm);
-  if (m->cfg.dtype == SNLP_DTYPE_BF16) return run_generic<__nv_bfloat16>(m, f, l0, nl, mode, resnorm);
-  return run_generic<float>(m, f, l0, nl, mode, resnorm);
+static int run_blocks(snlp_model *m, const Fwd &f, int l0, int nl) {
+  if (umma_path_ok(m)) return blocks_umma(m, f, l0, nl);
+  if (m->cfg.dtype == SNLP_DTYPE_BF16) return blocks_generic<__nv_bfloat16>(m, f, l0, nl);
+  return blocks_generic<float>(m, f, l0, nl);
 }
 
 static int native_mode(const snlp_model *m) { return m->cfg.n_streams > 1 ? SNLP_MODE_HCN : SNLP_MODE_IDN; }
@@ -685,7 +690,10 @@ static int premix(snlp_model *m, const Fwd &f, int l0, int nl) {
 static int sequential(snlp_model *m, const Fwd &f) {
   if (umma_path_ok(m)) TRY(prep_rows(m, f, 0, 1));
   else TRY(premix(m, f, 0, 1));
-  for (int l = 0; l < m->cfg.n_layer; ++l) TRY(run_layers(m, f, l, 1, native_mode(m), nullptr));
+  for (int l = 0; l < m->cfg.n_layer; ++l) {
+    TRY(run_blocks(m, f, l, 1));
+    TRY(correct(m, f, l, 1, native_mode(m), 1, down_splits(m, f.M), nullptr));
+  }
   return SNLP_OK;
 }
 
@@ -697,8 +705,15 @@ static int parallel(snlp_model *m, const Fwd &f, int K, int mode, float *resnorm
                                                                reinterpret_cast<float4 *>(m->trace) + n4, n4, c.n_layer));
   if (umma_path_ok(m)) TRY(prep_rows(m, f, 0, c.n_layer));
   else TRY(premix(m, f, 0, c.n_layer));
-  for (int k = 0; k < K; ++k)
-    TRY(run_layers(m, f, 0, c.n_layer, mode, resnorm_out ? resnorm_out + (size_t)k * c.n_layer * 2 : nullptr));
+  for (int k = 0; k < K; ++k) {
+    // Exactness-aware trimming: entering sweep k the states 0..k already equal the sequential trace (Newton on a
+    // block lower-bidiagonal system), so blocks 0..k-1 would reproduce, bit for bit, the branch outputs they
+    // wrote in sweep k-1.  Only blocks k..L-1 are evaluated; the correction still runs over every layer on the
+    // stored branch outputs, so the trace, the residual norms and the next sweep's inputs are unchanged.
+    const int b0 = k < c.n_layer ? k : c.n_layer;
+    if (b0 < c.n_layer) TRY(run_blocks(m, f, b0, c.n_layer - b0));
+    TRY(correct(m, f, 0, c.n_layer, mode, 1, down_splits(m, f.M), resnorm_out ? resnorm_out + (size_t)k * c.n_layer * 2 : nullptr));
+  }
   return SNLP_OK;
 }
 
