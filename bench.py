@@ -305,8 +305,9 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under profiles/
-NCU_TRAFFIC_BYTES: dict = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch (all 20 layers) of k_umma_gemm in this workload, from the
+# ncu capture summarised in profiles/k_umma_gemm_d20_decode.md
+NCU_TRAFFIC_BYTES: dict = {"qkv": 201.0e6, "out_proj": 66.1e6, "mlp_up": 268.1e6, "mlp_down": 266.2e6}
 
 
 # ----------------------------------------------------------------------------------------------
