@@ -23,6 +23,9 @@ What follows the paper literally:
   * ``mhc_block``               -- the two mHC sub-layer equations of App. C.2.
   * ``ssd_ideal_speedup``       -- the self-speculative-decoding estimate of Sec. 5.1.
 
+  * ``fused_chunk`` / ``forward_chunked`` -- fused cross-layer chunks of App. C.3 and the chunkwise update,
+                                   Eq. (11) (``snlp-iterative``), with the identity chunk surrogate.
+
 What the paper leaves open and this file fixes by definition (parity unpinned for
 these constants; they are definitions shared with the CUDA library, not checks):
   RMSNorm without weights, eps inside the square root; rotary pairs (i, i+hd/2) with
@@ -246,37 +249,47 @@ def residual_norms(cfg, W, trace, kv=None, pos0=0, dtype=np.float64):
     return out
 
 
-def forward_snlp(cfg, W, h0, K, mode, kv=None, pos0=0, dtype=np.float64, all_sweeps=False):
-    """Algorithm 2 with S = 0 (no sequential prefix) and ``h0`` initialisation.
+INIT_H0 = 0   # suffix states start at the prefix state h_S          (Alg. 2 line 5)
+INIT_FWD = 1  # suffix states start at a one-shot parallel forward f_l(h_S)   (Sec. 3.5, Sec. 5 "fwd")
 
-    Returns (trace after K sweeps [L+1, B, T, n, d], resnorm [K, L, 2]) where
+
+def forward_snlp(cfg, W, h0, K, mode, kv=None, pos0=0, dtype=np.float64, all_sweeps=False, S=0, init=INIT_H0):
+    """Algorithm 2: sequential prefix of S layers, then K sweeps over the suffix S..L-1.
+
+    init = INIT_H0: every suffix state starts at h_S (Alg. 2 line 5).  init = INIT_FWD: suffix state l+1
+    starts at F_l(h_S), one batched evaluation of every suffix block on the prefix state (Sec. 3.5).
+    Returns (trace after K sweeps [L+1, B, T, n, d], resnorm [K, L, 2]) where, for suffix layers,
     resnorm[k, l] = (sum |F_l(h_l^k) - h_{l+1}^k|^2, sum |h_{l+1}^k|^2): the residual of Eq. (2)
-    at the trace that ENTERS sweep k.  With all_sweeps=True also returns the list of traces
-    h^0 .. h^K.
+    at the trace that ENTERS sweep k (prefix layers: zeros).  With all_sweeps=True also returns the list of
+    traces h^0 .. h^K.  K = 0 is allowed when S > 0 or init = INIT_FWD (prefix / one-shot forward only).
     """
-    if K < 1:
-        raise ValueError("K must be >= 1")
+    L = cfg.n_layer
+    if K < 0 or not (0 <= S <= L):
+        raise ValueError("K must be >= 0 and 0 <= S <= L")
     h0 = np.asarray(h0, dtype=dtype)
     B, T = h0.shape[:2]
     if kv is None:
         kv = _scratch_kv(cfg, B, T, dtype)
-    L = cfg.n_layer
     old = np.empty((L + 1,) + h0.shape, dtype=dtype)
-    old[:] = h0  # h_l^(0) <- h_0 for every l
+    old[0] = h0
+    for l in range(S):  # sequential prefix (Alg. 2 lines 2-4)
+        old[l + 1] = block(cfg, W, l, old[l], kv, pos0, dtype)
+    hS = old[S].copy()
+    for l in range(S, L):
+        old[l + 1] = hS if init == INIT_H0 else block(cfg, W, l, hS, kv, pos0, dtype)
     res = np.zeros((K, L, 2), dtype=np.float64)
     history = [old.copy()]
     for k in range(K):
-        # parallel for: every block on its own current input
+        # parallel for: every suffix block on its own current input
         tilde = np.empty_like(old)
-        for l in range(L):
+        for l in range(S, L):
             tilde[l + 1] = block(cfg, W, l, old[l], kv, pos0, dtype)
             r = (tilde[l + 1] - old[l + 1]).astype(np.float64)
             res[k, l, 0] = np.sum(r * r)
             res[k, l, 1] = np.sum(old[l + 1].astype(np.float64) ** 2)
-        # sequential structured correction, Eq. (5)
-        new = np.empty_like(old)
-        new[0] = h0
-        for l in range(L):
+        # sequential structured correction, Eq. (5); h_S^(k+1) = h_S
+        new = old.copy()
+        for l in range(S, L):
             A = surrogate(cfg, W, l, mode, dtype)
             delta = new[l] - old[l]
             new[l + 1] = tilde[l + 1] + np.einsum("rs,btsd->btrd", A, delta)
@@ -285,6 +298,68 @@ def forward_snlp(cfg, W, h0, K, mode, kv=None, pos0=0, dtype=np.float64, all_swe
     if all_sweeps:
         return old, res, history
     return old, res
+
+
+# --------------------------------------------------------------------------- #
+# fused chunks (App. C.3) and the chunkwise update, Eq. (11)
+# --------------------------------------------------------------------------- #
+def fused_chunk(cfg, W, layers, h, kv, pos0, dtype):
+    """One fused chunk of residual blocks that all read the same input h[B, T, 1, d] (App. C.3):
+
+        a_C = sum_{l in C} O_l Attn_l(Q_l h, K_l h, V_l h)
+        u_C = h + a_C
+        m_C = sum_{l in C} P_l phi(W_l Norm(u_C))
+        F_C = u_C + m_C
+
+    Returns (F_C(h), a_C, m_C).  Every layer of the chunk keeps its own keys/values.
+    """
+    x = h[:, :, 0, :]
+    a = np.zeros_like(x)
+    for l in layers:
+        a = a + attention_branch(cfg, W, l, x, kv, pos0, dtype)
+    u = x + a
+    m = np.zeros_like(x)
+    for l in layers:
+        m = m + mlp_branch(cfg, W, l, u, dtype)
+    return (u + m)[:, :, None, :], a, m
+
+
+def forward_chunked(cfg, W, h0, K, fuse, kv=None, pos0=0, dtype=np.float64, S=0, init=INIT_H0, correct=True):
+    """Chunkwise SNLP with fused layers ("NxFM" configurations, Sec. 3.5): a sequential prefix of S layers, then
+    the suffix split into N = (L - S) / fuse chunks of `fuse` fused layers; K sweeps of Eq. (11) with the identity
+    chunk surrogate.  K = 0 with init = INIT_H0 is not meaningful; K = None runs the fused model sequentially
+    (chunk after chunk), the reference the paper compares fused-weight variants with.
+
+    Returns the list of chunk-boundary states [h_S, h_{S+fuse}, ..., h_L] (each [B, T, 1, d]).
+    """
+    if cfg.n_streams != 1:
+        raise ValueError("fused chunks are defined for residual (single-stream) blocks")
+    L = cfg.n_layer
+    if (L - S) % fuse:
+        raise ValueError("suffix length must be a multiple of the chunk size")
+    h0 = np.asarray(h0, dtype=dtype)
+    B, T = h0.shape[:2]
+    if kv is None:
+        kv = _scratch_kv(cfg, B, T, dtype)
+    h = h0
+    for l in range(S):
+        h = block(cfg, W, l, h, kv, pos0, dtype)
+    chunks = [list(range(S + c * fuse, S + (c + 1) * fuse)) for c in range((L - S) // fuse)]
+    N = len(chunks)
+    if K is None:  # sequential execution of the fused model
+        states = [h]
+        for C in chunks:
+            states.append(fused_chunk(cfg, W, C, states[-1], kv, pos0, dtype)[0])
+        return states
+    old = [h] + [h if init == INIT_H0 else fused_chunk(cfg, W, C, h, kv, pos0, dtype)[0] for C in chunks]
+    for _ in range(K):
+        tilde = [None] + [fused_chunk(cfg, W, chunks[c], old[c], kv, pos0, dtype)[0] for c in range(N)]
+        new = [h]
+        for c in range(N):
+            corr = (new[c] - old[c]) if correct else 0.0
+            new.append(tilde[c + 1] + corr)
+        old = new
+    return old
 
 
 # --------------------------------------------------------------------------- #

@@ -405,3 +405,93 @@ def test_fp32_instantiation_close_to_fp64():
     a = O.forward_snlp(cfg, W, h0, 2, O.MODE_IDN, dtype=np.float32)[0]
     b = O.forward_snlp(cfg, W, h0, 2, O.MODE_IDN)[0]
     assert a.dtype == np.float32 and relerr(a, b) < 1e-4
+
+
+# ------------------------------------------------------------------ prefix S, fwd initialisation, fused chunks
+@pytest.mark.parametrize("n_streams,mode", [(1, O.MODE_IDN), (4, O.MODE_HCN)])
+def test_prefix_and_fwd_init(n_streams, mode):
+    cfg = small_cfg(n_streams, L=5)
+    W = big_weights(cfg)
+    h0 = synth.make_hidden(cfg, 1, 4, seed=30).astype(np.float64)
+    seq = O.forward_sequential(cfg, W, h0)
+    L = cfg.n_layer
+    # S = L is the sequential forward; S = 0 / h0 init is the plain algorithm
+    assert relerr(O.forward_snlp(cfg, W, h0, 0, mode, S=L)[0], seq) < 1e-13
+    for S in (0, 2):
+        for init in (O.INIT_H0, O.INIT_FWD):
+            _, _, hist = O.forward_snlp(cfg, W, h0, 3, mode, S=S, init=init, all_sweeps=True)
+            extra = 1 if init == O.INIT_FWD else 0   # the one-shot forward already makes state S+1 exact
+            for k in range(4):
+                exact_upto = min(L, S + k + extra)
+                for l in range(exact_upto + 1):
+                    assert relerr(hist[k][l], seq[l]) < 1e-12, (S, init, k, l)
+                if exact_upto + 1 <= L:
+                    assert relerr(hist[k][exact_upto + 1], seq[exact_upto + 1]) > 1e-8, (S, init, k)
+    # fwd initialisation is one evaluation of every suffix block on the prefix state
+    tr = O.forward_snlp(cfg, W, h0, 0, mode, S=2, init=O.INIT_FWD)[0]
+    kv = O.LayerKV(L, 1, 4, cfg.n_head, cfg.head_dim)
+    for l in range(2, L):
+        assert relerr(tr[l + 1], O.block(cfg, W, l, seq[2], kv, 0, np.float64)) < 1e-13
+    # with a prefix the h0-initialised K = 1 closed form starts from h_S (App. C.1)
+    if n_streams == 1:
+        tr = O.forward_snlp(cfg, W, h0, 1, O.MODE_IDN, S=2)[0]
+        acc = seq[2].copy()
+        for l in range(2, L):
+            _, a, m = O.residual_block(cfg, W, l, seq[2], kv, 0, np.float64)
+            acc = acc + (a + m)[:, :, None, :]
+        assert relerr(tr[L], acc) < 1e-13
+
+
+def test_fused_chunks():
+    cfg = small_cfg(1, L=4)
+    W = big_weights(cfg)
+    h0 = synth.make_hidden(cfg, 1, 4, seed=31).astype(np.float64)
+    L = cfg.n_layer
+    # fuse = 1 is the unfused algorithm
+    st = O.forward_chunked(cfg, W, h0, 2, 1)
+    ref = O.forward_snlp(cfg, W, h0, 2, O.MODE_IDN)[0]
+    for l in range(L + 1):
+        assert relerr(st[l], ref[l]) < 1e-13
+    # sequential execution of the fuse = 1 model is Algorithm 1
+    seq = O.forward_sequential(cfg, W, h0)
+    st = O.forward_chunked(cfg, W, h0, None, 1)
+    assert relerr(st[-1], seq[-1]) < 1e-13
+    # brute force: one fused chunk of 2 layers against the scalar implementation's branches
+    from tests.naive_ref import NaiveModel
+    nv = NaiveModel(cfg, W)
+    xs = h0[0, :, 0, :].tolist()
+    a_sum = np.zeros((4, cfg.d_model))
+    for l in (1, 2):
+        a_sum += np.array(nv.attn(l, xs))
+    u = np.array(xs) + a_sum
+    m_sum = np.zeros_like(u)
+    for l in (1, 2):
+        m_sum += np.array(nv.mlp(l, u.tolist()))
+    kv = O.LayerKV(L, 1, 4, cfg.n_head, cfg.head_dim)
+    F, a, m = O.fused_chunk(cfg, W, [1, 2], h0, kv, 0, np.float64)
+    assert relerr(a[0], a_sum) < 1e-12 and relerr(m[0], m_sum) < 1e-12 and relerr(F[0, :, 0], u + m_sum) < 1e-12
+    # cross-layer coupling (App. C.3): fused minus "independent branches summed" is exactly the coupling term, and it
+    # vanishes when the attention out-projections are zero (every MLP branch then sees the same input h)
+    def independent(Wx):
+        out = h0.copy()
+        for l in (1, 2):
+            _, a_l, m_l = O.residual_block(cfg, Wx, l, h0, kv, 0, np.float64)
+            out = out + (a_l + m_l)[:, :, None, :]
+        return out
+    assert relerr(F, independent(W)) > 1e-6
+    Wz = big_weights(cfg)
+    Wz.wo = np.zeros_like(Wz.wo)
+    Fz = O.fused_chunk(cfg, Wz, [1, 2], h0, kv, 0, np.float64)[0]
+    assert relerr(Fz, independent(Wz)) < 1e-13
+    # chunkwise finite-step exactness against sequential execution of the SAME fused model
+    fseq = O.forward_chunked(cfg, W, h0, None, 2)
+    for K in (1, 2):
+        st = O.forward_chunked(cfg, W, h0, K, 2)
+        for c in range(K + 1):
+            assert relerr(st[c], fseq[c]) < 1e-12
+    assert relerr(O.forward_chunked(cfg, W, h0, 1, 2)[-1], fseq[-1]) > 1e-8
+    # one chunk holding the whole suffix (the "1xF4" shape): K = 1 from h0 equals its sequential execution
+    assert relerr(O.forward_chunked(cfg, W, h0, 1, 4)[-1], O.forward_chunked(cfg, W, h0, None, 4)[-1]) < 1e-13
+    # without correction information moves one chunk per sweep
+    a = O.forward_chunked(cfg, W, h0, 1, 2, correct=False)
+    assert relerr(a[-1], O.fused_chunk(cfg, W, [2, 3], h0, kv, 0, np.float64)[0]) < 1e-13
