@@ -117,6 +117,35 @@ int snlp_forward_sequential(snlp_model *m, const float *h0, int B, int T, float 
 int snlp_forward_parallel(snlp_model *m, const float *h0, int B, int T, int K, int mode,
                           float *trace_out, float *resnorm_out, void *stream);
 
+/* General form of Algorithm 2 (Sec. 3.2, 3.5).
+ *   prefix  S: the first S blocks run sequentially (Alg. 2 lines 2-4); the K sweeps cover blocks S .. L-1, with
+ *              h_S held fixed.  0 <= S <= L; S = L is Algorithm 1.
+ *   init      : SNLP_INIT_H0  -- every suffix state starts at the prefix state h_S (Alg. 2 line 5);
+ *               SNLP_INIT_FWD -- suffix state l+1 starts at F_l(h_S): one extra batched evaluation of all suffix
+ *               blocks on the prefix state ("fwd" initialisation of Sec. 3.5 / Sec. 5).
+ *   fuse    M: chunkwise execution with M fused layers per chunk ("NxFM", Sec. 3.5, App. C.3): the M layers of a
+ *              chunk read the chunk input; their attention outputs are summed before the MLPs, which all read
+ *              u_C = h + a_C; the correction of Eq. (11) runs between chunk outputs with the identity surrogate.
+ *              Needs n_streams == 1, (L - S) % M == 0 and mode IDN or NOCORR; M = 1 is the unfused algorithm.
+ *              Only the chunk-boundary states S, S+M, .., L of a trace are defined.
+ *   K       : number of sweeps, >= 0 (0 = prefix and initialisation only).
+ *   mode    : SNLP_MODE_IDN / HCN / NOCORR, or SNLP_MODE_SEQUENTIAL: run the (fused) chunks one after the other,
+ *             the exact forward of the fused model (K and init are ignored).
+ * resnorm_out: [K][L][2]; rows of prefix layers and of layers that are not chunk heads are zero. */
+#define SNLP_INIT_H0 0
+#define SNLP_INIT_FWD 1
+#define SNLP_MODE_SEQUENTIAL 3
+typedef struct {
+  int32_t K, mode, prefix, init, fuse;
+} snlp_solver;
+/* snlp_forward_parallel with a solver description.  Errors as snlp_forward_parallel, plus ARG for an invalid solver
+ * and UNSUPPORTED for fuse > 1 on a multi-stream model. */
+int snlp_forward_solver(snlp_model *m, const float *h0, int B, int T, const snlp_solver *solver, float *trace_out,
+                        float *resnorm_out, void *stream);
+/* snlp_decode_step with a solver description (K = 0 with prefix = L is the sequential step). */
+int snlp_decode_step_solver(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, const snlp_solver *solver, int32_t *tok_out,
+                            float *resnorm_out, void *stream);
+
 /* LMHead (Alg. 1 line 5 / Alg. 2 line 14): sum the streams of hL (device fp32 [rows][n][d]), RMSNorm,
  * project with lm_head.  logits (device fp32 [rows][vocab], nullable) and argmax (device int32 [rows],
  * nullable; ties -> lowest index); at least one of them must be given.

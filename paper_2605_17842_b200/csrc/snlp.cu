@@ -60,11 +60,12 @@ constexpr int kDecodeRows = 16;  // largest row count served by the decode-regim
 constexpr size_t kCorrSmallSmem = 160 * 1024;
 
 struct GraphKey {
-  int B, K, mode, nchunk;
+  int B, K, mode, prefix, init, fuse, nchunk;
   const void *tin, *tout, *res;
   const void *kv;
   bool operator<(const GraphKey &o) const {
-    return std::tie(B, K, mode, nchunk, tin, tout, res, kv) < std::tie(o.B, o.K, o.mode, o.nchunk, o.tin, o.tout, o.res, o.kv);
+    return std::tie(B, K, mode, prefix, init, fuse, nchunk, tin, tout, res, kv) <
+           std::tie(o.B, o.K, o.mode, o.prefix, o.init, o.fuse, o.nchunk, o.tin, o.tout, o.res, o.kv);
   }
 };
 struct GraphEntry { cudaGraphExec_t exec; int64_t nodes; };
@@ -686,35 +687,70 @@ static int premix(snlp_model *m, const Fwd &f, int l0, int nl) {
   return SNLP_OK;
 }
 
-// Alg. 1 over the internal trace (trace[0] must hold h_0).
-static int sequential(snlp_model *m, const Fwd &f) {
-  if (umma_path_ok(m)) TRY(prep_rows(m, f, 0, 1));
-  else TRY(premix(m, f, 0, 1));
-  for (int l = 0; l < m->cfg.n_layer; ++l) {
-    TRY(run_blocks(m, f, l, 1));
-    TRY(correct(m, f, l, 1, native_mode(m), 1, down_splits(m, f.M), nullptr));
+static int check_solver(const snlp_model *m, const snlp_solver &sol, const char *who) {
+  const int L = m->cfg.n_layer;
+  if (sol.mode < SNLP_MODE_IDN || sol.mode > SNLP_MODE_SEQUENTIAL) return fail(SNLP_ERR_ARG, "%s: unknown mode %d", who, sol.mode);
+  if (sol.K < 0) return fail(SNLP_ERR_ARG, "%s: K must be >= 0 (got %d)", who, sol.K);
+  if (sol.prefix < 0 || sol.prefix > L) return fail(SNLP_ERR_ARG, "%s: prefix must be in 0..%d (got %d)", who, L, sol.prefix);
+  if (sol.init != SNLP_INIT_H0 && sol.init != SNLP_INIT_FWD) return fail(SNLP_ERR_ARG, "%s: unknown init %d", who, sol.init);
+  if (sol.fuse < 1) return fail(SNLP_ERR_ARG, "%s: fuse must be >= 1 (got %d)", who, sol.fuse);
+  if (sol.fuse > 1) {
+    if (m->cfg.n_streams != 1) return fail(SNLP_ERR_UNSUPPORTED, "%s: fused chunks need a single-stream model", who);
+    if ((L - sol.prefix) % sol.fuse) return fail(SNLP_ERR_ARG, "%s: suffix length %d is not a multiple of fuse = %d", who, L - sol.prefix, sol.fuse);
+    if (sol.mode == SNLP_MODE_HCN) return fail(SNLP_ERR_ARG, "%s: fused chunks use the identity surrogate (mode IDN or NOCORR)", who);
+    return fail(SNLP_ERR_UNSUPPORTED, "%s: fuse > 1 is not built yet", who);
   }
   return SNLP_OK;
 }
 
-// Alg. 2 (S = 0, h0 init) over the internal trace (trace[0] must hold h_0).
-static int parallel(snlp_model *m, const Fwd &f, int K, int mode, float *resnorm_out) {
+// General Alg. 2 over the internal trace (trace[0] must hold h_0): sequential prefix, initialisation, K sweeps.
+static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *resnorm_out) {
   const snlp_config &c = m->cfg;
+  const int L = c.n_layer, S = sol.mode == SNLP_MODE_SEQUENTIAL ? L : sol.prefix;
+  if (resnorm_out && sol.K > 0) CU(cudaMemsetAsync(resnorm_out, 0, (size_t)sol.K * L * 2 * sizeof(float), f.st));
+  if (S > 0) {  // Alg. 2 lines 2-4
+    if (umma_path_ok(m)) TRY(prep_rows(m, f, 0, 1));
+    else TRY(premix(m, f, 0, 1));
+    for (int l = 0; l < S; ++l) {
+      TRY(run_blocks(m, f, l, 1));
+      TRY(correct(m, f, l, 1, native_mode(m), 1, down_splits(m, f.M), nullptr));
+    }
+  }
+  if (S == L) return SNLP_OK;
+  // Alg. 2 line 5: every suffix state starts at h_S
   const size_t n4 = (size_t)f.M * c.n_streams * c.d_model / 4;
-  KLAUNCH(m, f.st, KC_OTHER, k_bcast_trace<<<(unsigned)((n4 + 255) / 256), 256, 0, f.st>>>(reinterpret_cast<const float4 *>(m->trace),
-                                                               reinterpret_cast<float4 *>(m->trace) + n4, n4, c.n_layer));
-  if (umma_path_ok(m)) TRY(prep_rows(m, f, 0, c.n_layer));
-  else TRY(premix(m, f, 0, c.n_layer));
-  for (int k = 0; k < K; ++k) {
-    // Exactness-aware trimming: entering sweep k the states 0..k already equal the sequential trace (Newton on a
-    // block lower-bidiagonal system), so blocks 0..k-1 would reproduce, bit for bit, the branch outputs they
-    // wrote in sweep k-1.  Only blocks k..L-1 are evaluated; the correction still runs over every layer on the
-    // stored branch outputs, so the trace, the residual norms and the next sweep's inputs are unchanged.
-    const int b0 = k < c.n_layer ? k : c.n_layer;
-    if (b0 < c.n_layer) TRY(run_blocks(m, f, b0, c.n_layer - b0));
-    TRY(correct(m, f, 0, c.n_layer, mode, 1, down_splits(m, f.M), resnorm_out ? resnorm_out + (size_t)k * c.n_layer * 2 : nullptr));
+  KLAUNCH(m, f.st, KC_OTHER, k_bcast_trace<<<(unsigned)((n4 + 255) / 256), 256, 0, f.st>>>(reinterpret_cast<const float4 *>(m->trace) + (size_t)S * n4,
+                                                               reinterpret_cast<float4 *>(m->trace) + (size_t)(S + 1) * n4, n4, L - S));
+  if (umma_path_ok(m)) TRY(prep_rows(m, f, S, L - S));
+  else TRY(premix(m, f, S, L - S));
+  int exact = S;  // states 0..exact equal the sequential trace
+  if (sol.init == SNLP_INIT_FWD) {
+    // one batched evaluation of every suffix block on h_S; with A = 0 the correction just stores F_l(h_S)
+    TRY(run_blocks(m, f, S, L - S));
+    TRY(correct(m, f, S, L - S, SNLP_MODE_NOCORR, 1, down_splits(m, f.M), nullptr));
+    exact = S + 1;
+  }
+  for (int k = 0; k < sol.K; ++k) {
+    // Exactness-aware trimming: entering this sweep the states 0..exact already equal the sequential trace (Newton
+    // on a block lower-bidiagonal system), so blocks before `exact` would reproduce, bit for bit, the branch
+    // outputs they wrote in the previous pass.  Only blocks exact..L-1 are evaluated; the correction still runs
+    // over the whole suffix on the stored branch outputs, so trace, residual norms and next inputs are unchanged.
+    const int b0 = exact < L ? exact : L;
+    if (b0 < L) TRY(run_blocks(m, f, b0, L - b0));
+    TRY(correct(m, f, S, L - S, sol.mode, 1, down_splits(m, f.M), resnorm_out ? resnorm_out + (size_t)k * L * 2 : nullptr));
+    ++exact;
   }
   return SNLP_OK;
+}
+
+static int sequential(snlp_model *m, const Fwd &f) {
+  snlp_solver sol{0, SNLP_MODE_SEQUENTIAL, m->cfg.n_layer, SNLP_INIT_H0, 1};
+  return solve(m, f, sol, nullptr);
+}
+
+static int parallel(snlp_model *m, const Fwd &f, int K, int mode, float *resnorm_out) {
+  snlp_solver sol{K, mode, 0, SNLP_INIT_H0, 1};
+  return solve(m, f, sol, resnorm_out);
 }
 
 // LMHead on `rows` hidden states.  pre_xb / pre_ssq: the bf16 stream-summed rows and their sums of squares if the
@@ -834,6 +870,21 @@ extern "C" int snlp_forward_parallel(snlp_model *m, const float *h0, int B, int 
   return SNLP_OK;
 }
 
+extern "C" int snlp_forward_solver(snlp_model *m, const float *h0, int B, int T, const snlp_solver *solver, float *trace_out,
+                                   float *resnorm_out, void *stream) {
+  TRY(check_model(m, "snlp_forward_solver"));
+  if (!h0 || !solver) return fail(SNLP_ERR_ARG, "snlp_forward_solver: NULL pointer");
+  TRY(check_solver(m, *solver, "snlp_forward_solver"));
+  TRY(check_shape(m, B, T, "snlp_forward_solver"));
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t state = (size_t)B * T * m->cfg.n_streams * m->cfg.d_model;
+  CU(cudaMemcpyAsync(m->trace, h0, state * 4, cudaMemcpyDeviceToDevice, st));
+  Fwd f = scratch_fwd(m, B, T, st);
+  TRY(solve(m, f, *solver, resnorm_out));
+  if (trace_out) CU(cudaMemcpyAsync(trace_out, m->trace, (m->cfg.n_layer + 1) * state * 4, cudaMemcpyDeviceToDevice, st));
+  return SNLP_OK;
+}
+
 extern "C" int snlp_lm_head(snlp_model *m, const float *hL, int rows, float *logits, int32_t *argmax, void *stream) {
   TRY(check_model(m, "snlp_lm_head"));
   if (!hL || (!logits && !argmax)) return fail(SNLP_ERR_ARG, "snlp_lm_head: NULL pointer");
@@ -948,29 +999,26 @@ static int lm_head_tail(snlp_model *m, cudaStream_t st, int rows, int32_t *argma
 }
 
 // enqueue one decode step (no graph handling, no host-side length update)
-static int decode_launches(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, int K, int mode, int32_t *tok_out, float *resnorm_out,
+static int decode_launches(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, const snlp_solver &sol, int32_t *tok_out, float *resnorm_out,
                            cudaStream_t st) {
-  const snlp_config &c = m->cfg;
   TRY(embed_impl(m, st, tok_in, kv->B, m->trace));
   Fwd f = kv_fwd(m, kv, 1, st);
-  if (K == 0) TRY(sequential(m, f));
-  else TRY(parallel(m, f, K, mode, resnorm_out));
-  const size_t nd = (size_t)c.n_streams * c.d_model;
+  TRY(solve(m, f, sol, resnorm_out));
   TRY(lm_head_tail(m, st, kv->B, tok_out));
   KLAUNCH(m, st, KC_OTHER, k_add_int<<<1, 1, 0, st>>>(kv->pos, 1));
   return SNLP_OK;
 }
 
-static int decode_step_impl(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, int K, int mode, int32_t *tok_out, float *resnorm_out,
+static int decode_step_impl(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, const snlp_solver &sol, int32_t *tok_out, float *resnorm_out,
                             cudaStream_t st) {
   if (!m->use_graphs || m->timing) {
-    TRY(decode_launches(m, kv, tok_in, K, mode, tok_out, resnorm_out, st));
+    TRY(decode_launches(m, kv, tok_in, sol, tok_out, resnorm_out, st));
     kv->len += 1;
     return SNLP_OK;
   }
   const bool fast = fast_decode_ok(m, kv->B);
   const int chunk_len = attn_csub(kv->B * m->cfg.n_head) * kAttnSub;
-  GraphKey key{kv->B, K, mode, fast ? kv->len / chunk_len + 1 : 0, tok_in, tok_out, resnorm_out, kv};
+  GraphKey key{kv->B, sol.K, sol.mode, sol.prefix, sol.init, sol.fuse, fast ? kv->len / chunk_len + 1 : 0, tok_in, tok_out, resnorm_out, kv};
   auto it = m->graphs.find(key);
   if (it == m->graphs.end()) {
     if (m->graphs.size() >= 256) {
@@ -981,7 +1029,7 @@ static int decode_step_impl(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, i
     CU(cudaStreamBeginCapture(m->cap_stream, cudaStreamCaptureModeThreadLocal));
     m->capturing = true;
     m->cap_nodes = 0;
-    const int rc = decode_launches(m, kv, tok_in, K, mode, tok_out, resnorm_out, m->cap_stream);
+    const int rc = decode_launches(m, kv, tok_in, sol, tok_out, resnorm_out, m->cap_stream);
     m->capturing = false;
     cudaError_t e = cudaStreamEndCapture(m->cap_stream, &graph);
     if (rc != SNLP_OK) {
@@ -1010,7 +1058,18 @@ extern "C" int snlp_decode_step(snlp_model *m, snlp_kv *kv, const int32_t *tok_i
   if (K < 0) return fail(SNLP_ERR_ARG, "snlp_decode_step: K must be >= 0 (got %d)", K);
   TRY(check_mode(mode, "snlp_decode_step"));
   if (kv->len + 1 > kv->max_ctx) return fail(SNLP_ERR_SHAPE, "snlp_decode_step: cache is full (len %d, max_ctx %d)", kv->len, kv->max_ctx);
-  return decode_step_impl(m, kv, tok_in, K, mode, tok_out, K > 0 ? resnorm_out : nullptr, (cudaStream_t)stream);
+  const snlp_solver sol = K == 0 ? snlp_solver{0, SNLP_MODE_SEQUENTIAL, m->cfg.n_layer, SNLP_INIT_H0, 1} : snlp_solver{K, mode, 0, SNLP_INIT_H0, 1};
+  return decode_step_impl(m, kv, tok_in, sol, tok_out, K > 0 ? resnorm_out : nullptr, (cudaStream_t)stream);
+}
+
+extern "C" int snlp_decode_step_solver(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, const snlp_solver *solver, int32_t *tok_out,
+                                       float *resnorm_out, void *stream) {
+  TRY(check_model(m, "snlp_decode_step_solver"));
+  if (!kv || !tok_in || !tok_out || !solver) return fail(SNLP_ERR_ARG, "snlp_decode_step_solver: NULL pointer");
+  if (kv->m != m) return fail(SNLP_ERR_ARG, "snlp_decode_step_solver: cache belongs to another model");
+  TRY(check_solver(m, *solver, "snlp_decode_step_solver"));
+  if (kv->len + 1 > kv->max_ctx) return fail(SNLP_ERR_SHAPE, "snlp_decode_step_solver: cache is full (len %d, max_ctx %d)", kv->len, kv->max_ctx);
+  return decode_step_impl(m, kv, tok_in, *solver, tok_out, solver->K > 0 ? resnorm_out : nullptr, (cudaStream_t)stream);
 }
 
 extern "C" int snlp_draft_and_verify(snlp_model *m, snlp_kv *kv, int32_t *last_tok, int block, int K, int mode, int32_t *emitted,
@@ -1030,7 +1089,8 @@ extern "C" int snlp_draft_and_verify(snlp_model *m, snlp_kv *kv, int32_t *last_t
   int32_t *ids = m->spec;                          // [block+1]: last_tok, x_1..x_block
   int32_t *y = m->spec + (c.max_rows + 1);         // [block+1]: verifier tokens
   CU(cudaMemcpyAsync(ids, last_tok, 4, cudaMemcpyDeviceToDevice, st));
-  for (int i = 0; i < block; ++i) TRY(decode_step_impl(m, kv, ids + i, K, mode, ids + i + 1, nullptr, st));
+  const snlp_solver draft{K, mode, 0, SNLP_INIT_H0, 1};
+  for (int i = 0; i < block; ++i) TRY(decode_step_impl(m, kv, ids + i, draft, ids + i + 1, nullptr, st));
   KLAUNCH(m, st, KC_OTHER, k_set_int<<<1, 1, 0, st>>>(kv->pos, len0));
   kv->len = len0;
   TRY(embed_impl(m, st, ids, block + 1, m->trace));

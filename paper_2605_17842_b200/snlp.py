@@ -17,11 +17,12 @@ LIB_PATH = os.path.join(_HERE, "libsnlp.so")
 OK = 0
 ERR_ARG, ERR_SHAPE, ERR_STATE, ERR_OOM, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = -1, -2, -3, -4, -5, -6, -7
 DTYPE_FP32, DTYPE_BF16 = 0, 1
-MODE_IDN, MODE_HCN, MODE_NOCORR = 0, 1, 2
+MODE_IDN, MODE_HCN, MODE_NOCORR, MODE_SEQUENTIAL = 0, 1, 2, 3
+INIT_H0, INIT_FWD = 0, 1
 
 EXPORTS = [
     "snlp_create", "snlp_destroy", "snlp_load_weights", "snlp_embed", "snlp_forward_sequential",
-    "snlp_forward_parallel", "snlp_lm_head", "snlp_kv_create", "snlp_kv_destroy", "snlp_kv_len",
+    "snlp_forward_parallel", "snlp_forward_solver", "snlp_decode_step_solver", "snlp_lm_head", "snlp_kv_create", "snlp_kv_destroy", "snlp_kv_len",
     "snlp_kv_truncate", "snlp_prefill", "snlp_decode_step", "snlp_draft_and_verify", "snlp_set_flag",
     "snlp_launch_count", "snlp_kernel_times", "snlp_device_status", "snlp_lm_head_greedy_static", "snlp_last_error",
 ]
@@ -31,6 +32,14 @@ class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layer", "d_model", "n_head", "head_dim", "d_ff", "vocab", "n_streams",
                                          "dtype", "max_rows", "max_batch", "max_ctx")] + \
                [("rms_eps", C.c_float), ("rope_base", C.c_float)]
+
+
+class Solver(C.Structure):
+    """snlp_solver: K sweeps, mode, sequential prefix S, initialisation, fused layers per chunk."""
+    _fields_ = [(n, C.c_int32) for n in ("K", "mode", "prefix", "init", "fuse")]
+
+    def __init__(self, K=1, mode=0, prefix=0, init=0, fuse=1):
+        super().__init__(K, mode, prefix, init, fuse)
 
 
 class Weights(C.Structure):
@@ -171,6 +180,19 @@ class Model:
         _check(_lib.snlp_forward_parallel(self._h, _ptr(h0), C.c_int(B), C.c_int(T), C.c_int(K), C.c_int(mode),
                                           _ptr(tr), _ptr(rn), _stream()))
         return tr, rn
+
+    def forward_solver(self, h0: torch.Tensor, solver: "Solver", want_trace: bool = True, want_resnorm: bool = True):
+        B, T = h0.shape[:2]
+        tr = self._trace(h0) if want_trace else None
+        rn = torch.zeros((max(solver.K, 1), self.n_layer, 2), dtype=torch.float32, device=h0.device) if want_resnorm else None
+        _check(_lib.snlp_forward_solver(self._h, _ptr(h0), C.c_int(B), C.c_int(T), C.byref(solver), _ptr(tr), _ptr(rn), _stream()))
+        return tr, rn
+
+    def decode_step_solver(self, kv: "KVCache", tok_in: torch.Tensor, solver: "Solver", tok_out: torch.Tensor | None = None):
+        if tok_out is None:
+            tok_out = torch.empty_like(tok_in)
+        _check(_lib.snlp_decode_step_solver(self._h, kv._h, _ptr(tok_in), C.byref(solver), _ptr(tok_out), C.c_void_p(0), _stream()))
+        return tok_out
 
     def lm_head(self, hL: torch.Tensor, want_logits: bool = True):
         rows = hL.numel() // (self.n_streams * self.d_model)
