@@ -154,6 +154,7 @@ int snlp_lm_head(snlp_model *m, const float *hL, int rows, float *logits, int32_
 
 /* KV cache for B sequences of up to max_ctx positions: per layer K and V [B][max_ctx][d] in the
  * model's dtype; keys are stored after rotary and QK-norm.  All sequences share one length.
+ * A cache may outlive its model (snlp_destroy leaves it valid for snlp_kv_destroy only).
  * Errors: ARG, SHAPE (B > max_batch, max_ctx > config.max_ctx), OOM. */
 int snlp_kv_create(snlp_model *m, int B, int max_ctx, snlp_kv **out);
 int snlp_kv_destroy(snlp_kv *kv);

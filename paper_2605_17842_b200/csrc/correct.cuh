@@ -13,7 +13,8 @@ struct CorrParams {
   const float *m;    // [m_splits][L][M][d] MLP-branch outputs
   size_t a_ss, m_ss; // split strides (elements)
   int a_splits, m_splits;
-  int l0, nl, L;
+  int l0, nl, L;     // nl steps starting at state l0
+  int lstep;         // layers per step: 1, or the number of fused layers of a chunk (states l0, l0+lstep, ...)
   int M, d;
   int mode;          // SNLP_MODE_*
   const HcCoef *coef;
@@ -61,7 +62,7 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
     for (int s = 0; s < NS; ++s) oldp[s] = newp[s] = tr4[(size_t)p.l0 * state4 + st_off + (size_t)s * d4];
   }
   for (int i = 0; i < p.nl; ++i) {
-    const int l = p.l0 + i;
+    const int l = p.l0 + i * p.lstep, ln = l + p.lstep;  // this step maps state l to state ln
     float rs = 0.f, hs = 0.f, xs = 0.f;
     if (active) {
       float4 av = a4[(size_t)l * Md4 + bm_off];
@@ -72,7 +73,7 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
       float4 oldn[NS], newn[NS], tilde[NS];
 #pragma unroll
       for (int r = 0; r < NS; ++r) {
-        oldn[r] = tr4[(size_t)(l + 1) * state4 + st_off + (size_t)r * d4];
+        oldn[r] = tr4[(size_t)ln * state4 + st_off + (size_t)r * d4];
         if (NS == 1) {
           tilde[r] = f4_add(f4_add(oldp[0], av), mv);  // F_l(h_l^k) = (h + a) + m
         } else {
@@ -101,29 +102,29 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
         const float4 rr = f4_sub(tilde[r], oldn[r]);
         rs += f4_sq(rr);
         hs += f4_sq(oldn[r]);
-        tr4[(size_t)(l + 1) * state4 + st_off + (size_t)r * d4] = newn[r];
+        tr4[(size_t)ln * state4 + st_off + (size_t)r * d4] = newn[r];
       }
       float4 nxt = newn[0];  // the next layer's attention-branch input
-      if (NS > 1 && l + 1 < p.L) {
-        const HcCoef &cn = p.coef[l + 1];
+      if (NS > 1 && ln < p.L) {
+        const HcCoef &cn = p.coef[ln];
         float4 sa = f4_scale(cn.pa[0], newn[0]), sm = f4_scale(cn.pmra[0], newn[0]);
 #pragma unroll
         for (int s = 1; s < NS; ++s) {
           sa = f4_fma(cn.pa[s], newn[s], sa);
           sm = f4_fma(cn.pmra[s], newn[s], sm);
         }
-        reinterpret_cast<float4 *>(p.xa)[(size_t)(l + 1) * Md4 + bm_off] = sa;
-        reinterpret_cast<float4 *>(p.xm)[(size_t)(l + 1) * Md4 + bm_off] = sm;
+        reinterpret_cast<float4 *>(p.xa)[(size_t)ln * Md4 + bm_off] = sa;
+        reinterpret_cast<float4 *>(p.xm)[(size_t)ln * Md4 + bm_off] = sm;
         nxt = sa;
       }
-      if (NS > 1 && l + 1 == p.L) {  // after the last block: the LM head reads the sum of the streams
+      if (NS > 1 && ln == p.L) {  // after the last block: the LM head reads the sum of the streams
 #pragma unroll
         for (int s = 1; s < NS; ++s) nxt = f4_add(nxt, newn[s]);
       }
       if (p.xb != nullptr) {
         __nv_bfloat162 lo = __floats2bfloat162_rn(nxt.x, nxt.y), hi = __floats2bfloat162_rn(nxt.z, nxt.w);
         uint2 pk = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
-        reinterpret_cast<uint2 *>(p.xb)[(size_t)(l + 1) * Md4 + bm_off] = pk;
+        reinterpret_cast<uint2 *>(p.xb)[(size_t)ln * Md4 + bm_off] = pk;
         xs = f4_sq(nxt);
       }
 #pragma unroll
@@ -132,7 +133,7 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
     if (p.xb != nullptr) {
       // d is a multiple of 128 here, so the 32 lanes of a warp hold 128 consecutive columns of one row
       xs = warp_sum(xs);
-      if (lane == 0 && active) p.ssq_x[((size_t)(l + 1) * (d4 >> 5) + (c4 >> 5)) * p.M + row] = xs;
+      if (lane == 0 && active) p.ssq_x[((size_t)ln * (d4 >> 5) + (c4 >> 5)) * p.M + row] = xs;
     }
     if (want_norm) {
       rs = warp_sum(rs);
@@ -157,7 +158,7 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
   for (int i = threadIdx.x; i < p.nl * 2; i += blockDim.x) {
     double s = 0.0;
     for (unsigned b = 0; b < gridDim.x; ++b) s += (double)__ldcg(&p.partial[(size_t)b * p.nl * 2 + i]);
-    p.resnorm[(size_t)p.l0 * 2 + i] = (float)s;
+    p.resnorm[(size_t)(p.l0 + (i >> 1) * p.lstep) * 2 + (i & 1)] = (float)s;
   }
   if (threadIdx.x == 0) *p.counter = 0u;
 }
@@ -231,7 +232,7 @@ __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
   const bool want_norm = p.partial != nullptr;
   if (active) {
     for (int i = ll; i < p.nl; i += 8) {
-      const int l = p.l0 + i;
+      const int l = p.l0 + i * p.lstep, ln = l + p.lstep;  // this step maps state l to state ln
       float4 av = a4[(size_t)l * Md4 + bm_off];
       for (int q = 1; q < p.a_splits; ++q) av = f4_add(av, a4[(size_t)q * (p.a_ss >> 2) + (size_t)l * Md4 + bm_off]);
       float4 mv = m4[(size_t)l * Md4 + bm_off];
@@ -239,7 +240,7 @@ __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
       sa[i * 32 + c] = av;
       sm[i * 32 + c] = mv;
 #pragma unroll
-      for (int r = 0; r < NS; ++r) so[(i * NS + r) * 32 + c] = tr4[(size_t)(l + 1) * state4 + st_off + (size_t)r * d4];
+      for (int r = 0; r < NS; ++r) so[(i * NS + r) * 32 + c] = tr4[(size_t)ln * state4 + st_off + (size_t)r * d4];
     }
   }
   __syncthreads();
@@ -251,7 +252,7 @@ __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
     for (int s = 0; s < NS; ++s) oldp[s] = newp[s] = tr4[(size_t)p.l0 * state4 + st_off + (size_t)s * d4];
   }
   for (int i = 0; i < p.nl; ++i) {
-    const int l = p.l0 + i;
+    const int l = p.l0 + i * p.lstep, ln = l + p.lstep;  // this step maps state l to state ln
     float rs = 0.f, hs = 0.f, xs = 0.f;
     if (active) {
       const float4 av = sa[i * 32 + c], mv = sm[i * 32 + c];
@@ -288,28 +289,28 @@ __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
         const float4 rr = f4_sub(tilde[r], oldn[r]);
         rs += f4_sq(rr);
         hs += f4_sq(oldn[r]);
-        tr4[(size_t)(l + 1) * state4 + st_off + (size_t)r * d4] = newn[r];
+        tr4[(size_t)ln * state4 + st_off + (size_t)r * d4] = newn[r];
       }
       float4 nxt = newn[0];
-      if (NS > 1 && l + 1 < p.L) {
-        const HcCoef &cn = p.coef[l + 1];
+      if (NS > 1 && ln < p.L) {
+        const HcCoef &cn = p.coef[ln];
         float4 xa = f4_scale(cn.pa[0], newn[0]), xm = f4_scale(cn.pmra[0], newn[0]);
 #pragma unroll
         for (int s = 1; s < NS; ++s) {
           xa = f4_fma(cn.pa[s], newn[s], xa);
           xm = f4_fma(cn.pmra[s], newn[s], xm);
         }
-        reinterpret_cast<float4 *>(p.xa)[(size_t)(l + 1) * Md4 + bm_off] = xa;
-        reinterpret_cast<float4 *>(p.xm)[(size_t)(l + 1) * Md4 + bm_off] = xm;
+        reinterpret_cast<float4 *>(p.xa)[(size_t)ln * Md4 + bm_off] = xa;
+        reinterpret_cast<float4 *>(p.xm)[(size_t)ln * Md4 + bm_off] = xm;
         nxt = xa;
       }
-      if (NS > 1 && l + 1 == p.L) {
+      if (NS > 1 && ln == p.L) {
 #pragma unroll
         for (int s = 1; s < NS; ++s) nxt = f4_add(nxt, newn[s]);
       }
       if (p.xb != nullptr) {
         __nv_bfloat162 lo = __floats2bfloat162_rn(nxt.x, nxt.y), hi = __floats2bfloat162_rn(nxt.z, nxt.w);
-        reinterpret_cast<uint2 *>(p.xb)[(size_t)(l + 1) * Md4 + bm_off] = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+        reinterpret_cast<uint2 *>(p.xb)[(size_t)ln * Md4 + bm_off] = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
         xs = f4_sq(nxt);
       }
 #pragma unroll
@@ -317,7 +318,7 @@ __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
     }
     if (p.xb != nullptr) {  // this warp holds 128 consecutive columns of the row: partial blockIdx.x
       xs = warp_sum(xs);
-      if (c == 0) p.ssq_x[((size_t)(l + 1) * gridDim.x + blockIdx.x) * p.M + row] = xs;
+      if (c == 0) p.ssq_x[((size_t)ln * gridDim.x + blockIdx.x) * p.M + row] = xs;
     }
     if (want_norm) {
       rs = warp_sum(rs);
@@ -340,7 +341,7 @@ __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
   for (int i = c; i < p.nl * 2; i += 32) {
     double s = 0.0;
     for (unsigned b = 0; b < nblk; ++b) s += (double)__ldcg(&p.partial[(size_t)b * p.nl * 2 + i]);
-    p.resnorm[(size_t)p.l0 * 2 + i] = (float)s;
+    p.resnorm[(size_t)(p.l0 + (i >> 1) * p.lstep) * 2 + (i & 1)] = (float)s;
   }
   __syncwarp();
   if (c == 0) *p.counter = 0u;

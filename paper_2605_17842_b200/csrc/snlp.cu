@@ -105,6 +105,7 @@ struct snlp_model {
   bool capturing = false;
   int64_t cap_nodes = 0;
   std::map<GraphKey, GraphEntry> graphs;
+  std::vector<snlp_kv *> caches;  // live KV caches of this model (orphaned, not freed, by snlp_destroy)
   WMap w_qkv, w_o, w_up, w_dn, w_lm;
   bool have_wmaps = false;
   int n_sm = 148;
@@ -314,6 +315,7 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
 extern "C" int snlp_destroy(snlp_model *m) {
   if (!m) return fail(SNLP_ERR_ARG, "snlp_destroy: NULL handle");
   cudaDeviceSynchronize();
+  for (snlp_kv *kv : m->caches) kv->m = nullptr;  // their memory stays valid until snlp_kv_destroy
   for (auto &g : m->graphs) cudaGraphExecDestroy(g.second.exec);
   if (m->cap_stream) cudaStreamDestroy(m->cap_stream);
   for (const PendingTime &t : m->pending) { cudaEventDestroy(t.e0); cudaEventDestroy(t.e1); }
@@ -444,13 +446,19 @@ static int gemm(snlp_model *m, cudaStream_t st, int cls, const T *A, size_t a_ls
   return SNLP_OK;
 }
 
-static int correct(snlp_model *m, const Fwd &f, int l0, int nl, int mode, int a_splits, int m_splits, float *resnorm) {
+// The structured correction over `nsteps` steps of `lstep` layers starting at state l0 (lstep > 1: fused chunks).
+// a/m: branch outputs at the first layer slot of every step, each the sum of `*_splits` arrays `*_ss` elements apart.
+static int correct(snlp_model *m, const Fwd &f, int l0, int nsteps, int lstep, int mode, int a_splits, size_t a_ss, int m_splits, size_t m_ss,
+                   float *resnorm) {
+  const int nl = nsteps;
   const snlp_config &c = m->cfg;
   CorrParams p{};
   p.trace = m->trace;
   p.a = m->a;
   p.m = m->mb;
-  p.a_ss = p.m_ss = (size_t)c.n_layer * f.M * c.d_model;
+  p.a_ss = a_ss;
+  p.m_ss = m_ss;
+  p.lstep = lstep;
   p.a_splits = a_splits;
   p.m_splits = m_splits;
   p.l0 = l0;
@@ -492,36 +500,44 @@ static int correct(snlp_model *m, const Fwd &f, int l0, int nl, int mode, int a_
   return SNLP_OK;
 }
 
-// Blocks l0 .. l0+nl-1, each on its own current input state (branch outputs a, m; the correction is separate).
+// Blocks l0 .. l0+nl-1 (branch outputs a, m; the correction is separate).  fuse == 1: each block on its own current
+// input state.  fuse > 1: fused chunks (App. C.3): the layers of a chunk read the chunk's input; the per-layer
+// attention outputs a[l] are summed by the consumer (a_splits = fuse), likewise the MLP outputs.
 template <typename T>
-static int blocks_generic(snlp_model *m, const Fwd &f, int l0, int nl) {
+static int blocks_generic(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
   const snlp_config &c = m->cfg;
   const int M = f.M, d = c.d_model, ff = c.d_ff, H = c.n_head, hd = c.head_dim, n = c.n_streams;
   const size_t Md = (size_t)M * d;
   cudaStream_t st = f.st;
-  const float *xa_src = n == 1 ? m->trace + l0 * Md : m->xa + l0 * Md;
-  const float *xm_src = n == 1 ? m->trace + l0 * Md : m->xm + l0 * Md;
-  T *xn = (T *)m->xn + l0 * Md, *q = (T *)m->q + l0 * Md, *att = (T *)m->att + l0 * Md;
-  T *z = (T *)m->z + (size_t)l0 * M * ff;
-  float *qkv = m->qkv_raw + (size_t)l0 * M * 3 * d, *a = m->a + l0 * Md, *y = m->y_raw + (size_t)l0 * M * ff, *mb = m->mb + l0 * Md;
-  T *kc = (T *)f.kc + (size_t)l0 * f.kv_ls, *vc = (T *)f.vc + (size_t)l0 * f.kv_ls;
-
-  KLAUNCH(m, st, KC_OTHER, k_rmsnorm_cast<T><<<dim3(M, nl), 256, 0, st>>>(xa_src, Md, (size_t)d, 1, xn, Md, d, c.rms_eps));
-  TRY(gemm<T>(m, st, KC_QKV, xn, Md, (const T *)m->wqkv + (size_t)l0 * 3 * d * d, (size_t)3 * d * d, qkv, (size_t)M * 3 * d, M, 3 * d, d, nl));
-  KLAUNCH(m, st, KC_OTHER, k_rope_qknorm_store<T><<<dim3(M, 3 * H, nl), 128, 0, st>>>(qkv, (size_t)M * 3 * d, q, Md, kc, vc, f.kv_ls, f.kv_bs, f.T, H, hd, f.pos,
-                                                             m->rope, c.rms_eps));
-  KLAUNCH(m, st, KC_ATTN, k_attn_generic<T><<<dim3((M * H + 3) / 4, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, att, Md, M, f.T, H, hd, f.pos));
-  TRY(gemm<T>(m, st, KC_OPROJ, att, Md, (const T *)m->wo + (size_t)l0 * d * d, (size_t)d * d, a, Md, M, d, d, nl));
-  KLAUNCH(m, st, KC_OTHER, k_resid_rmsnorm_cast<T><<<dim3(M, nl), 256, 0, st>>>(xm_src, Md, (size_t)d, a, Md, 1, 0, m->coef, l0, xn, Md, d, c.rms_eps));
-  TRY(gemm<T>(m, st, KC_UP, xn, Md, (const T *)m->wup + (size_t)l0 * ff * d, (size_t)ff * d, y, (size_t)M * ff, M, ff, d, nl));
-  {
-    const size_t tot = (size_t)nl * M * ff;
-    KLAUNCH(m, st, KC_OTHER, k_relu2_cast<T><<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(y, z, tot));
+  // g layers per launch group, all reading the group's first state when fused
+  const int g = fuse > 1 ? fuse : nl;
+  for (int h0 = l0; h0 < l0 + nl; h0 += g) {
+    const float *xa_src = n == 1 ? m->trace + h0 * Md : m->xa + h0 * Md;
+    const float *xm_src = n == 1 ? m->trace + h0 * Md : m->xm + h0 * Md;
+    T *xn = (T *)m->xn + h0 * Md, *q = (T *)m->q + h0 * Md, *att = (T *)m->att + h0 * Md;
+    T *z = (T *)m->z + (size_t)h0 * M * ff;
+    float *qkv = m->qkv_raw + (size_t)h0 * M * 3 * d, *a = m->a + h0 * Md, *y = m->y_raw + (size_t)h0 * M * ff, *mb = m->mb + h0 * Md;
+    T *kc = (T *)f.kc + (size_t)h0 * f.kv_ls, *vc = (T *)f.vc + (size_t)h0 * f.kv_ls;
+    const int nin = fuse > 1 ? 1 : g;             // distinct input states of the group
+    const size_t in_ls = fuse > 1 ? 0 : Md;       // layer stride of the (possibly shared) GEMM input
+    KLAUNCH(m, st, KC_OTHER, k_rmsnorm_cast<T><<<dim3(M, nin), 256, 0, st>>>(xa_src, Md, (size_t)d, 1, xn, Md, d, c.rms_eps));
+    TRY(gemm<T>(m, st, KC_QKV, xn, in_ls, (const T *)m->wqkv + (size_t)h0 * 3 * d * d, (size_t)3 * d * d, qkv, (size_t)M * 3 * d, M, 3 * d, d, g));
+    KLAUNCH(m, st, KC_OTHER, k_rope_qknorm_store<T><<<dim3(M, 3 * H, g), 128, 0, st>>>(qkv, (size_t)M * 3 * d, q, Md, kc, vc, f.kv_ls, f.kv_bs, f.T, H, hd, f.pos,
+                                                               m->rope, c.rms_eps));
+    KLAUNCH(m, st, KC_ATTN, k_attn_generic<T><<<dim3((M * H + 3) / 4, g), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, att, Md, M, f.T, H, hd, f.pos));
+    TRY(gemm<T>(m, st, KC_OPROJ, att, Md, (const T *)m->wo + (size_t)h0 * d * d, (size_t)d * d, a, Md, M, d, d, g));
+    KLAUNCH(m, st, KC_OTHER, k_resid_rmsnorm_cast<T><<<dim3(M, nin), 256, 0, st>>>(xm_src, Md, (size_t)d, a, Md, fuse > 1 ? fuse : 1, Md, m->coef, h0, xn, Md, d,
+                                                                c.rms_eps));
+    TRY(gemm<T>(m, st, KC_UP, xn, in_ls, (const T *)m->wup + (size_t)h0 * ff * d, (size_t)ff * d, y, (size_t)M * ff, M, ff, d, g));
+    {
+      const size_t tot = (size_t)g * M * ff;
+      KLAUNCH(m, st, KC_OTHER, k_relu2_cast<T><<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(y, z, tot));
+    }
+    TRY(gemm<T>(m, st, KC_DOWN, z, (size_t)M * ff, (const T *)m->wdn + (size_t)h0 * d * ff, (size_t)d * ff, mb, Md, M, d, ff, g));
   }
-  return gemm<T>(m, st, KC_DOWN, z, (size_t)M * ff, (const T *)m->wdn + (size_t)l0 * d * ff, (size_t)d * ff, mb, Md, M, d, ff, nl);
+  return SNLP_OK;
 }
 
-// Tensor-core GEMM of the prefill regime: C[l] = A[l] (M x K, bf16) * W[l]^T (N x K, bf16), nl layers per launch.
 // The tensor-core path (both regimes): bf16, head_dim 128, dims in whole 128-column tiles, weight maps built.
 static bool umma_path_ok(const snlp_model *m) {
   const snlp_config &c = m->cfg;
@@ -558,8 +574,12 @@ static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat1
   const bool small = M <= kDecodeRows;
   if (EPI == UEPI_LMHEAD && !small) return fail(SNLP_ERR_UNSUPPORTED, "LM-head epilogue needs <= %d rows", kDecodeRows);
   CUtensorMap ta;
-  if (!make_tmap_bf16(m->encode_tiled, &ta, A, K, M, nl, a_ls ? a_ls : (size_t)M * K, small ? 16 : kUmmaBM))
+  if (p.a_share < 1) p.a_share = 1;
+  if (p.kfuse < 1) p.kfuse = 1;
+  if (!make_tmap_bf16(m->encode_tiled, &ta, A, K, M, (uint64_t)nl * p.kfuse, a_ls ? a_ls : (size_t)M * K, small ? 16 : kUmmaBM))
     return fail(SNLP_ERR_CUDA, "cuTensorMapEncodeTiled failed (M=%d K=%d)", M, K);
+  if (p.a_share < 1) p.a_share = 1;
+  if (p.kfuse < 1) p.kfuse = 1;
   p.M = M; p.N = N; p.K = K; p.ksplit = ksplit; p.kslice = K / ksplit;
   p.Mt = small ? 1 : (M + kUmmaBM - 1) / kUmmaBM; p.Nt = N / w.BN; p.nl = nl; p.l0 = l0; p.err = m->dev_err;
   const int items = p.Mt * p.Nt * ksplit * nl;
@@ -586,7 +606,7 @@ static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat1
 // xb/ssq_x of the range must be current (prep_rows, or the previous correction).
 static int down_splits(const snlp_model *m, int M);
 
-static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl) {
+static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
   typedef __nv_bfloat16 T;
   const snlp_config &c = m->cfg;
   const int M = f.M, d = c.d_model, ff = c.d_ff, H = c.n_head, n = c.n_streams, P = d / 128, L = c.n_layer;
@@ -605,6 +625,7 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl) {
     p.ssq = m->ssq_x + (size_t)l0 * P * M; p.nparts = P; p.eps = c.rms_eps;
     p.q = q; p.q_ls = Md; p.kc = kc; p.vc = vc; p.kv_ls = f.kv_ls; p.kv_bs = f.kv_bs;
     p.T = f.T; p.d = d; p.pos_base = f.pos; p.rope = m->rope; p.qk_eps = c.rms_eps;
+    p.a_share = fuse;
     TRY(umma_gemm<UEPI_QKV>(m, st, KC_QKV, xb, Md, m->w_qkv, l0, p, M, 3 * d, d, 1, nl));
   }
   if (small) {
@@ -620,18 +641,21 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl) {
     UmmaParams p{};
     p.c = a; p.z = ub; p.out_ls = Md;
     p.xm = xm_src; p.xm_ls = Md; p.coef = m->coef + l0; p.ssq_out = m->ssq_u + (size_t)l0 * Pu * M;
-    TRY(umma_gemm<UEPI_RESID>(m, st, KC_OPROJ, att, Md, m->w_o, l0, p, M, d, d, 1, nl));
+    p.kfuse = fuse;   // a chunk's out-projections are one product over the concatenated attention outputs
+    TRY(umma_gemm<UEPI_RESID>(m, st, KC_OPROJ, att, Md, m->w_o, l0, p, M, d, d, 1, nl / fuse));
   }
   {
     UmmaParams p{};
     p.z = z; p.out_ls = (size_t)M * ff;
     p.ssq = m->ssq_u + (size_t)l0 * Pu * M; p.nparts = Pu; p.eps = c.rms_eps;
+    p.a_share = fuse;
     TRY(umma_gemm<UEPI_RELU2_BF16>(m, st, KC_UP, ub, Md, m->w_up, l0, p, M, ff, d, 1, nl));
   }
   {
     UmmaParams p{};
     p.c = mb; p.out_ls = Md; p.out_ss = (size_t)L * Md;
-    TRY(umma_gemm<UEPI_F32>(m, st, KC_DOWN, z, (size_t)M * ff, m->w_dn, l0, p, M, d, ff, sd, nl));
+    p.kfuse = fuse;
+    TRY(umma_gemm<UEPI_F32>(m, st, KC_DOWN, z, (size_t)M * ff, m->w_dn, l0, p, M, d, ff, sd, nl / fuse));
   }
   return SNLP_OK;
 }
@@ -670,10 +694,18 @@ static int init_kernel_attributes() {
   return SNLP_OK;
 }
 
-static int run_blocks(snlp_model *m, const Fwd &f, int l0, int nl) {
-  if (umma_path_ok(m)) return blocks_umma(m, f, l0, nl);
-  if (m->cfg.dtype == SNLP_DTYPE_BF16) return blocks_generic<__nv_bfloat16>(m, f, l0, nl);
-  return blocks_generic<float>(m, f, l0, nl);
+static int run_blocks(snlp_model *m, const Fwd &f, int l0, int nl, int fuse = 1) {
+  if (umma_path_ok(m)) return blocks_umma(m, f, l0, nl, fuse);
+  if (m->cfg.dtype == SNLP_DTYPE_BF16) return blocks_generic<__nv_bfloat16>(m, f, l0, nl, fuse);
+  return blocks_generic<float>(m, f, l0, nl, fuse);
+}
+
+// The correction over layers l0 .. l0+nl-1 in steps of `fuse` layers, on the branch outputs run_blocks left.
+static int correct_range(snlp_model *m, const Fwd &f, int l0, int nl, int fuse, int mode, float *resnorm) {
+  const size_t Md = (size_t)f.M * m->cfg.d_model;
+  if (umma_path_ok(m))  // a, m at the chunk's first layer slot; m possibly in K-split partials
+    return correct(m, f, l0, nl / fuse, fuse, mode, 1, 0, down_splits(m, f.M), (size_t)m->cfg.n_layer * Md, resnorm);
+  return correct(m, f, l0, nl / fuse, fuse, mode, fuse, Md, fuse, Md, resnorm);  // per-layer outputs, summed here
 }
 
 static int native_mode(const snlp_model *m) { return m->cfg.n_streams > 1 ? SNLP_MODE_HCN : SNLP_MODE_IDN; }
@@ -698,47 +730,57 @@ static int check_solver(const snlp_model *m, const snlp_solver &sol, const char 
     if (m->cfg.n_streams != 1) return fail(SNLP_ERR_UNSUPPORTED, "%s: fused chunks need a single-stream model", who);
     if ((L - sol.prefix) % sol.fuse) return fail(SNLP_ERR_ARG, "%s: suffix length %d is not a multiple of fuse = %d", who, L - sol.prefix, sol.fuse);
     if (sol.mode == SNLP_MODE_HCN) return fail(SNLP_ERR_ARG, "%s: fused chunks use the identity surrogate (mode IDN or NOCORR)", who);
-    return fail(SNLP_ERR_UNSUPPORTED, "%s: fuse > 1 is not built yet", who);
   }
   return SNLP_OK;
 }
 
-// General Alg. 2 over the internal trace (trace[0] must hold h_0): sequential prefix, initialisation, K sweeps.
+// General Alg. 2 over the internal trace (trace[0] must hold h_0): sequential prefix, initialisation, K sweeps over the
+// suffix in chunks of `fuse` fused layers (Eq. 5 for fuse = 1, Eq. 11 otherwise).
 static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *resnorm_out) {
   const snlp_config &c = m->cfg;
-  const int L = c.n_layer, S = sol.mode == SNLP_MODE_SEQUENTIAL ? L : sol.prefix;
-  if (resnorm_out && sol.K > 0) CU(cudaMemsetAsync(resnorm_out, 0, (size_t)sol.K * L * 2 * sizeof(float), f.st));
+  const int L = c.n_layer, F = sol.fuse;
+  const bool seq = sol.mode == SNLP_MODE_SEQUENTIAL;
+  const int S = (seq && F == 1) ? L : sol.prefix;
+  if (resnorm_out && sol.K > 0 && !seq) CU(cudaMemsetAsync(resnorm_out, 0, (size_t)sol.K * L * 2 * sizeof(float), f.st));
   if (S > 0) {  // Alg. 2 lines 2-4
     if (umma_path_ok(m)) TRY(prep_rows(m, f, 0, 1));
     else TRY(premix(m, f, 0, 1));
     for (int l = 0; l < S; ++l) {
       TRY(run_blocks(m, f, l, 1));
-      TRY(correct(m, f, l, 1, native_mode(m), 1, down_splits(m, f.M), nullptr));
+      TRY(correct_range(m, f, l, 1, 1, native_mode(m), nullptr));
     }
   }
   if (S == L) return SNLP_OK;
+  if (seq) {  // sequential execution of the fused model: chunk after chunk
+    if (umma_path_ok(m)) TRY(prep_rows(m, f, S, 1));
+    for (int h = S; h < L; h += F) {
+      TRY(run_blocks(m, f, h, F, F));
+      TRY(correct_range(m, f, h, F, F, SNLP_MODE_IDN, nullptr));
+    }
+    return SNLP_OK;
+  }
   // Alg. 2 line 5: every suffix state starts at h_S
   const size_t n4 = (size_t)f.M * c.n_streams * c.d_model / 4;
   KLAUNCH(m, f.st, KC_OTHER, k_bcast_trace<<<(unsigned)((n4 + 255) / 256), 256, 0, f.st>>>(reinterpret_cast<const float4 *>(m->trace) + (size_t)S * n4,
                                                                reinterpret_cast<float4 *>(m->trace) + (size_t)(S + 1) * n4, n4, L - S));
   if (umma_path_ok(m)) TRY(prep_rows(m, f, S, L - S));
   else TRY(premix(m, f, S, L - S));
-  int exact = S;  // states 0..exact equal the sequential trace
+  int exact = S;  // states 0..exact equal the sequential trace (of the fused model when F > 1)
   if (sol.init == SNLP_INIT_FWD) {
-    // one batched evaluation of every suffix block on h_S; with A = 0 the correction just stores F_l(h_S)
-    TRY(run_blocks(m, f, S, L - S));
-    TRY(correct(m, f, S, L - S, SNLP_MODE_NOCORR, 1, down_splits(m, f.M), nullptr));
-    exact = S + 1;
+    // one batched evaluation of every suffix chunk on h_S; with A = 0 the correction just stores F(h_S)
+    TRY(run_blocks(m, f, S, L - S, F));
+    TRY(correct_range(m, f, S, L - S, F, SNLP_MODE_NOCORR, nullptr));
+    exact = S + F;
   }
   for (int k = 0; k < sol.K; ++k) {
     // Exactness-aware trimming: entering this sweep the states 0..exact already equal the sequential trace (Newton
-    // on a block lower-bidiagonal system), so blocks before `exact` would reproduce, bit for bit, the branch
-    // outputs they wrote in the previous pass.  Only blocks exact..L-1 are evaluated; the correction still runs
+    // on a block lower-bidiagonal system), so chunks before `exact` would reproduce, bit for bit, the branch
+    // outputs they wrote in the previous pass.  Only chunks from `exact` on are evaluated; the correction still runs
     // over the whole suffix on the stored branch outputs, so trace, residual norms and next inputs are unchanged.
     const int b0 = exact < L ? exact : L;
-    if (b0 < L) TRY(run_blocks(m, f, b0, L - b0));
-    TRY(correct(m, f, S, L - S, sol.mode, 1, down_splits(m, f.M), resnorm_out ? resnorm_out + (size_t)k * L * 2 : nullptr));
-    ++exact;
+    if (b0 < L) TRY(run_blocks(m, f, b0, L - b0, F));
+    TRY(correct_range(m, f, S, L - S, F, sol.mode, resnorm_out ? resnorm_out + (size_t)k * L * 2 : nullptr));
+    exact += F;
   }
   return SNLP_OK;
 }
@@ -913,6 +955,7 @@ extern "C" int snlp_kv_create(snlp_model *m, int B, int max_ctx, snlp_kv **out) 
     delete kv;
     return fail(SNLP_ERR_CUDA, "snlp_kv_create: cudaMemset failed");
   }
+  m->caches.push_back(kv);
   *out = kv;
   return SNLP_OK;
 }
@@ -920,10 +963,12 @@ extern "C" int snlp_kv_create(snlp_model *m, int B, int max_ctx, snlp_kv **out) 
 extern "C" int snlp_kv_destroy(snlp_kv *kv) {
   if (!kv) return fail(SNLP_ERR_ARG, "snlp_kv_destroy: NULL handle");
   cudaDeviceSynchronize();
-  // graphs captured against this cache hold its pointers
-  for (auto it = kv->m->graphs.begin(); it != kv->m->graphs.end();) {
-    if (it->first.kv == kv) { cudaGraphExecDestroy(it->second.exec); it = kv->m->graphs.erase(it); }
-    else ++it;
+  if (kv->m) {  // the model is still alive: drop the graphs captured against this cache (they hold its pointers)
+    for (auto it = kv->m->graphs.begin(); it != kv->m->graphs.end();) {
+      if (it->first.kv == kv) { cudaGraphExecDestroy(it->second.exec); it = kv->m->graphs.erase(it); }
+      else ++it;
+    }
+    kv->m->caches.erase(std::remove(kv->m->caches.begin(), kv->m->caches.end(), kv), kv->m->caches.end());
   }
   cudaFree(kv->k); cudaFree(kv->v); cudaFree(kv->pos);
   delete kv;
@@ -938,6 +983,7 @@ extern "C" int snlp_kv_len(const snlp_kv *kv, int32_t *len) {
 
 extern "C" int snlp_kv_truncate(snlp_kv *kv, int new_len, void *stream) {
   if (!kv) return fail(SNLP_ERR_ARG, "snlp_kv_truncate: NULL handle");
+  if (!kv->m) return fail(SNLP_ERR_STATE, "snlp_kv_truncate: the model of this cache has been destroyed");
   if (new_len < 0 || new_len > kv->len) return fail(SNLP_ERR_ARG, "snlp_kv_truncate: new_len = %d outside 0..%d", new_len, kv->len);
   KLAUNCH(kv->m, (cudaStream_t)stream, KC_OTHER, k_set_int<<<1, 1, 0, (cudaStream_t)stream>>>(kv->pos, new_len));
   kv->len = new_len;

@@ -38,6 +38,12 @@ struct UmmaParams {
   int kslice, ksplit;      // K split: kslice = K / ksplit (a multiple of 64)
   int Mt, Nt, nl, l0;      // row tiles, column tiles, layers of the launch; l0 = first layer's coordinate in the weight map
   int nstages;             // ring depth
+  // Fused chunks (several layers reading one input, App. C.3).  a_share > 1: the `nl` items' layers are grouped in
+  // chunks of a_share and every layer of a chunk reads the A rows (and their sums of squares) of the chunk's first
+  // layer -- the column-concatenated form (QKV, MLP up).  kfuse > 1: an item is a chunk; its reduction runs over the
+  // kfuse layers' A rows and weights in turn and accumulates into one output -- the K-concatenated form
+  // (attention out-projection, MLP down); outputs and epilogue inputs are indexed by the chunk's first layer.
+  int a_share, kfuse;
   float *c;                // UEPI_F32 / UEPI_RESID: [ksplit][nl][M][N] fp32
   __nv_bfloat16 *z;        // UEPI_RELU2_BF16: [nl][M][N] bf16;  UEPI_RESID: bf16(u) [nl][M][N]
   size_t out_ls, out_ss;   // layer / split stride of the outputs above (elements)
@@ -191,12 +197,12 @@ struct UmmaCfg {
 
 // ---- epilogue of the prefill regime: thread = accumulator row ----------------------------------------
 template <int BN, int EPI>
-__device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t tbase, int row, int n_tile, int ks, int l) {
+__device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t tbase, int row, int n_tile, int ks, int l, int ls) {
   const bool live = row < p.M;
   float rstd = 1.f;
   if ((EPI == UEPI_QKV || EPI == UEPI_RELU2_BF16) && p.ssq != nullptr && live) {
     float ss = 0.f;
-    for (int i = 0; i < p.nparts; ++i) ss += p.ssq[((size_t)l * p.nparts + i) * p.M + row];
+    for (int i = 0; i < p.nparts; ++i) ss += p.ssq[((size_t)ls * p.nparts + i) * p.M + row];
     rstd = rsqrtf(ss / (float)p.K + p.eps);
   }
   if (EPI == UEPI_F32 || EPI == UEPI_RELU2_BF16) {
@@ -331,13 +337,13 @@ __device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t
 // ---- epilogue of the decode regime: accumulator rows (tokens) already transposed into outs[16][BN+1] ----
 // ew = epilogue warp 0..3, lane; one warp per token, lanes across the tile's columns.
 template <int BN, int EPI>
-__device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const float *outs, int ew, int lane, int n_tile, int ks, int l) {
+__device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const float *outs, int ew, int lane, int n_tile, int ks, int l, int ls) {
   for (int tok = ew; tok < p.M; tok += 4) {
     const float *y = outs + tok * (BN + 1);
     float rstd = 1.f;
     if ((EPI == UEPI_QKV || EPI == UEPI_RELU2_BF16 || EPI == UEPI_LMHEAD) && p.ssq != nullptr) {
       float ss = 0.f;
-      for (int i = 0; i < p.nparts; ++i) ss += p.ssq[((size_t)l * p.nparts + i) * p.M + tok];
+      for (int i = 0; i < p.nparts; ++i) ss += p.ssq[((size_t)ls * p.nparts + i) * p.M + tok];
       rstd = rsqrtf(ss / (float)p.K + p.eps);
     }
     const size_t n0 = (size_t)n_tile * BN;
@@ -434,7 +440,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nkb = p.kslice / kUmmaBK;
+  const int nkb1 = p.kslice / kUmmaBK;      // k-blocks of one layer's K slice
+  const int nkb = nkb1 * p.kfuse;           // k-blocks of one item
   const int n_items = p.Mt * p.Nt * p.ksplit * p.nl;
   const int my_items = (int)blockIdx.x < n_items ? (n_items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
   constexpr uint32_t kTmemCols = 2 * BN;
@@ -466,7 +473,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
   const int m_tile = it_ % p.Mt;                                  \
   const int n_tile = (it_ / p.Mt) % p.Nt;                         \
   const int ks = (it_ / (p.Mt * p.Nt)) % p.ksplit;                \
-  const int l = it_ / (p.Mt * p.Nt * p.ksplit);
+  const int li_ = it_ / (p.Mt * p.Nt * p.ksplit);                 /* layer (or chunk) of the launch */ \
+  const int la = p.a_share > 1 ? (li_ / p.a_share) * p.a_share : li_ * p.kfuse; /* A rows' layer slot */ \
+  const int l = li_ * p.kfuse;                                    /* output / weight layer slot */
 
   if (warp == 0) {
     if (lane == 0) {
@@ -479,9 +488,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
           ok = mbar_wait(&empty[s], ((g / S) & 1) ^ 1u, abort_flag, p.err);
           if (!ok) break;
           mbar_expect_tx(&full[s], Cfg::kABytes + Cfg::kBBytes);
-          const int k0 = ks * p.kslice + kb * kUmmaBK;
-          tma_load_3d(sA + (size_t)s * Cfg::kABytes, &tmA, &full[s], k0, m_tile * kUmmaBM, l);
-          tma_load_3d(sB + (size_t)s * Cfg::kBBytes, &tmB, &full[s], k0, n_tile * BN, p.l0 + l);
+          const int j = kb / nkb1, k0 = ks * p.kslice + (kb % nkb1) * kUmmaBK;   // j: layer inside a K-concatenated chunk
+          tma_load_3d(sA + (size_t)s * Cfg::kABytes, &tmA, &full[s], k0, m_tile * kUmmaBM, la + j);
+          tma_load_3d(sB + (size_t)s * Cfg::kBBytes, &tmB, &full[s], k0, n_tile * BN, p.l0 + l + j);
           issued = g + 1;
         }
       }
@@ -530,7 +539,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
       tc_fence_after();
       const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * BN;
       if (AM == kUmmaBM) {
-        umma_epilogue_rows<BN, EPI>(p, tbase, m_tile * kUmmaBM + quarter * 32 + lane, n_tile, ks, l);
+        umma_epilogue_rows<BN, EPI>(p, tbase, m_tile * kUmmaBM + quarter * 32 + lane, n_tile, ks, l, la);
         tc_fence_before();
         epi_bar_sync();
         if (et == 0) mbar_arrive(&accempty[b]);
@@ -549,7 +558,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
         tc_fence_before();
         epi_bar_sync();
         if (et == 0) mbar_arrive(&accempty[b]);
-        umma_epilogue_small<BN, EPI>(p, outs, ew, lane, n_tile, ks, l);
+        umma_epilogue_small<BN, EPI>(p, outs, ew, lane, n_tile, ks, l, la);
         epi_bar_sync();  // outs is reused by the next item
       }
     }

@@ -79,3 +79,19 @@ def test_error_codes(env):
     assert torch.isfinite(tr).all()
     # the context is still healthy after all the refused calls
     torch.cuda.synchronize()
+
+
+def test_cache_may_outlive_its_model(env):
+    snlp, cfg, W = env
+    m = snlp.Model(cfg, max_rows=16, max_batch=1, max_ctx=16)
+    m.load_weights(W)
+    kv = m.kv_cache(1, 16)
+    ids = torch.zeros((1, 4), dtype=torch.int32, device="cuda")
+    t = m.prefill(kv, ids)
+    m.decode_step(kv, t, 2)          # leaves a captured graph that refers to the cache
+    torch.cuda.synchronize()
+    m.close()                        # model first ...
+    with pytest.raises(snlp.SnlpError) as e:
+        kv.truncate(1)
+    assert e.value.code == snlp.ERR_STATE
+    kv.close()                       # ... then the cache: must not touch the freed model

@@ -76,3 +76,64 @@ def test_decode_step_with_prefix_and_fwd_init():
         b = m.decode_step_solver(kv, a, sol).clone()
         assert torch.equal(a, ref[0]) and torch.equal(b, ref[1])
     assert len(kv) == 22
+
+
+FUSED = {
+    "f32": (synth.ModelConfig(6, 64, 2, 32, 128, 128, 1, "fp32"), 2, 9),
+    "bf16_decode": (synth.ModelConfig(6, 256, 2, 128, 512, 1024, 1, "bf16"), 2, 5),
+    "bf16_prefill": (synth.ModelConfig(6, 256, 2, 128, 640, 1024, 1, "bf16"), 1, 140),
+}
+
+
+@pytest.mark.parametrize("name", list(FUSED))
+def test_fused_chunks_match_oracle(name):
+    """Chunkwise SNLP with fused layers (NxFM): the chunk-boundary states against the oracle's forward_chunked."""
+    from paper_2605_17842_b200 import snlp
+    cfg, B, T = FUSED[name]
+    W = synth.make_weights(cfg, seed=1234, std=0.05, embed_std=1.0)
+    h0 = synth.make_hidden(cfg, B, T, seed=7)
+    m = make_model(cfg, W, max_rows=B * T, max_batch=B)
+    L = cfg.n_layer
+    for S, F, K, init in [(0, 2, 1, O.INIT_H0), (0, 2, 2, O.INIT_H0), (0, 3, 1, O.INIT_FWD), (2, 2, 1, O.INIT_H0), (0, 6, 1, O.INIT_H0)]:
+        want = O.forward_chunked(cfg, W, h0.astype(np.float64), K, F, S=S, init=init)
+        tr, _ = m.forward_solver(dev(h0), snlp.Solver(K=K, mode=O.MODE_IDN, prefix=S, init=init, fuse=F))
+        got = tr.cpu().numpy()[S::F]
+        assert got.shape[0] == len(want)
+        assert layer_relerr(got, np.stack(want)) <= TOL[cfg.dtype], (S, F, K, init)
+        # sequential execution of the same fused model, and chunkwise finite-step exactness against it (bit for bit)
+        fseq_want = O.forward_chunked(cfg, W, h0.astype(np.float64), None, F, S=S)
+        fseq, _ = m.forward_solver(dev(h0), snlp.Solver(K=0, mode=snlp.MODE_SEQUENTIAL, prefix=S, fuse=F))
+        assert layer_relerr(fseq.cpu().numpy()[S::F], np.stack(fseq_want)) <= TOL[cfg.dtype], (S, F)
+        nexact = min((L - S) // F, K + (1 if init == O.INIT_FWD else 0))
+        assert torch.equal(tr[S::F][:nexact + 1], fseq[S::F][:nexact + 1]), (S, F, K, init)
+    # fuse = 1 through the same entry point is the unfused algorithm
+    a, _ = m.forward_solver(dev(h0), snlp.Solver(K=2, mode=O.MODE_IDN, fuse=1))
+    b, _ = m.forward_parallel(dev(h0), 2, O.MODE_IDN)
+    assert torch.equal(a, b)
+    # without correction (A = 0) information moves one chunk per sweep
+    want = O.forward_chunked(cfg, W, h0.astype(np.float64), 1, 2, correct=False)
+    tr, _ = m.forward_solver(dev(h0), snlp.Solver(K=1, mode=O.MODE_NOCORR, fuse=2))
+    assert layer_relerr(tr.cpu().numpy()[0::2], np.stack(want)) <= TOL[cfg.dtype]
+    m.device_status()
+
+
+def test_fused_decode_steps_are_consistent():
+    """Decoding with fused chunks: enough sweeps reproduce sequential execution of the fused model, token for token."""
+    from paper_2605_17842_b200 import snlp
+    cfg = synth.ModelConfig(6, 256, 2, 128, 512, 1024, 1, "bf16")
+    W = synth.make_weights(cfg, seed=1234, std=0.05, embed_std=1.0)
+    m = make_model(cfg, W, max_rows=32, max_batch=2, max_ctx=64)
+    ids = dev(synth.make_ids(cfg, 2, 20, seed=5))
+    kv = m.kv_cache(2, 64)
+    first = m.prefill(kv, ids)
+    seq = snlp.Solver(K=0, mode=snlp.MODE_SEQUENTIAL, fuse=2)
+    ref = [m.decode_step_solver(kv, first, seq).clone()]
+    ref.append(m.decode_step_solver(kv, ref[-1], seq).clone())
+    kv.truncate(20)
+    sol = snlp.Solver(K=3, mode=O.MODE_IDN, fuse=2)     # 3 chunks, 3 sweeps: exact
+    a = m.decode_step_solver(kv, first, sol).clone()
+    b = m.decode_step_solver(kv, a, sol).clone()
+    assert torch.equal(a, ref[0]) and torch.equal(b, ref[1])
+    with pytest.raises(snlp.SnlpError) as e:
+        m.decode_step_solver(kv, first, snlp.Solver(K=1, mode=O.MODE_HCN, fuse=2))
+    assert e.value.code == snlp.ERR_ARG
