@@ -43,6 +43,9 @@ CONFIGS = {
     "d12": ModelConfig(12, 768, 6, 128, 3072, 32768, 1, "bf16"),
     "d20": ModelConfig(20, 1280, 10, 128, 5120, 65536, 1, "bf16"),
     "d20_hc": ModelConfig(20, 1280, 10, 128, 5120, 65536, 4, "bf16"),
+    # the shape of the paper's own 0.5B model without x0-residual / value embeddings (Sec. 5: 32 layers, n_embd 640,
+    # 5 heads); MLP width 4 d and the 65536-entry vocabulary are the Nanochat defaults, not stated in the paper
+    "paper_0p5b": ModelConfig(32, 640, 5, 128, 2560, 65536, 1, "bf16"),
 }
 
 
