@@ -288,7 +288,6 @@ static __global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat
   const __nv_bfloat16 *kp = kc + (size_t)l * kv_ls + (size_t)b * kv_bs + h * 128 + li * 8;
   const __nv_bfloat16 *vp = vc + (size_t)l * kv_ls + (size_t)b * kv_bs + h * 128 + li * 8;
   float *pbase = part + (size_t)((size_t)l * gridDim.y + bh) * Tq * nchunk * kAttnPartStride;
-  constexpr int J = kAttnSub / 8;
   for (int t = 0; t < Tq; ++t) {
     const int pos_q = pos0 + t;
     float *dst = pbase + ((size_t)t * nchunk + chunk) * kAttnPartStride;
@@ -302,21 +301,23 @@ static __global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat
     for (int i = 0; i < 8; ++i) qv[i] = qs[t][li * 8 + i];
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     float mrun = -INFINITY, lrun = 0.f;
-    for (int sb = 0; sb < csub; ++sb) {
-      const int base = kbeg + sb * kAttnSub;
-      if (base > pos_q) break;
-      uint4 kr[J], vr[J];
+    // The chunk is walked in 32-key mini-blocks (4 keys per half-warp), software-pipelined through two register
+    // buffers: the loads of the next mini-block are in flight while the current one is reduced.
+    constexpr int JM = 4;
+    auto load_mb = [&](uint4 (&kr)[JM], uint4 (&vr)[JM], int base) {
 #pragma unroll
-      for (int j = 0; j < J; ++j) {
+      for (int j = 0; j < JM; ++j) {
         const int key = base + hw + 8 * j;
         const bool ok = key <= pos_q;
         kr[j] = ok ? ldg_stream(kp + (size_t)key * d) : make_uint4(0, 0, 0, 0);
         vr[j] = ok ? ldg_stream(vp + (size_t)key * d) : make_uint4(0, 0, 0, 0);
       }
-      float s[J];
+    };
+    auto reduce_mb = [&](const uint4 (&kr)[JM], const uint4 (&vr)[JM], int base) {
+      float s[JM];
       float mloc = -INFINITY;
 #pragma unroll
-      for (int j = 0; j < J; ++j) {
+      for (int j = 0; j < JM; ++j) {
         const int key = base + hw + 8 * j;
         const __nv_bfloat162 *k2 = reinterpret_cast<const __nv_bfloat162 *>(&kr[j]);
         float dot = 0.f;
@@ -333,14 +334,14 @@ static __global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat
         s[j] = key <= pos_q ? dot : -INFINITY;
         mloc = fmaxf(mloc, s[j]);
       }
-      if (mloc == -INFINITY) continue;  // none of this half-warp's keys of the sub-block is visible
+      if (mloc == -INFINITY) return;  // none of this half-warp's keys of the mini-block is visible
       const float mnew = fmaxf(mrun, mloc);
       const float resc = mrun == -INFINITY ? 0.f : __expf(mrun - mnew);
       lrun *= resc;
 #pragma unroll
       for (int i = 0; i < 8; ++i) acc[i] *= resc;
 #pragma unroll
-      for (int j = 0; j < J; ++j) {
+      for (int j = 0; j < JM; ++j) {
         const float pj = s[j] == -INFINITY ? 0.f : __expf(s[j] - mnew);
         lrun += pj;
         const __nv_bfloat162 *v2 = reinterpret_cast<const __nv_bfloat162 *>(&vr[j]);
@@ -352,6 +353,20 @@ static __global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat
         }
       }
       mrun = mnew;
+    };
+    {
+      const int vis = (pos_q - kbeg) / 32 + 1;                         // mini-blocks with at least one visible key
+      const int nmb = vis < csub * (kAttnSub / 32) ? vis : csub * (kAttnSub / 32);
+      uint4 ka[JM], va[JM], kb2[JM], vb2[JM];
+      load_mb(ka, va, kbeg);
+      for (int mb = 0; mb < nmb; mb += 2) {
+        if (mb + 1 < nmb) load_mb(kb2, vb2, kbeg + (mb + 1) * 32);
+        reduce_mb(ka, va, kbeg + mb * 32);
+        if (mb + 1 < nmb) {
+          if (mb + 2 < nmb) load_mb(ka, va, kbeg + (mb + 2) * 32);
+          reduce_mb(kb2, vb2, kbeg + (mb + 1) * 32);
+        }
+      }
     }
 #pragma unroll
     for (int i = 0; i < 8; ++i) hacc[hw][li * 8 + i] = acc[i];
