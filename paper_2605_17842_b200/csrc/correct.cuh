@@ -57,23 +57,34 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
 
   float4 oldp[NS], newp[NS];
+  // operands of one step: branch outputs and the old next state; fetched one step ahead of their use
+  float4 av_n, mv_n, oldn_n[NS];
+  auto fetch = [&](int i, float4 &av, float4 &mv, float4 (&on)[NS]) {
+    const int l = p.l0 + i * p.lstep, ln = l + p.lstep;
+    av = a4[(size_t)l * Md4 + bm_off];
+    for (int q = 1; q < p.a_splits; ++q) av = f4_add(av, a4[(size_t)q * (p.a_ss >> 2) + (size_t)l * Md4 + bm_off]);
+    mv = m4[(size_t)l * Md4 + bm_off];
+    for (int q = 1; q < p.m_splits; ++q) mv = f4_add(mv, m4[(size_t)q * (p.m_ss >> 2) + (size_t)l * Md4 + bm_off]);
+#pragma unroll
+    for (int r = 0; r < NS; ++r) on[r] = tr4[(size_t)ln * state4 + st_off + (size_t)r * d4];
+  };
   if (active) {
 #pragma unroll
     for (int s = 0; s < NS; ++s) oldp[s] = newp[s] = tr4[(size_t)p.l0 * state4 + st_off + (size_t)s * d4];
+    if (p.nl > 0) fetch(0, av_n, mv_n, oldn_n);
   }
   for (int i = 0; i < p.nl; ++i) {
     const int l = p.l0 + i * p.lstep, ln = l + p.lstep;  // this step maps state l to state ln
     float rs = 0.f, hs = 0.f, xs = 0.f;
     if (active) {
-      float4 av = a4[(size_t)l * Md4 + bm_off];
-      for (int q = 1; q < p.a_splits; ++q) av = f4_add(av, a4[(size_t)q * (p.a_ss >> 2) + (size_t)l * Md4 + bm_off]);
-      float4 mv = m4[(size_t)l * Md4 + bm_off];
-      for (int q = 1; q < p.m_splits; ++q) mv = f4_add(mv, m4[(size_t)q * (p.m_ss >> 2) + (size_t)l * Md4 + bm_off]);
+      const float4 av = av_n, mv = mv_n;
       const HcCoef &c = p.coef[l];
       float4 oldn[NS], newn[NS], tilde[NS];
 #pragma unroll
+      for (int r = 0; r < NS; ++r) oldn[r] = oldn_n[r];
+      if (i + 1 < p.nl) fetch(i + 1, av_n, mv_n, oldn_n);  // the next step's loads overlap this step's arithmetic and stores
+#pragma unroll
       for (int r = 0; r < NS; ++r) {
-        oldn[r] = tr4[(size_t)ln * state4 + st_off + (size_t)r * d4];
         if (NS == 1) {
           tilde[r] = f4_add(f4_add(oldp[0], av), mv);  // F_l(h_l^k) = (h + a) + m
         } else {

@@ -250,7 +250,7 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
   if (c.dtype == SNLP_DTYPE_BF16 && d % 128 == 0) {
     A(&m->ub, L * R * d * es);
     A(&m->ssq_x, (L + 1) * (d / 128) * R * 4);
-    A(&m->ssq_u, L * (d / 128) * R * 4);
+    A(&m->ssq_u, L * 2 * (d / 128) * R * 4);
     A(&m->ssq_lm, (size_t)(d / 128) * kDecodeRows * 4);
   }
   A(&m->q, L * R * d * es);
@@ -618,7 +618,7 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
   T *z = (T *)m->z + (size_t)l0 * M * ff;
   float *a = m->a + l0 * Md, *mb = m->mb + l0 * Md;
   T *kc = (T *)f.kc + (size_t)l0 * f.kv_ls, *vc = (T *)f.vc + (size_t)l0 * f.kv_ls;
-  const int Pu = d / m->w_o.BN;  // column tiles of the out-projection = partials of sum u^2
+  const int Pu = 2 * (d / m->w_o.BN);  // partials of sum u^2: two per column tile of the out-projection
   const int sd = down_splits(m, M);
   {
     UmmaParams p{};

@@ -56,7 +56,8 @@ struct UmmaParams {
   float *logits; float *pm_val; int *pm_idx;                            // UEPI_LMHEAD
 };
 
-constexpr int kUmmaThreads = 192;   // warp 0: TMA, warp 1: MMA + TMEM allocation, warps 2-5: epilogue
+constexpr int kUmmaThreads = 320;   // warp 0: TMA, warp 1: MMA + TMEM allocation, warps 2-9: epilogue (two per TMEM lane quarter)
+constexpr int kUmmaEpiThreads = 256;
 constexpr int kUmmaBM = 128;
 constexpr int kUmmaBK = 64;         // 64 bf16 = one 128-byte swizzle row
 constexpr int kUmmaSmemBudget = 222 * 1024;
@@ -150,12 +151,12 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-// Barrier over the 128 epilogue threads (named barrier 1), plain and with an AND-reduced predicate: after a
+// Barrier over the 256 epilogue threads (named barrier 1), plain and with an AND-reduced predicate: after a
 // bounded wait every thread learns whether all of them got through, so they leave the item loop together.
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ bool epi_all(bool v) {
   uint32_t out;
-  asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 q, %1, 0;\n bar.red.and.pred p, 1, 128, q;\n selp.b32 %0, 1, 0, p;\n}"
+  asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 q, %1, 0;\n bar.red.and.pred p, 1, 256, q;\n selp.b32 %0, 1, 0, p;\n}"
                : "=r"(out)
                : "r"((uint32_t)v)
                : "memory");
@@ -196,8 +197,9 @@ struct UmmaCfg {
 };
 
 // ---- epilogue of the prefill regime: thread = accumulator row ----------------------------------------
+// grp = 0/1: which half of the tile's columns (or which head of a 256-wide QKV tile) this warp owns.
 template <int BN, int EPI>
-__device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t tbase, int row, int n_tile, int ks, int l, int ls) {
+__device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t tbase, int row, int n_tile, int ks, int l, int ls, int grp) {
   const bool live = row < p.M;
   float rstd = 1.f;
   if ((EPI == UEPI_QKV || EPI == UEPI_RELU2_BF16) && p.ssq != nullptr && live) {
@@ -205,9 +207,10 @@ __device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t
     for (int i = 0; i < p.nparts; ++i) ss += p.ssq[((size_t)ls * p.nparts + i) * p.M + row];
     rstd = rsqrtf(ss / (float)p.K + p.eps);
   }
+  constexpr int kHalf = BN / 64;  // 32-column chunks per warp group
   if (EPI == UEPI_F32 || EPI == UEPI_RELU2_BF16) {
 #pragma unroll 1
-    for (int c = 0; c < BN / 32; ++c) {
+    for (int c = grp * kHalf; c < (grp + 1) * kHalf; ++c) {
       uint32_t r[32];
       tmem_ld32(tbase + c * 32, r);
       if (live) {
@@ -238,7 +241,7 @@ __device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t
     const float kappa = p.coef[l].kappa;
     float ss = 0.f;
 #pragma unroll 1
-    for (int c = 0; c < BN / 32; ++c) {
+    for (int c = grp * kHalf; c < (grp + 1) * kHalf; ++c) {
       uint32_t r[32];
       tmem_ld32(tbase + c * 32, r);
       if (live) {
@@ -265,11 +268,11 @@ __device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t
         }
       }
     }
-    if (live) p.ssq_out[((size_t)l * p.Nt + n_tile) * p.M + row] = ss;
+    if (live) p.ssq_out[(((size_t)l * p.Nt + n_tile) * 2 + grp) * p.M + row] = ss;
   } else if (EPI == UEPI_QKV) {
     const int Tn = p.T, b = live ? row / Tn : 0, pos = *p.pos_base + (live ? row % Tn : 0);
 #pragma unroll 1
-    for (int hh = 0; hh < BN / 128; ++hh) {
+    for (int hh = grp; hh < BN / 128; hh += 2) {   // a 256-wide tile holds two heads, one per warp group
       const int n = n_tile * BN + hh * 128, kind = n / p.d, hcol = n % p.d;
       const uint32_t tcol = tbase + hh * 128;
       __nv_bfloat16 *dst;
@@ -335,10 +338,10 @@ __device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t
 }
 
 // ---- epilogue of the decode regime: accumulator rows (tokens) already transposed into outs[16][BN+1] ----
-// ew = epilogue warp 0..3, lane; one warp per token, lanes across the tile's columns.
+// ew = epilogue warp 0..7, lane; one warp per token, lanes across the tile's columns.
 template <int BN, int EPI>
 __device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const float *outs, int ew, int lane, int n_tile, int ks, int l, int ls) {
-  for (int tok = ew; tok < p.M; tok += 4) {
+  for (int tok = ew; tok < p.M; tok += 8) {
     const float *y = outs + tok * (BN + 1);
     float rstd = 1.f;
     if ((EPI == UEPI_QKV || EPI == UEPI_RELU2_BF16 || EPI == UEPI_LMHEAD) && p.ssq != nullptr) {
@@ -373,7 +376,10 @@ __device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const f
         ss = fmaf(u, u, ss);
       }
       ss = warp_sum(ss);
-      if (lane == 0) p.ssq_out[((size_t)l * p.Nt + n_tile) * p.M + tok] = ss;
+      if (lane == 0) {  // two partials per tile, as in the prefill regime (the second is zero here)
+        p.ssq_out[(((size_t)l * p.Nt + n_tile) * 2) * p.M + tok] = ss;
+        p.ssq_out[(((size_t)l * p.Nt + n_tile) * 2 + 1) * p.M + tok] = 0.f;
+      }
     } else if (EPI == UEPI_QKV) {
       const int b = tok / p.T, pos = *p.pos_base + (tok % p.T);
 #pragma unroll 1
@@ -420,7 +426,7 @@ __device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const f
   }
 }
 
-// grid = min(items, #SMs), 192 threads, dynamic shared memory UmmaCfg<BN, AM>::kSmem.
+// grid = min(items, #SMs), 320 threads, dynamic shared memory UmmaCfg<BN, AM>::kSmem.
 // tmA: 3-D map over A {K, M, nl}, box {64, AM, 1}; tmB: 3-D map over the stacked weights {K, N, L}, box {64, BN, 1};
 // both bf16, 128-byte swizzle, rows outside the tensor read as zero.
 template <int BN, int AM, int EPI>
@@ -530,7 +536,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
       }
     }
   } else {
-    const int et = threadIdx.x - 64, ew = et >> 5;
+    const int et = threadIdx.x - 64, ew = et >> 5, grp = ew >> 2;   // two warp groups share the columns
     const int quarter = warp & 3;  // tensor-memory lanes this warp may read: 32*quarter .. +31
     for (int i = 0; i < my_items; ++i) {
       SNLP_DECODE_ITEM(i)
@@ -539,14 +545,14 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
       tc_fence_after();
       const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * BN;
       if (AM == kUmmaBM) {
-        umma_epilogue_rows<BN, EPI>(p, tbase, m_tile * kUmmaBM + quarter * 32 + lane, n_tile, ks, l, la);
+        umma_epilogue_rows<BN, EPI>(p, tbase, m_tile * kUmmaBM + quarter * 32 + lane, n_tile, ks, l, la, grp);
         tc_fence_before();
         epi_bar_sync();
         if (et == 0) mbar_arrive(&accempty[b]);
       } else {
-        if (quarter == 0) {  // the token rows live in lanes 0..15
+        if (quarter == 0) {  // the token rows live in lanes 0..15; each group's quarter-0 warp moves half the columns
 #pragma unroll 1
-          for (int c = 0; c < BN / 32; ++c) {
+          for (int c = grp * (BN / 64); c < (grp + 1) * (BN / 64); ++c) {
             uint32_t r[32];
             tmem_ld32(tbase + c * 32, r);
             if (lane < 16) {
