@@ -14,15 +14,6 @@ constexpr int kFaRows = 64;   // query rows per CTA
 constexpr int kFaKeys = 64;   // keys per tile
 constexpr int kFaSmem = (kFaRows + 4 * kFaKeys) * 128 * 2;  // Q + 2 x (K, V) tiles
 
-__device__ __forceinline__ void cp_async16(void *smem, const void *gmem, bool valid) {
-  const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
-  const int sz = valid ? 16 : 0;  // src-size 0 => the 16 bytes are zero-filled
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(s), "l"(gmem), "r"(sz) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], const void *p) {
   const uint32_t s = (uint32_t)__cvta_generic_to_shared(p);
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(s));

@@ -22,7 +22,7 @@ struct CorrParams {
   __nv_bfloat16 *xb; // nullable: [L+1][M][d] bf16 copy of the next sweep's attention-branch input (h_l, or pa_l . x_l);
                      //           slot L = the LM-head input (sum of the streams of the last state)
   float *ssq_x;      //           [L+1][d/128][M] its row sums of squares, one partial per 128 columns
-  float *partial;    // [gridDim.x][nl][2] scratch for the norms (nullable => no norms)
+  float *partial;    // [nl][2][gridDim.x] scratch for the norms (nullable => no norms); k_correct_small: [blocks][nl][2]
   float *resnorm;    // [L][2] (entries l0 .. l0+nl-1 written)
   unsigned *counter; // zero on entry, left zero on exit
 };
@@ -35,10 +35,21 @@ __device__ __forceinline__ float4 f4_fma(float s, float4 a, float4 b) {
 __device__ __forceinline__ float4 f4_scale(float s, float4 a) { return make_float4(s * a.x, s * a.y, s * a.z, s * a.w); }
 __device__ __forceinline__ float f4_sq(float4 a) { return a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w; }
 
+// Depth of the operand ring of k_correct (steps in flight per thread) and its shared-memory size.
+__host__ __device__ constexpr int corr_depth(int ns) { return ns <= 1 ? 4 : (ns <= 4 ? 3 : 2); }
+__host__ __device__ constexpr size_t corr_ring_bytes(int ns, int threads) { return (size_t)corr_depth(ns) * (2 + ns) * threads * sizeof(float4); }
+
 // NS = number of residual streams (compile time so the per-thread state stays in registers).
+// The kernel is bound by HBM bandwidth and each thread's loop over the layers is a chain of dependent steps, so the
+// operands of the next corr_depth(NS)-1 steps are kept in flight with cp.async into a per-thread ring in shared memory
+// (a thread only ever reads its own slots, so no block barrier is involved).  With K-split branch outputs (a_splits or
+// m_splits > 1) the operands are summed from global memory directly, one step ahead.
+// Dynamic shared memory: corr_ring_bytes(NS, blockDim.x) + [warps][nl][2] floats.
 template <int NS>
 __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
-  extern __shared__ float s_norm[];  // [warps][nl][2]
+  extern __shared__ float4 s_ring[];  // [depth][2 + NS][blockDim.x]
+  constexpr int D = corr_depth(NS);
+  float *s_norm = reinterpret_cast<float *>(s_ring + (size_t)D * (2 + NS) * blockDim.x);  // [warps][nl][2]
   const int d4 = p.d >> 2;
   const size_t total = (size_t)p.M * d4;
   const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -55,9 +66,10 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
   const bool native = (NS == 1) ? (p.mode != 2) : (p.mode == 1);  // direct form == the block itself
   const bool want_norm = p.partial != nullptr;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  const bool ring = p.a_splits == 1 && p.m_splits == 1;
 
   float4 oldp[NS], newp[NS];
-  // operands of one step: branch outputs and the old next state; fetched one step ahead of their use
+  // operands of one step: branch outputs and the old next state
   float4 av_n, mv_n, oldn_n[NS];
   auto fetch = [&](int i, float4 &av, float4 &mv, float4 (&on)[NS]) {
     const int l = p.l0 + i * p.lstep, ln = l + p.lstep;
@@ -68,21 +80,46 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
 #pragma unroll
     for (int r = 0; r < NS; ++r) on[r] = tr4[(size_t)ln * state4 + st_off + (size_t)r * d4];
   };
+  auto slot = [&](int i, int k) { return s_ring + ((size_t)(i % D) * (2 + NS) + k) * blockDim.x + threadIdx.x; };
+  auto issue = [&](int i) {  // start the copies of step i's operands into ring slot i % D
+    if (active && i < p.nl) {
+      const int l = p.l0 + i * p.lstep, ln = l + p.lstep;
+      cp_async16(slot(i, 0), a4 + (size_t)l * Md4 + bm_off, true);
+      cp_async16(slot(i, 1), m4 + (size_t)l * Md4 + bm_off, true);
+#pragma unroll
+      for (int r = 0; r < NS; ++r) cp_async16(slot(i, 2 + r), tr4 + (size_t)ln * state4 + st_off + (size_t)r * d4, true);
+    }
+    cp_async_commit();  // one group per step, empty or not, so the wait below can count groups
+  };
   if (active) {
 #pragma unroll
     for (int s = 0; s < NS; ++s) oldp[s] = newp[s] = tr4[(size_t)p.l0 * state4 + st_off + (size_t)s * d4];
-    if (p.nl > 0) fetch(0, av_n, mv_n, oldn_n);
+    if (!ring && p.nl > 0) fetch(0, av_n, mv_n, oldn_n);
+  }
+  if (ring) {
+#pragma unroll
+    for (int i = 0; i < D - 1; ++i) issue(i);
   }
   for (int i = 0; i < p.nl; ++i) {
     const int l = p.l0 + i * p.lstep, ln = l + p.lstep;  // this step maps state l to state ln
     float rs = 0.f, hs = 0.f, xs = 0.f;
+    if (ring) {
+      issue(i + D - 1);       // its slot was read in the previous iteration
+      cp_async_wait<D - 1>();  // step i's group has landed
+      if (active) {
+        av_n = *slot(i, 0);
+        mv_n = *slot(i, 1);
+#pragma unroll
+        for (int r = 0; r < NS; ++r) oldn_n[r] = *slot(i, 2 + r);
+      }
+    }
     if (active) {
       const float4 av = av_n, mv = mv_n;
       const HcCoef &c = p.coef[l];
       float4 oldn[NS], newn[NS], tilde[NS];
 #pragma unroll
       for (int r = 0; r < NS; ++r) oldn[r] = oldn_n[r];
-      if (i + 1 < p.nl) fetch(i + 1, av_n, mv_n, oldn_n);  // the next step's loads overlap this step's arithmetic and stores
+      if (!ring && i + 1 < p.nl) fetch(i + 1, av_n, mv_n, oldn_n);  // the next step's loads overlap this step's arithmetic and stores
 #pragma unroll
       for (int r = 0; r < NS; ++r) {
         if (NS == 1) {
@@ -157,7 +194,7 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
   for (int i = threadIdx.x; i < p.nl * 2; i += blockDim.x) {
     float s = 0.f;
     for (int w = 0; w < nwarp; ++w) s += s_norm[w * p.nl * 2 + i];
-    p.partial[(size_t)blockIdx.x * p.nl * 2 + i] = s;
+    p.partial[(size_t)i * gridDim.x + blockIdx.x] = s;  // [nl * 2][blocks]
   }
   __threadfence();
   __syncthreads();
@@ -166,10 +203,14 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
   __syncthreads();
   if (!last) return;
   __threadfence();
-  for (int i = threadIdx.x; i < p.nl * 2; i += blockDim.x) {
+  // The last block adds the per-block partials in a fixed order: one warp per output, its lanes striding over the
+  // blocks, then a butterfly.  (One thread per output walking all blocks kept a single SM busy for tens of
+  // microseconds after every other block had left.)
+  for (int i = warp; i < p.nl * 2; i += nwarp) {
     double s = 0.0;
-    for (unsigned b = 0; b < gridDim.x; ++b) s += (double)__ldcg(&p.partial[(size_t)b * p.nl * 2 + i]);
-    p.resnorm[(size_t)(p.l0 + (i >> 1) * p.lstep) * 2 + (i & 1)] = (float)s;
+    for (unsigned b = lane; b < gridDim.x; b += 32) s += (double)__ldcg(&p.partial[(size_t)i * gridDim.x + b]);
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) p.resnorm[(size_t)(p.l0 + (i >> 1) * p.lstep) * 2 + (i & 1)] = (float)s;
   }
   if (threadIdx.x == 0) *p.counter = 0u;
 }

@@ -82,7 +82,8 @@ struct snlp_model {
   // weights
   void *embed = nullptr, *lm_head = nullptr, *wqkv = nullptr, *wo = nullptr, *wup = nullptr, *wdn = nullptr;
   HcCoef *coef = nullptr;
-  float2 *rope = nullptr;
+  float2 *rope = nullptr;    // [max_ctx][hd/2] (cos, sin)
+  float2 *rope_t = nullptr;  // the same table transposed, [hd/2][max_ctx]: coalesced when the lanes of a warp hold consecutive positions
   // workspace (R = max_rows)
   float *trace = nullptr, *xa = nullptr, *xm = nullptr, *qkv_raw = nullptr, *a = nullptr, *y_raw = nullptr, *mb = nullptr;
   void *ub = nullptr;
@@ -235,6 +236,7 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
   A(&m->wdn, L * d * ff * es);
   A(&m->coef, L * sizeof(HcCoef));
   A(&m->rope, (size_t)c.max_ctx * (c.head_dim / 2) * sizeof(float2));
+  A(&m->rope_t, (size_t)c.max_ctx * (c.head_dim / 2) * sizeof(float2));
   A(&m->trace, (L + 1) * R * n * d * 4);
   if (n > 1) {
     A(&m->xa, L * R * d * 4);
@@ -285,7 +287,11 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
         const double ang = (double)pos * std::pow((double)c.rope_base, -2.0 * i / c.head_dim);
         tab[(size_t)pos * half + i] = make_float2((float)std::cos(ang), (float)std::sin(ang));
       }
-    if (cudaMemcpy(m->rope, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice) != cudaSuccess)
+    std::vector<float2> tab_t(tab.size());
+    for (int pos = 0; pos < c.max_ctx; ++pos)
+      for (int i = 0; i < half; ++i) tab_t[(size_t)i * c.max_ctx + pos] = tab[(size_t)pos * half + i];
+    if (cudaMemcpy(m->rope, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(m->rope_t, tab_t.data(), tab_t.size() * sizeof(float2), cudaMemcpyHostToDevice) != cudaSuccess)
       rc = fail(SNLP_ERR_CUDA, "rotary table upload failed");
   }
   if (rc == SNLP_OK) rc = init_kernel_attributes();
@@ -478,7 +484,8 @@ static int correct(snlp_model *m, const Fwd &f, int l0, int nsteps, int lstep, i
   const size_t total = (size_t)f.M * (c.d_model / 4);
   const int threads = 256;
   const unsigned blocks = (unsigned)((total + threads - 1) / threads);
-  const size_t sm = resnorm ? (size_t)(threads / 32) * nl * 2 * sizeof(float) : 0;
+  const size_t sm = corr_ring_bytes(c.n_streams, threads) + (resnorm ? (size_t)(threads / 32) * nl * 2 * sizeof(float) : 0);
+  if (sm > corr_ring_bytes(c.n_streams, threads) + 16384) return fail(SNLP_ERR_UNSUPPORTED, "correction: more than 256 layers in one range");
   const size_t sm_small = (size_t)nl * 32 * (2 + c.n_streams) * sizeof(float4) + (size_t)nl * 2 * sizeof(float);
   if (f.M <= kDecodeRows && c.n_streams <= 4 && sm_small <= kCorrSmallSmem) {
     dim3 grid((c.d_model / 4 + 31) / 32, f.M);
@@ -624,7 +631,7 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
     UmmaParams p{};
     p.ssq = m->ssq_x + (size_t)l0 * P * M; p.nparts = P; p.eps = c.rms_eps;
     p.q = q; p.q_ls = Md; p.kc = kc; p.vc = vc; p.kv_ls = f.kv_ls; p.kv_bs = f.kv_bs;
-    p.T = f.T; p.d = d; p.pos_base = f.pos; p.rope = m->rope; p.qk_eps = c.rms_eps;
+    p.T = f.T; p.d = d; p.pos_base = f.pos; p.rope = m->rope; p.rope_t = m->rope_t; p.rope_ld = c.max_ctx; p.qk_eps = c.rms_eps;
     p.a_share = fuse;
     TRY(umma_gemm<UEPI_QKV>(m, st, KC_QKV, xb, Md, m->w_qkv, l0, p, M, 3 * d, d, 1, nl));
   }
@@ -687,6 +694,9 @@ static int init_kernel_attributes() {
   CU((umma_attr<128, 16, UEPI_LMHEAD>()));
   CU((umma_attr<256, 16, UEPI_LMHEAD>()));
   CU(cudaFuncSetAttribute(k_attn_prefill, cudaFuncAttributeMaxDynamicSharedMemorySize, kFaSmem));
+#define ATTR(NS) CU(cudaFuncSetAttribute(k_correct<NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(corr_ring_bytes(NS, 256) + 16384)));
+  ATTR(1) ATTR(2) ATTR(3) ATTR(4) ATTR(5) ATTR(6) ATTR(7) ATTR(8)
+#undef ATTR
   CU(cudaFuncSetAttribute(k_correct_small<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
   CU(cudaFuncSetAttribute(k_correct_small<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
   CU(cudaFuncSetAttribute(k_correct_small<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));

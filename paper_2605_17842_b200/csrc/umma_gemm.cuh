@@ -52,6 +52,7 @@ struct UmmaParams {
   __nv_bfloat16 *q; size_t q_ls;             // UEPI_QKV
   __nv_bfloat16 *kc, *vc; size_t kv_ls, kv_bs;
   int T, d; const int *pos_base; const float2 *rope; float qk_eps;
+  const float2 *rope_t; int rope_ld;  // rope transposed [hd/2][rope_ld], read by the prefill-regime epilogue (thread = row)
   const float *xm; size_t xm_ls; const HcCoef *coef; float *ssq_out;   // UEPI_RESID; ssq_out [nl][Nt][M]
   float *logits; float *pm_val; int *pm_idx;                            // UEPI_LMHEAD
 };
@@ -60,7 +61,7 @@ constexpr int kUmmaThreads = 320;   // warp 0: TMA, warp 1: MMA + TMEM allocatio
 constexpr int kUmmaEpiThreads = 256;
 constexpr int kUmmaBM = 128;
 constexpr int kUmmaBK = 64;         // 64 bf16 = one 128-byte swizzle row
-constexpr int kUmmaSmemBudget = 222 * 1024;
+constexpr int kUmmaSmemBudget = 227 * 1024;  // the most one CTA may take
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -189,7 +190,8 @@ template <int BN, int AM>
 struct UmmaCfg {
   static constexpr int kABytes = AM * kUmmaBK * 2;
   static constexpr int kBBytes = BN * kUmmaBK * 2;
-  static constexpr int kOuts = AM == 16 ? 16 * (BN + 1) * 4 : 0;   // transposed accumulator of the decode regime
+  // decode regime: the transposed accumulator outs[16][BN+1]; prefill regime: one 32 x 32 fp32 staging tile per epilogue warp
+  static constexpr int kOuts = AM == 16 ? 16 * (BN + 1) * 4 : 8 * 4096;
   static constexpr int kFixed = kOuts + 1024 /*alignment slack*/ + 512 /*barriers*/;
   static constexpr int kStagesMax = (kUmmaSmemBudget - kFixed) / (kABytes + kBBytes);
   static constexpr int kStages = kStagesMax > 10 ? 10 : kStagesMax;
@@ -199,7 +201,8 @@ struct UmmaCfg {
 // ---- epilogue of the prefill regime: thread = accumulator row ----------------------------------------
 // grp = 0/1: which half of the tile's columns (or which head of a 256-wide QKV tile) this warp owns.
 template <int BN, int EPI>
-__device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t tbase, int row, int n_tile, int ks, int l, int ls, int grp) {
+__device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t tbase, int row, int n_tile, int ks, int l, int ls, int grp,
+                                                   float4 *stg) {
   const bool live = row < p.M;
   float rstd = 1.f;
   if ((EPI == UEPI_QKV || EPI == UEPI_RELU2_BF16) && p.ssq != nullptr && live) {
@@ -238,37 +241,65 @@ __device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t
       }
     }
   } else if (EPI == UEPI_RESID) {
+    // Ten bytes move per accumulator element here (x read, a and u written), so the accesses must be whole lines:
+    // each 32 x 32 chunk goes through the warp's staging tile (float4 slots XOR-swizzled by row, conflict-free
+    // both ways) and is then handled with 8 lanes per row, 4 rows per instruction.
     const float kappa = p.coef[l].kappa;
-    float ss = 0.f;
+    const int lane = threadIdx.x & 31, row0 = row - lane, rsub = lane >> 3, c4 = lane & 7;
+    float ss[8];
+#pragma unroll
+    for (int it = 0; it < 8; ++it) ss[it] = 0.f;
+    // The residual-stream values of a chunk are fetched before anything of it is stored, and one chunk ahead:
+    // interleaved with the stores they would be issued one at a time (the compiler must assume that a store may
+    // alias the next load), which leaves the epilogue waiting on eight DRAM latencies per chunk.
+    float4 xv[8], xn[8];
+    auto load_x = [&](int c, float4 (&dst)[8]) {
+      const size_t col = (size_t)n_tile * BN + c * 32 + c4 * 4;
+#pragma unroll
+      for (int it = 0; it < 8; ++it) {
+        const int grow = row0 + it * 4 + rsub;
+        dst[it] = grow < p.M ? __ldg(reinterpret_cast<const float4 *>(p.xm + (size_t)l * p.xm_ls + (size_t)grow * p.N + col))
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    };
+    load_x(grp * kHalf, xn);
 #pragma unroll 1
     for (int c = grp * kHalf; c < (grp + 1) * kHalf; ++c) {
+#pragma unroll
+      for (int it = 0; it < 8; ++it) xv[it] = xn[it];
+      if (c + 1 < (grp + 1) * kHalf) load_x(c + 1, xn);
       uint32_t r[32];
       tmem_ld32(tbase + c * 32, r);
-      if (live) {
-        const size_t col = (size_t)n_tile * BN + c * 32;
-        const size_t off = (size_t)l * p.out_ls + (size_t)row * p.N + col;
-        const float4 *xs = reinterpret_cast<const float4 *>(p.xm + (size_t)l * p.xm_ls + (size_t)row * p.N + col);
-        float4 *adst = reinterpret_cast<float4 *>(p.c + off);
-        uint4 *udst = reinterpret_cast<uint4 *>(p.z + off);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          uint32_t w[4];
+      for (int j = 0; j < 8; ++j)
+        stg[lane * 8 + (j ^ (lane & 7))] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                                                       __uint_as_float(r[4 * j + 3]));
+      __syncwarp();
+      const size_t col = (size_t)n_tile * BN + c * 32 + c4 * 4;
 #pragma unroll
-          for (int q = 0; q < 2; ++q) {
-            const float4 x = xs[2 * j + q];
-            const float a0 = __uint_as_float(r[8 * j + 4 * q]), a1 = __uint_as_float(r[8 * j + 4 * q + 1]);
-            const float a2 = __uint_as_float(r[8 * j + 4 * q + 2]), a3 = __uint_as_float(r[8 * j + 4 * q + 3]);
-            adst[2 * j + q] = make_float4(a0, a1, a2, a3);
-            const float u0 = fmaf(kappa, a0, x.x), u1 = fmaf(kappa, a1, x.y), u2 = fmaf(kappa, a2, x.z), u3 = fmaf(kappa, a3, x.w);
-            ss += u0 * u0 + u1 * u1 + u2 * u2 + u3 * u3;
-            w[2 * q] = pack_bf16x2(u0, u1);
-            w[2 * q + 1] = pack_bf16x2(u2, u3);
-          }
-          udst[j] = make_uint4(w[0], w[1], w[2], w[3]);
+      for (int it = 0; it < 8; ++it) {
+        const int rr = it * 4 + rsub, grow = row0 + rr;
+        if (grow < p.M) {
+          const float4 a = stg[rr * 8 + (c4 ^ (rr & 7))];
+          const size_t off = (size_t)l * p.out_ls + (size_t)grow * p.N + col;
+          const float4 x = xv[it];
+          *reinterpret_cast<float4 *>(p.c + off) = a;
+          const float u0 = fmaf(kappa, a.x, x.x), u1 = fmaf(kappa, a.y, x.y), u2 = fmaf(kappa, a.z, x.z), u3 = fmaf(kappa, a.w, x.w);
+          ss[it] += u0 * u0 + u1 * u1 + u2 * u2 + u3 * u3;
+          *reinterpret_cast<uint2 *>(p.z + off) = make_uint2(pack_bf16x2(u0, u1), pack_bf16x2(u2, u3));
         }
       }
+      __syncwarp();
     }
-    if (live) p.ssq_out[(((size_t)l * p.Nt + n_tile) * 2 + grp) * p.M + row] = ss;
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {  // the 8 lanes of a row hold its partial sums
+      float v = ss[it];
+      v += __shfl_xor_sync(0xffffffffu, v, 1);
+      v += __shfl_xor_sync(0xffffffffu, v, 2);
+      v += __shfl_xor_sync(0xffffffffu, v, 4);
+      const int grow = row0 + it * 4 + rsub;
+      if (c4 == 0 && grow < p.M) p.ssq_out[(((size_t)l * p.Nt + n_tile) * 2 + grp) * p.M + grow] = v;
+    }
   } else if (EPI == UEPI_QKV) {
     const int Tn = p.T, b = live ? row / Tn : 0, pos = *p.pos_base + (live ? row % Tn : 0);
 #pragma unroll 1
@@ -307,7 +338,8 @@ __device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t
           }
         }
         const float rn = rsqrtf(ss * (1.f / 128.f) + p.qk_eps) * rstd;
-        const float2 *cs = p.rope + (size_t)pos * 64;
+        const float2 *cs = p.rope_t + pos;  // lanes hold consecutive positions: every table read is one coalesced line
+        const size_t cld = (size_t)p.rope_ld;
 #pragma unroll 1
         for (int c = 0; c < 2; ++c) {
           uint32_t lo[32], hi[32];
@@ -321,7 +353,7 @@ __device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t
 #pragma unroll
               for (int q = 0; q < 4; ++q) {
                 const int i0 = 8 * j + 2 * q;
-                const float2 ca = cs[c * 32 + i0], cb = cs[c * 32 + i0 + 1];
+                const float2 ca = __ldg(cs + (c * 32 + i0) * cld), cb = __ldg(cs + (c * 32 + i0 + 1) * cld);
                 const float xa1 = __uint_as_float(lo[i0]) * rn, xa2 = __uint_as_float(hi[i0]) * rn;
                 const float xb1 = __uint_as_float(lo[i0 + 1]) * rn, xb2 = __uint_as_float(hi[i0 + 1]) * rn;
                 w1[q] = pack_bf16x2(xa1 * ca.x - xa2 * ca.y, xb1 * cb.x - xb2 * cb.y);
@@ -545,7 +577,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
       tc_fence_after();
       const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * BN;
       if (AM == kUmmaBM) {
-        umma_epilogue_rows<BN, EPI>(p, tbase, m_tile * kUmmaBM + quarter * 32 + lane, n_tile, ks, l, la, grp);
+        umma_epilogue_rows<BN, EPI>(p, tbase, m_tile * kUmmaBM + quarter * 32 + lane, n_tile, ks, l, la, grp,
+                                    reinterpret_cast<float4 *>(outs) + ew * 256);
         tc_fence_before();
         epi_bar_sync();
         if (et == 0) mbar_arrive(&accempty[b]);
