@@ -17,7 +17,7 @@
 #include "decode.cuh"
 #include "generic.cuh"
 #include "umma_gemm.cuh"
-#include "attn_prefill.cuh"
+#include "attn_umma.cuh"
 
 using namespace snlp;
 
@@ -129,6 +129,7 @@ struct Fwd {
   size_t kv_ls, kv_bs;  // elements
   const int *pos;       // device: first position of this call
   int pos_hi;           // host copy of *pos
+  int kv_rows;          // rows per sequence in the key / value store
   cudaStream_t st;
 };
 
@@ -641,8 +642,18 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
     KLAUNCH(m, st, KC_ATTN, k_attn_decode<<<dim3(nchunk, f.B * H, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, m->attn_part, m->attn_counters, att, Md,
                                                                             f.T, H, f.pos, csub));
   } else {
-    KLAUNCH(m, st, KC_ATTN, k_attn_prefill<<<dim3((f.T + kFaRows - 1) / kFaRows, f.B * H, nl), 128, kFaSmem, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, att, Md,
-                                                                                                    f.T, H, f.pos));
+    // tensor-core attention: 128-query items over the (layer, sequence, head, query tile) grid, persistent CTAs
+    CUtensorMap tq, tk, tv, to;
+    if (!make_tmap_bf16(m->encode_tiled, &tq, q, d, M, nl, Md, kFuTile) ||
+        !make_tmap_kv(m->encode_tiled, &tk, kc, d, f.kv_rows, f.B, nl, f.kv_bs, f.kv_ls) ||
+        !make_tmap_kv(m->encode_tiled, &tv, vc, d, f.kv_rows, f.B, nl, f.kv_bs, f.kv_ls) ||
+        !make_tmap_kv(m->encode_tiled, &to, att, d, f.T, f.B, nl, (size_t)f.T * d, Md))
+      return fail(SNLP_ERR_CUDA, "cuTensorMapEncodeTiled failed for the attention operands");
+    FaUmmaParams ap{};
+    ap.T = f.T; ap.H = H; ap.BH = f.B * H; ap.nq = (f.T + kFuTile - 1) / kFuTile;
+    ap.n_items = ap.nq * ap.BH * nl; ap.pos_base = f.pos; ap.err = m->dev_err;
+    const int grid = ap.n_items < m->n_sm ? ap.n_items : m->n_sm;
+    KLAUNCH(m, st, KC_ATTN, k_attn_umma<<<grid, kFuThreads, kFuSmem, st>>>(tq, tk, tv, to, ap, nl));
   }
   {
     UmmaParams p{};
@@ -693,7 +704,7 @@ static int init_kernel_attributes() {
   CU(umma_attr_all<UEPI_RESID>());
   CU((umma_attr<128, 16, UEPI_LMHEAD>()));
   CU((umma_attr<256, 16, UEPI_LMHEAD>()));
-  CU(cudaFuncSetAttribute(k_attn_prefill, cudaFuncAttributeMaxDynamicSharedMemorySize, kFaSmem));
+  CU(cudaFuncSetAttribute(k_attn_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, kFuSmem));
 #define ATTR(NS) CU(cudaFuncSetAttribute(k_correct<NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(corr_ring_bytes(NS, 256) + 16384)));
   ATTR(1) ATTR(2) ATTR(3) ATTR(4) ATTR(5) ATTR(6) ATTR(7) ATTR(8)
 #undef ATTR
@@ -884,6 +895,7 @@ static Fwd scratch_fwd(snlp_model *m, int B, int T, cudaStream_t st) {
   f.kc = m->sk; f.vc = m->sv;
   f.kv_bs = (size_t)T * m->cfg.d_model;
   f.kv_ls = (size_t)B * f.kv_bs;
+  f.kv_rows = T;
   f.pos = m->zero; f.pos_hi = 0; f.st = st;
   return f;
 }
@@ -1006,6 +1018,7 @@ static Fwd kv_fwd(snlp_model *m, snlp_kv *kv, int T, cudaStream_t st) {
   f.kc = kv->k; f.vc = kv->v;
   f.kv_bs = (size_t)kv->max_ctx * m->cfg.d_model;
   f.kv_ls = (size_t)kv->B * f.kv_bs;
+  f.kv_rows = kv->max_ctx;
   f.pos = kv->pos; f.pos_hi = kv->len; f.st = st;
   return f;
 }
