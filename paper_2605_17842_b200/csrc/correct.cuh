@@ -67,6 +67,7 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
   const bool want_norm = p.partial != nullptr;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
   const bool ring = p.a_splits == 1 && p.m_splits == 1;
+  const bool need_old = want_norm || !native;   // the old next state enters only the residual norm and the surrogate forms
 
   float4 oldp[NS], newp[NS];
   // operands of one step: branch outputs and the old next state
@@ -78,7 +79,7 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
     mv = m4[(size_t)l * Md4 + bm_off];
     for (int q = 1; q < p.m_splits; ++q) mv = f4_add(mv, m4[(size_t)q * (p.m_ss >> 2) + (size_t)l * Md4 + bm_off]);
 #pragma unroll
-    for (int r = 0; r < NS; ++r) on[r] = tr4[(size_t)ln * state4 + st_off + (size_t)r * d4];
+    for (int r = 0; r < NS; ++r) on[r] = need_old ? tr4[(size_t)ln * state4 + st_off + (size_t)r * d4] : make_float4(0.f, 0.f, 0.f, 0.f);
   };
   auto slot = [&](int i, int k) { return s_ring + ((size_t)(i % D) * (2 + NS) + k) * blockDim.x + threadIdx.x; };
   auto issue = [&](int i) {  // start the copies of step i's operands into ring slot i % D
@@ -86,8 +87,10 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
       const int l = p.l0 + i * p.lstep, ln = l + p.lstep;
       cp_async16(slot(i, 0), a4 + (size_t)l * Md4 + bm_off, true);
       cp_async16(slot(i, 1), m4 + (size_t)l * Md4 + bm_off, true);
+      if (need_old) {
 #pragma unroll
-      for (int r = 0; r < NS; ++r) cp_async16(slot(i, 2 + r), tr4 + (size_t)ln * state4 + st_off + (size_t)r * d4, true);
+        for (int r = 0; r < NS; ++r) cp_async16(slot(i, 2 + r), tr4 + (size_t)ln * state4 + st_off + (size_t)r * d4, true);
+      }
     }
     cp_async_commit();  // one group per step, empty or not, so the wait below can count groups
   };
@@ -110,7 +113,7 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
         av_n = *slot(i, 0);
         mv_n = *slot(i, 1);
 #pragma unroll
-        for (int r = 0; r < NS; ++r) oldn_n[r] = *slot(i, 2 + r);
+        for (int r = 0; r < NS; ++r) oldn_n[r] = need_old ? *slot(i, 2 + r) : make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
     if (active) {
@@ -243,6 +246,45 @@ __global__ void k_prep_rows(const float *__restrict__ trace, int l0, int M, int 
   reinterpret_cast<uint2 *>(xb)[(size_t)l * Md4 + row * d4 + c4] = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
   const float ss = warp_sum(f4_sq(v));
   if ((threadIdx.x & 31) == 0) ssq_x[((size_t)l * (d4 >> 5) + (c4 >> 5)) * M + row] = ss;
+}
+
+// Alg. 2 line 5 fused with the first branch inputs: every state l0+1 .. L starts as a copy of state l0, and layers
+// l0 .. L-1 get their bf16 attention-branch input, its sums of squares and (mHC) the fp32 MLP pre-map, all from one read
+// of the row.  Same values as k_bcast_trace followed by k_prep_rows.  grid (M), d/4 threads (d a multiple of 128).
+template <int NS>
+__global__ void k_init_rows(float *__restrict__ trace, int l0, int L, int M, int d, const HcCoef *__restrict__ coef,
+                            __nv_bfloat16 *__restrict__ xb, float *__restrict__ ssq_x, float *__restrict__ xm) {
+  const int d4 = d >> 2, c4 = threadIdx.x;
+  const size_t row = blockIdx.x, Md4 = (size_t)M * d4;
+  float4 *tr4 = reinterpret_cast<float4 *>(trace);
+  float4 x[NS];
+#pragma unroll
+  for (int s = 0; s < NS; ++s) x[s] = tr4[(size_t)l0 * Md4 * NS + row * NS * d4 + (size_t)s * d4 + c4];
+  float4 v = x[0];
+  uint2 pk = make_uint2(0, 0);
+  float ss = 0.f;
+  for (int l = l0; l < L; ++l) {
+#pragma unroll
+    for (int s = 0; s < NS; ++s) tr4[(size_t)(l + 1) * Md4 * NS + row * NS * d4 + (size_t)s * d4 + c4] = x[s];
+    if (NS > 1) {
+      const HcCoef &c = coef[l];
+      float4 sa = f4_scale(c.pa[0], x[0]), sm = f4_scale(c.pmra[0], x[0]);
+#pragma unroll
+      for (int s = 1; s < NS; ++s) {
+        sa = f4_fma(c.pa[s], x[s], sa);
+        sm = f4_fma(c.pmra[s], x[s], sm);
+      }
+      reinterpret_cast<float4 *>(xm)[(size_t)l * Md4 + row * d4 + c4] = sm;
+      v = sa;
+    }
+    if (NS > 1 || l == l0) {   // single stream: the same input for every layer
+      __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+      pk = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+      ss = warp_sum(f4_sq(v));
+    }
+    reinterpret_cast<uint2 *>(xb)[(size_t)l * Md4 + row * d4 + c4] = pk;
+    if ((threadIdx.x & 31) == 0) ssq_x[((size_t)l * (d4 >> 5) + (c4 >> 5)) * M + row] = ss;
+  }
 }
 
 // LM-head input from arbitrary hidden-state rows: xb = bf16(sum of the NS streams), per-128-column sums of squares.

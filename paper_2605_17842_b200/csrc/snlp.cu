@@ -781,11 +781,18 @@ static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *res
     return SNLP_OK;
   }
   // Alg. 2 line 5: every suffix state starts at h_S
-  const size_t n4 = (size_t)f.M * c.n_streams * c.d_model / 4;
-  KLAUNCH(m, f.st, KC_OTHER, k_bcast_trace<<<(unsigned)((n4 + 255) / 256), 256, 0, f.st>>>(reinterpret_cast<const float4 *>(m->trace) + (size_t)S * n4,
-                                                               reinterpret_cast<float4 *>(m->trace) + (size_t)(S + 1) * n4, n4, L - S));
-  if (umma_path_ok(m)) TRY(prep_rows(m, f, S, L - S));
-  else TRY(premix(m, f, S, L - S));
+  if (umma_path_ok(m)) {
+    switch (c.n_streams) {   // one kernel: the copies and the layers' first branch inputs
+#define CASE(NS) case NS: KLAUNCH(m, f.st, KC_OTHER, k_init_rows<NS><<<f.M, c.d_model / 4, 0, f.st>>>(m->trace, S, L, f.M, c.d_model, m->coef, (__nv_bfloat16 *)m->xn, m->ssq_x, m->xm)); break;
+      CASE(1) CASE(2) CASE(3) CASE(4) CASE(5) CASE(6) CASE(7) CASE(8)
+#undef CASE
+    }
+  } else {
+    const size_t n4 = (size_t)f.M * c.n_streams * c.d_model / 4;
+    KLAUNCH(m, f.st, KC_OTHER, k_bcast_trace<<<(unsigned)((n4 + 255) / 256), 256, 0, f.st>>>(reinterpret_cast<const float4 *>(m->trace) + (size_t)S * n4,
+                                                                 reinterpret_cast<float4 *>(m->trace) + (size_t)(S + 1) * n4, n4, L - S));
+    TRY(premix(m, f, S, L - S));
+  }
   int exact = S;  // states 0..exact equal the sequential trace (of the fused model when F > 1)
   if (sol.init == SNLP_INIT_FWD) {
     // one batched evaluation of every suffix chunk on h_S; with A = 0 the correction just stores F(h_S)
