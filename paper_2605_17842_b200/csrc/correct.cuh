@@ -18,7 +18,7 @@ struct CorrParams {
   int M, d;
   int mode;          // SNLP_MODE_*
   const HcCoef *coef;
-  float *xa, *xm;    // [L][M][d] pre-mapped inputs for the next sweep (n > 1 only)
+  float *xa, *xm;    // [L][M][d] pre-mapped inputs for the next sweep (n > 1 only); xa nullable (not needed where xb is read)
   __nv_bfloat16 *xb; // nullable: [L+1][M][d] bf16 copy of the next sweep's attention-branch input (h_l, or pa_l . x_l);
                      //           slot L = the LM-head input (sum of the streams of the last state)
   float *ssq_x;      //           [L+1][d/128][M] its row sums of squares, one partial per 128 columns
@@ -46,7 +46,7 @@ __host__ __device__ constexpr size_t corr_ring_bytes(int ns, int threads) { retu
 // m_splits > 1) the operands are summed from global memory directly, one step ahead.
 // Dynamic shared memory: corr_ring_bytes(NS, blockDim.x) + [warps][nl][2] floats.
 template <int NS>
-__global__ void __launch_bounds__(256) k_correct(CorrParams p) {
+__global__ void __launch_bounds__(256, 2) k_correct(CorrParams p) {
   extern __shared__ float4 s_ring[];  // [depth][2 + NS][blockDim.x]
   constexpr int D = corr_depth(NS);
   float *s_norm = reinterpret_cast<float *>(s_ring + (size_t)D * (2 + NS) * blockDim.x);  // [warps][nl][2]
@@ -118,7 +118,19 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
     }
     if (active) {
       const float4 av = av_n, mv = mv_n;
-      const HcCoef &c = p.coef[l];
+      // this layer's coefficients into registers once (read through the non-coherent path: a reference into global
+      // memory would have to be re-read after every store of the step, which may alias it for all the compiler knows)
+      const HcCoef *cp = p.coef + l;
+      float cA[NS * NS], cca[NS], ccm[NS];
+      if (NS > 1) {
+#pragma unroll
+        for (int r = 0; r < NS; ++r) {
+#pragma unroll
+          for (int s = 0; s < NS; ++s) cA[r * NS + s] = __ldg(&cp->A[r * NS + s]);
+          cca[r] = __ldg(&cp->ca[r]);
+          ccm[r] = __ldg(&cp->cm[r]);
+        }
+      }
       float4 oldn[NS], newn[NS], tilde[NS];
 #pragma unroll
       for (int r = 0; r < NS; ++r) oldn[r] = oldn_n[r];
@@ -128,10 +140,10 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
         if (NS == 1) {
           tilde[r] = f4_add(f4_add(oldp[0], av), mv);  // F_l(h_l^k) = (h + a) + m
         } else {
-          float4 t = f4_scale(c.A[r * NS], oldp[0]);
+          float4 t = f4_scale(cA[r * NS], oldp[0]);
 #pragma unroll
-          for (int s = 1; s < NS; ++s) t = f4_fma(c.A[r * NS + s], oldp[s], t);
-          tilde[r] = f4_fma(c.cm[r], mv, f4_fma(c.ca[r], av, t));
+          for (int s = 1; s < NS; ++s) t = f4_fma(cA[r * NS + s], oldp[s], t);
+          tilde[r] = f4_fma(ccm[r], mv, f4_fma(cca[r], av, t));
         }
       }
 #pragma unroll
@@ -142,10 +154,10 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
           if (NS == 1) {
             newn[r] = f4_add(f4_add(newp[0], av), mv);               // prefix sum over depth
           } else {
-            float4 t = f4_scale(c.A[r * NS], newp[0]);
+            float4 t = f4_scale(cA[r * NS], newp[0]);
 #pragma unroll
-            for (int s = 1; s < NS; ++s) t = f4_fma(c.A[r * NS + s], newp[s], t);
-            newn[r] = f4_fma(c.cm[r], mv, f4_fma(c.ca[r], av, t));   // affine scan with A_l
+            for (int s = 1; s < NS; ++s) t = f4_fma(cA[r * NS + s], newp[s], t);
+            newn[r] = f4_fma(ccm[r], mv, f4_fma(cca[r], av, t));   // affine scan with A_l
           }
         } else {
           newn[r] = f4_add(tilde[r], f4_sub(newp[r], oldp[r]));      // identity surrogate on n streams
@@ -157,14 +169,14 @@ __global__ void __launch_bounds__(256) k_correct(CorrParams p) {
       }
       float4 nxt = newn[0];  // the next layer's attention-branch input
       if (NS > 1 && ln < p.L) {
-        const HcCoef &cn = p.coef[ln];
-        float4 sa = f4_scale(cn.pa[0], newn[0]), sm = f4_scale(cn.pmra[0], newn[0]);
+        const HcCoef *cn = p.coef + ln;
+        float4 sa = f4_scale(__ldg(&cn->pa[0]), newn[0]), sm = f4_scale(__ldg(&cn->pmra[0]), newn[0]);
 #pragma unroll
         for (int s = 1; s < NS; ++s) {
-          sa = f4_fma(cn.pa[s], newn[s], sa);
-          sm = f4_fma(cn.pmra[s], newn[s], sm);
+          sa = f4_fma(__ldg(&cn->pa[s]), newn[s], sa);
+          sm = f4_fma(__ldg(&cn->pmra[s]), newn[s], sm);
         }
-        reinterpret_cast<float4 *>(p.xa)[(size_t)ln * Md4 + bm_off] = sa;
+        if (p.xa != nullptr) reinterpret_cast<float4 *>(p.xa)[(size_t)ln * Md4 + bm_off] = sa;
         reinterpret_cast<float4 *>(p.xm)[(size_t)ln * Md4 + bm_off] = sm;
         nxt = sa;
       }
@@ -394,7 +406,7 @@ __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
           xa = f4_fma(cn.pa[s], newn[s], xa);
           xm = f4_fma(cn.pmra[s], newn[s], xm);
         }
-        reinterpret_cast<float4 *>(p.xa)[(size_t)ln * Md4 + bm_off] = xa;
+        if (p.xa != nullptr) reinterpret_cast<float4 *>(p.xa)[(size_t)ln * Md4 + bm_off] = xa;
         reinterpret_cast<float4 *>(p.xm)[(size_t)ln * Md4 + bm_off] = xm;
         nxt = xa;
       }

@@ -475,7 +475,7 @@ static int correct(snlp_model *m, const Fwd &f, int l0, int nsteps, int lstep, i
   p.d = c.d_model;
   p.mode = mode;
   p.coef = m->coef;
-  p.xa = m->xa;
+  p.xa = umma_path_ok(m) ? nullptr : m->xa;   // the tensor-core path reads the bf16 copy xb instead
   p.xm = m->xm;
   p.xb = umma_path_ok(m) ? (__nv_bfloat16 *)m->xn : nullptr;
   p.ssq_x = m->ssq_x;
