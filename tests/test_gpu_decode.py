@@ -104,26 +104,29 @@ def test_decode_with_K_equal_L_equals_sequential_decode_on_gpu(cfg):
     assert torch.equal(outs[0], outs[1])
 
 
-@pytest.mark.parametrize("cfg", [F32, BF16])
-def test_step_by_step_decode_agrees_with_chunked_prefill(cfg):
+@pytest.mark.parametrize("cfg,B,Tp,chunk", [(F32, 2, 20, 6), (BF16, 2, 20, 6), (BF16, 1, 300, 160)])
+def test_step_by_step_decode_agrees_with_chunked_prefill(cfg, B, Tp, chunk):
     """Prefill of T tokens in one call, in chunks (max_rows smaller than B*T), and token by token all
-    leave a cache from which the next greedy token is the same."""
+    leave a cache from which the next greedy token is the same.  The last case runs the prefill-regime kernels with a
+    second chunk that starts at position 160: its causal mask crosses key tiles and its queries see cached keys."""
     W = weights(cfg)
-    B, Tp = 2, 20
+    ctx = Tp + 12
     ids_np = synth.make_ids(cfg, B, Tp, seed=6)
     ids = dev(ids_np)
-    big = make_model(cfg, W, max_rows=B * Tp, max_batch=B, max_ctx=32)
-    kv = big.kv_cache(B, 32)
+    big = make_model(cfg, W, max_rows=B * Tp, max_batch=B, max_ctx=ctx)
+    kv = big.kv_cache(B, ctx)
     t_one = big.prefill(kv, ids).cpu().numpy()
-    small = make_model(cfg, W, max_rows=B * 6, max_batch=B, max_ctx=32)   # 4 chunks: 6, 6, 6, 2
-    kv2 = small.kv_cache(B, 32)
+    small = make_model(cfg, W, max_rows=B * chunk, max_batch=B, max_ctx=ctx)   # e.g. 4 chunks: 6, 6, 6, 2
+    kv2 = small.kv_cache(B, ctx)
     t_chunk = small.prefill(kv2, ids).cpu().numpy()
     assert len(kv2) == Tp
-    kv3 = big.kv_cache(B, 32)
+    kv3 = big.kv_cache(B, ctx)
     for s in range(Tp):
         t_step = big.decode_step(kv3, dev(ids_np[:, s].copy()), 0)
+    small.device_status()
+    big.device_status()
     # the oracle's token (fp64) settles fp32; in bf16 the three library paths may differ only at near-ties
-    kv_o = oracle_kv(cfg, B, 32)
+    kv_o = oracle_kv(cfg, B, ctx)
     logits = O.prefill(cfg, W, ids_np, kv_o)
     tau = margin_tau(cfg, W) if cfg.dtype == "bf16" else 0.0
     for got in (t_one, t_chunk, t_step.cpu().numpy()):
