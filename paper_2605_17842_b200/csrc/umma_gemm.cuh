@@ -587,6 +587,16 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
     for (int i = 0; i < my_items; ++i) {
       SNLP_DECODE_ITEM(i)
       const int b = i & 1;
+      if (EPI == UEPI_RESID && AM == kUmmaBM) {
+        // While the tile's products are still being accumulated, pull the residual-stream lines this warp will add
+        // into L2 (one 128-byte line per row and 32-column chunk), so the epilogue's reads do not wait on DRAM.
+        const int prow = m_tile * kUmmaBM + quarter * 32 + lane;
+        if (prow < p.M) {
+          const float *px = p.xm + (size_t)l * p.xm_ls + (size_t)prow * p.N + (size_t)n_tile * BN + grp * (BN / 2);
+#pragma unroll
+          for (int c = 0; c < BN / 64; ++c) asm volatile("prefetch.global.L2 [%0];" ::"l"(px + c * 32));
+        }
+      }
       if (!epi_all(mbar_wait(&accfull[b], (i >> 1) & 1, abort_flag, p.err))) break;
       tc_fence_after();
       const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * BN;
