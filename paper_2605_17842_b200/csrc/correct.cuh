@@ -45,7 +45,8 @@ __host__ __device__ constexpr size_t corr_ring_bytes(int ns, int threads) { retu
 // (a thread only ever reads its own slots, so no block barrier is involved).  With K-split branch outputs (a_splits or
 // m_splits > 1) the operands are summed from global memory directly, one step ahead.
 // Dynamic shared memory: corr_ring_bytes(NS, blockDim.x) + [warps][nl][2] floats.
-template <int NS>
+// NATIVE: the surrogate is the block's own affine map (IDN on a single stream, HCN on n streams), known at compile time.
+template <int NS, bool NATIVE>
 __global__ void __launch_bounds__(256, 2) k_correct(CorrParams p) {
   extern __shared__ float4 s_ring[];  // [depth][2 + NS][blockDim.x]
   constexpr int D = corr_depth(NS);
@@ -63,7 +64,7 @@ __global__ void __launch_bounds__(256, 2) k_correct(CorrParams p) {
   float4 *tr4 = reinterpret_cast<float4 *>(p.trace);
   const size_t bm_off = row * d4 + c4;             // offset inside an [M][d] plane
   const size_t st_off = row * NS * d4 + c4;        // offset of stream 0 inside a state
-  const bool native = (NS == 1) ? (p.mode != 2) : (p.mode == 1);  // direct form == the block itself
+  const bool native = NATIVE;  // direct form == the block itself
   const bool want_norm = p.partial != nullptr;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
   const bool ring = p.a_splits == 1 && p.m_splits == 1;
@@ -148,9 +149,9 @@ __global__ void __launch_bounds__(256, 2) k_correct(CorrParams p) {
       }
 #pragma unroll
       for (int r = 0; r < NS; ++r) {
-        if (p.mode == 2) {
+        if (!NATIVE && p.mode == 2) {
           newn[r] = tilde[r];                                        // A = 0
-        } else if (native) {
+        } else if (NATIVE) {
           if (NS == 1) {
             newn[r] = f4_add(f4_add(newp[0], av), mv);               // prefix sum over depth
           } else {

@@ -498,8 +498,9 @@ static int correct(snlp_model *m, const Fwd &f, int l0, int nsteps, int lstep, i
     }
   } else {
     TimedLaunch tl_(m, f.st, KC_CORRECT);
+    const bool native = c.n_streams == 1 ? mode != SNLP_MODE_NOCORR : mode == SNLP_MODE_HCN;
     switch (c.n_streams) {
-#define CASE(NS) case NS: k_correct<NS><<<blocks, threads, sm, f.st>>>(p); break;
+#define CASE(NS) case NS: if (native) k_correct<NS, true><<<blocks, threads, sm, f.st>>>(p); else k_correct<NS, false><<<blocks, threads, sm, f.st>>>(p); break;
       CASE(1) CASE(2) CASE(3) CASE(4) CASE(5) CASE(6) CASE(7) CASE(8)
 #undef CASE
     }
@@ -705,7 +706,8 @@ static int init_kernel_attributes() {
   CU((umma_attr<128, 16, UEPI_LMHEAD>()));
   CU((umma_attr<256, 16, UEPI_LMHEAD>()));
   CU(cudaFuncSetAttribute(k_attn_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, kFuSmem));
-#define ATTR(NS) CU(cudaFuncSetAttribute(k_correct<NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(corr_ring_bytes(NS, 256) + 16384)));
+#define ATTR(NS) CU(cudaFuncSetAttribute(k_correct<NS, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(corr_ring_bytes(NS, 256) + 16384))); \
+  CU(cudaFuncSetAttribute(k_correct<NS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(corr_ring_bytes(NS, 256) + 16384)));
   ATTR(1) ATTR(2) ATTR(3) ATTR(4) ATTR(5) ATTR(6) ATTR(7) ATTR(8)
 #undef ATTR
   CU(cudaFuncSetAttribute(k_correct_small<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
