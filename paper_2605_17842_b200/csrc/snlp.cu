@@ -17,6 +17,7 @@
 #include "decode.cuh"
 #include "generic.cuh"
 #include "umma_gemm.cuh"
+#include "umma_gemm2.cuh"
 #include "attn_umma.cuh"
 
 using namespace snlp;
@@ -70,7 +71,7 @@ struct GraphKey {
 };
 struct GraphEntry { cudaGraphExec_t exec; int64_t nodes; };
 struct PendingTime { int cls; cudaEvent_t e0, e1; };
-struct WMap { CUtensorMap tm; int BN; };  // TMA map over one stacked weight array, box {64, BN, 1}
+struct WMap { CUtensorMap tm, tm_half; int BN; };  // TMA maps over one stacked weight array, boxes {64, BN, 1} and (for CTA pairs) {64, 128, 1}
 enum { KC_QKV = 0, KC_ATTN, KC_OPROJ, KC_UP, KC_DOWN, KC_CORRECT, KC_LMHEAD, KC_OTHER, KC_COUNT };
 static_assert(KC_COUNT == SNLP_NUM_KERNEL_CLASSES, "kernel class count");
 
@@ -382,7 +383,8 @@ extern "C" int snlp_load_weights(snlp_model *m, const snlp_weights *w) {
   if (m->encode_tiled && c.dtype == SNLP_DTYPE_BF16 && d % 128 == 0 && ff % 128 == 0 && V % 128 == 0) {
     auto mk = [&](WMap &w, const void *base, uint64_t K, uint64_t N, uint64_t layers) {
       w.BN = N % 256 == 0 ? 256 : 128;
-      return make_tmap_bf16(m->encode_tiled, &w.tm, base, K, N, layers, N * K, w.BN);
+      return make_tmap_bf16(m->encode_tiled, &w.tm, base, K, N, layers, N * K, w.BN) &&
+             make_tmap_bf16(m->encode_tiled, &w.tm_half, base, K, N, layers, N * K, 128);
     };
     m->have_wmaps = mk(m->w_qkv, m->wqkv, d, 3 * d, L) && mk(m->w_o, m->wo, d, d, L) && mk(m->w_up, m->wup, d, ff, L) &&
                     mk(m->w_dn, m->wdn, ff, d, L) && mk(m->w_lm, m->lm_head, d, V, 1);
@@ -573,6 +575,7 @@ static cudaError_t umma_attr_all() {
   if (e == cudaSuccess) e = umma_attr<256, 128, EPI>();
   if (e == cudaSuccess) e = umma_attr<128, 16, EPI>();
   if (e == cudaSuccess) e = umma_attr<256, 16, EPI>();
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_umma_gemm2<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kU2Smem);
   return e;
 }
 
@@ -591,6 +594,14 @@ static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat1
   if (p.kfuse < 1) p.kfuse = 1;
   p.M = M; p.N = N; p.K = K; p.ksplit = ksplit; p.kslice = K / ksplit;
   p.Mt = small ? 1 : (M + kUmmaBM - 1) / kUmmaBM; p.Nt = N / w.BN; p.nl = nl; p.l0 = l0; p.err = m->dev_err;
+  if (!small && w.BN == 256 && M > kUmmaBM && EPI != UEPI_LMHEAD) {
+    // prefill regime with more than one row tile: 256 x 256 tiles on CTA pairs (same results, less operand traffic per SM)
+    p.Mt = (M + 2 * kUmmaBM - 1) / (2 * kUmmaBM);
+    p.nstages = kU2Stages;
+    const int items2 = p.Mt * p.Nt * ksplit * nl, pairs = items2 < m->n_sm / 2 ? items2 : m->n_sm / 2;
+    KLAUNCH(m, st, cls, k_umma_gemm2<EPI><<<2 * pairs, kUmmaThreads, kU2Smem, st>>>(ta, w.tm_half, p));
+    return SNLP_OK;
+  }
   const int items = p.Mt * p.Nt * ksplit * nl;
   const int grid = items < m->n_sm ? items : m->n_sm;
 #define SNLP_UMMA_LAUNCH(BN_, AM_)                                                                                                   \
