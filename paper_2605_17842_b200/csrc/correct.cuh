@@ -47,7 +47,7 @@ __host__ __device__ constexpr size_t corr_ring_bytes(int ns, int threads) { retu
 // Dynamic shared memory: corr_ring_bytes(NS, blockDim.x) + [warps][nl][2] floats.
 // NATIVE: the surrogate is the block's own affine map (IDN on a single stream, HCN on n streams), known at compile time.
 template <int NS, bool NATIVE>
-__global__ void __launch_bounds__(256, 2) k_correct(CorrParams p) {
+__global__ void __launch_bounds__(256, NS == 1 ? 4 : 2) k_correct(CorrParams p) {
   extern __shared__ float4 s_ring[];  // [depth][2 + NS][blockDim.x]
   constexpr int D = corr_depth(NS);
   float *s_norm = reinterpret_cast<float *>(s_ring + (size_t)D * (2 + NS) * blockDim.x);  // [warps][nl][2]

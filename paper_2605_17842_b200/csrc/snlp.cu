@@ -265,7 +265,8 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
   A(&m->xlm, R * d * es);
   const size_t nchunk_max = ((size_t)c.max_ctx + kAttnSub - 1) / kAttnSub;
   A(&m->attn_part, L * (size_t)kDecodeRows * c.n_head * nchunk_max * kAttnPartStride * 4);
-  const size_t corr_blocks = (R * (d / 4) + 255) / 256;
+  // partial norms: one slot per block of k_correct (256 threads over R x d/4) or of k_correct_small ((d/128) x rows, rows <= 16)
+  const size_t corr_blocks = std::max<size_t>((R * (d / 4) + 255) / 256, (size_t)((d + 127) / 128) * kDecodeRows);
   A(&m->corr_part, corr_blocks * L * 2 * 4);
   m->logit_rows = (int)(R < 64 ? R : 64);
   A(&m->logits, (size_t)m->logit_rows * V * 4);
