@@ -438,6 +438,15 @@ def run_prefill_workload(args, name):
             if k in flops:
                 classes[k]["TFLOPs"] = flops[k] / (ms / nrep * 1e-3) / 1e12
                 classes[k]["frac_of_bf16_peak"] = classes[k]["TFLOPs"] / burst
+    # the correction is HBM-bound: new states written, a and m read, bf16 inputs (and the mHC MLP pre-map) written; the
+    # sweep timed here is the first one after initialisation, which does not read old states (they all equal h_0); later
+    # sweeps read them too (n * 4 more bytes per element)
+    n = cfg.n_streams
+    corr_bytes = L * M * d * (n * 4 + 2 * 4 + 2 + (4 if n > 1 else 0))
+    if "correction" in classes:
+        hbm = peaks()[0]
+        classes["correction"]["alg_GBs"] = corr_bytes / (classes["correction"]["ms_per_sweep"] * 1e-3) / 1e9
+        classes["correction"]["frac_of_hbm_peak"] = classes["correction"]["alg_GBs"] / hbm
     dom = max(("qkv", "out_proj", "mlp_up", "mlp_down"), key=lambda k: kt[k][0])
     sweep_ms = sum(v["ms_per_sweep"] for v in classes.values())
     line = {"metric": f"{name} forward ms (sequential and SNLP K sweeps)", "value": out[f"K{Ks[0]}_ms"], "unit": "ms",
@@ -445,7 +454,7 @@ def run_prefill_workload(args, name):
             "config": {"workload": f"{name}: L{L} d{d} ff{ff} n_streams {cfg.n_streams}, B{B} x T{T}, mode {'HCN' if mode else 'IDN'}"},
             "forward_ms": out, "speedup_vs_own_sequential": {k: out["sequential_ms"] / v for k, v in out.items() if k != "sequential_ms"},
             "sweep_ms_sum_of_kernels": sweep_ms, "kernels": classes,
-            "roofline": {"bound": "tensor", "kernel": f"k_umma_gemm ({dom})", "achieved": classes[dom]["TFLOPs"], "peak": burst,
+            "roofline": {"bound": "tensor", "kernel": f"k_umma_gemm2 ({dom}; 256x256 tiles on CTA pairs)", "achieved": classes[dom]["TFLOPs"], "peak": burst,
                          "unit": "TFLOP/s", "frac": classes[dom]["TFLOPs"] / burst, "peak_source": src + " burst", "traffic": None},
             "gemm_flops_per_sweep": sum(flops[k] for k in ("qkv", "out_proj", "mlp_up", "mlp_down")), "attention_flops_per_sweep": flops["attention"]}
     print(json.dumps(line))

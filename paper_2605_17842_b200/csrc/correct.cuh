@@ -17,6 +17,7 @@ struct CorrParams {
   int lstep;         // layers per step: 1, or the number of fused layers of a chunk (states l0, l0+lstep, ...)
   int M, d;
   int mode;          // SNLP_MODE_*
+  int implicit_old;  // 1: the states after l0 have not been materialised yet and all equal state l0 (first pass after Alg. 2 line 5)
   const HcCoef *coef;
   float *xa, *xm;    // [L][M][d] pre-mapped inputs for the next sweep (n > 1 only); xa nullable (not needed where xb is read)
   __nv_bfloat16 *xb; // nullable: [L+1][M][d] bf16 copy of the next sweep's attention-branch input (h_l, or pa_l . x_l);
@@ -68,7 +69,7 @@ __global__ void __launch_bounds__(256, NS == 1 ? 4 : 2) k_correct(CorrParams p) 
   const bool want_norm = p.partial != nullptr;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
   const bool ring = p.a_splits == 1 && p.m_splits == 1;
-  const bool need_old = want_norm || !native;   // the old next state enters only the residual norm and the surrogate forms
+  const bool need_old = (want_norm || !native) && !p.implicit_old;   // the old next state enters only the residual norm and the surrogate forms
 
   float4 oldp[NS], newp[NS];
   // operands of one step: branch outputs and the old next state
@@ -134,7 +135,7 @@ __global__ void __launch_bounds__(256, NS == 1 ? 4 : 2) k_correct(CorrParams p) 
       }
       float4 oldn[NS], newn[NS], tilde[NS];
 #pragma unroll
-      for (int r = 0; r < NS; ++r) oldn[r] = oldn_n[r];
+      for (int r = 0; r < NS; ++r) oldn[r] = p.implicit_old ? oldp[r] : oldn_n[r];   // implicit: every old state is the first one
       if (!ring && i + 1 < p.nl) fetch(i + 1, av_n, mv_n, oldn_n);  // the next step's loads overlap this step's arithmetic and stores
 #pragma unroll
       for (int r = 0; r < NS; ++r) {
@@ -264,9 +265,10 @@ __global__ void k_prep_rows(const float *__restrict__ trace, int l0, int M, int 
 // Alg. 2 line 5 fused with the first branch inputs: every state l0+1 .. L starts as a copy of state l0, and layers
 // l0 .. L-1 get their bf16 attention-branch input, its sums of squares and (mHC) the fp32 MLP pre-map, all from one read
 // of the row.  Same values as k_bcast_trace followed by k_prep_rows.  grid (M), d/4 threads (d a multiple of 128).
+// write_trace == 0 leaves the copies out: the first pass then reads state l0 wherever it needs a later state.
 template <int NS>
 __global__ void k_init_rows(float *__restrict__ trace, int l0, int L, int M, int d, const HcCoef *__restrict__ coef,
-                            __nv_bfloat16 *__restrict__ xb, float *__restrict__ ssq_x, float *__restrict__ xm) {
+                            __nv_bfloat16 *__restrict__ xb, float *__restrict__ ssq_x, float *__restrict__ xm, int write_trace) {
   const int d4 = d >> 2, c4 = threadIdx.x;
   const size_t row = blockIdx.x, Md4 = (size_t)M * d4;
   float4 *tr4 = reinterpret_cast<float4 *>(trace);
@@ -277,8 +279,10 @@ __global__ void k_init_rows(float *__restrict__ trace, int l0, int L, int M, int
   uint2 pk = make_uint2(0, 0);
   float ss = 0.f;
   for (int l = l0; l < L; ++l) {
+    if (write_trace) {
 #pragma unroll
-    for (int s = 0; s < NS; ++s) tr4[(size_t)(l + 1) * Md4 * NS + row * NS * d4 + (size_t)s * d4 + c4] = x[s];
+      for (int s = 0; s < NS; ++s) tr4[(size_t)(l + 1) * Md4 * NS + row * NS * d4 + (size_t)s * d4 + c4] = x[s];
+    }
     if (NS > 1) {
       const HcCoef &c = coef[l];
       float4 sa = f4_scale(c.pa[0], x[0]), sm = f4_scale(c.pmra[0], x[0]);
@@ -347,7 +351,7 @@ __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
       sa[i * 32 + c] = av;
       sm[i * 32 + c] = mv;
 #pragma unroll
-      for (int r = 0; r < NS; ++r) so[(i * NS + r) * 32 + c] = tr4[(size_t)ln * state4 + st_off + (size_t)r * d4];
+      for (int r = 0; r < NS; ++r) so[(i * NS + r) * 32 + c] = tr4[(size_t)(p.implicit_old ? p.l0 : ln) * state4 + st_off + (size_t)r * d4];
     }
   }
   __syncthreads();

@@ -131,6 +131,7 @@ struct Fwd {
   const int *pos;       // device: first position of this call
   int pos_hi;           // host copy of *pos
   int kv_rows;          // rows per sequence in the key / value store
+  int implicit_state = -1;  // >= 0: states after this one are not materialised yet and equal it (first pass after Alg. 2 line 5)
   cudaStream_t st;
 };
 
@@ -477,6 +478,7 @@ static int correct(snlp_model *m, const Fwd &f, int l0, int nsteps, int lstep, i
   p.M = f.M;
   p.d = c.d_model;
   p.mode = mode;
+  p.implicit_old = f.implicit_state >= 0 ? 1 : 0;
   p.coef = m->coef;
   p.xa = umma_path_ok(m) ? nullptr : m->xa;   // the tensor-core path reads the bf16 copy xb instead
   p.xm = m->xm;
@@ -634,7 +636,10 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
   const bool small = M <= kDecodeRows;
   const size_t Md = (size_t)M * d;
   cudaStream_t st = f.st;
-  const float *xm_src = n == 1 ? m->trace + l0 * Md : m->xm + l0 * Md;
+  // residual stream read by the out-projection epilogue: h_l (single stream; before the first correction every h_l is
+  // still the one materialised state), or the fp32 MLP pre-map (mHC)
+  const bool implicit = n == 1 && f.implicit_state >= 0;
+  const float *xm_src = n == 1 ? m->trace + (implicit ? f.implicit_state : l0) * Md : m->xm + l0 * Md;
   T *xb = (T *)m->xn + l0 * Md, *ub = (T *)m->ub + l0 * Md, *q = (T *)m->q + l0 * Md, *att = (T *)m->att + l0 * Md;
   T *z = (T *)m->z + (size_t)l0 * M * ff;
   float *a = m->a + l0 * Md, *mb = m->mb + l0 * Md;
@@ -671,7 +676,7 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
   {
     UmmaParams p{};
     p.c = a; p.z = ub; p.out_ls = Md;
-    p.xm = xm_src; p.xm_ls = Md; p.coef = m->coef + l0; p.ssq_out = m->ssq_u + (size_t)l0 * Pu * M;
+    p.xm = xm_src; p.xm_ls = implicit ? 0 : Md; p.coef = m->coef + l0; p.ssq_out = m->ssq_u + (size_t)l0 * Pu * M;
     p.kfuse = fuse;   // a chunk's out-projections are one product over the concatenated attention outputs
     TRY(umma_gemm<UEPI_RESID>(m, st, KC_OPROJ, att, Md, m->w_o, l0, p, M, d, d, 1, nl / fuse));
   }
@@ -797,7 +802,7 @@ static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *res
   // Alg. 2 line 5: every suffix state starts at h_S
   if (umma_path_ok(m)) {
     switch (c.n_streams) {   // one kernel: the copies and the layers' first branch inputs
-#define CASE(NS) case NS: KLAUNCH(m, f.st, KC_OTHER, k_init_rows<NS><<<f.M, c.d_model / 4, 0, f.st>>>(m->trace, S, L, f.M, c.d_model, m->coef, (__nv_bfloat16 *)m->xn, m->ssq_x, m->xm)); break;
+#define CASE(NS) case NS: KLAUNCH(m, f.st, KC_OTHER, k_init_rows<NS><<<f.M, c.d_model / 4, 0, f.st>>>(m->trace, S, L, f.M, c.d_model, m->coef, (__nv_bfloat16 *)m->xn, m->ssq_x, m->xm, 0)); break;
       CASE(1) CASE(2) CASE(3) CASE(4) CASE(5) CASE(6) CASE(7) CASE(8)
 #undef CASE
     }
@@ -808,11 +813,22 @@ static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *res
     TRY(premix(m, f, S, L - S));
   }
   int exact = S;  // states 0..exact equal the sequential trace (of the fused model when F > 1)
+  // On the tensor-core path the copies of h_S are not written: the first pass reads h_S itself wherever it needs a later
+  // state, and its correction writes every state for the first time.
+  Fwd first = f;
+  if (umma_path_ok(m)) first.implicit_state = S;
+  bool fresh = true;
+  if (umma_path_ok(m) && sol.K == 0 && sol.init != SNLP_INIT_FWD) {   // nothing will write the states: materialise them after all
+    const size_t n4 = (size_t)f.M * c.n_streams * c.d_model / 4;
+    KLAUNCH(m, f.st, KC_OTHER, k_bcast_trace<<<(unsigned)((n4 + 255) / 256), 256, 0, f.st>>>(reinterpret_cast<const float4 *>(m->trace) + (size_t)S * n4,
+                                                                 reinterpret_cast<float4 *>(m->trace) + (size_t)(S + 1) * n4, n4, L - S));
+  }
   if (sol.init == SNLP_INIT_FWD) {
     // one batched evaluation of every suffix chunk on h_S; with A = 0 the correction just stores F(h_S)
-    TRY(run_blocks(m, f, S, L - S, F));
-    TRY(correct_range(m, f, S, L - S, F, SNLP_MODE_NOCORR, nullptr));
+    TRY(run_blocks(m, first, S, L - S, F));
+    TRY(correct_range(m, first, S, L - S, F, SNLP_MODE_NOCORR, nullptr));
     exact = S + F;
+    fresh = false;
   }
   for (int k = 0; k < sol.K; ++k) {
     // Exactness-aware trimming: entering this sweep the states 0..exact already equal the sequential trace (Newton
@@ -820,8 +836,10 @@ static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *res
     // outputs they wrote in the previous pass.  Only chunks from `exact` on are evaluated; the correction still runs
     // over the whole suffix on the stored branch outputs, so trace, residual norms and next inputs are unchanged.
     const int b0 = exact < L ? exact : L;
-    if (b0 < L) TRY(run_blocks(m, f, b0, L - b0, F));
-    TRY(correct_range(m, f, S, L - S, F, sol.mode, resnorm_out ? resnorm_out + (size_t)k * L * 2 : nullptr));
+    const Fwd &fk = fresh ? first : f;
+    if (b0 < L) TRY(run_blocks(m, fk, b0, L - b0, F));
+    TRY(correct_range(m, fk, S, L - S, F, sol.mode, resnorm_out ? resnorm_out + (size_t)k * L * 2 : nullptr));
+    fresh = false;
     exact += F;
   }
   return SNLP_OK;
