@@ -17,6 +17,7 @@ struct CorrParams {
   int lstep;         // layers per step: 1, or the number of fused layers of a chunk (states l0, l0+lstep, ...)
   int M, d;
   int mode;          // SNLP_MODE_*
+  int skip_next;     // 1: no sweep follows, so the next sweep's branch inputs (xa, xm, xb, ssq_x) are not produced (k_correct only)
   int implicit_old;  // 1: the states after l0 have not been materialised yet and all equal state l0 (first pass after Alg. 2 line 5)
   const HcCoef *coef;
   float *xa, *xm;    // [L][M][d] pre-mapped inputs for the next sweep (n > 1 only); xa nullable (not needed where xb is read)
@@ -170,7 +171,7 @@ __global__ void __launch_bounds__(256, NS == 1 ? 4 : 2) k_correct(CorrParams p) 
         tr4[(size_t)ln * state4 + st_off + (size_t)r * d4] = newn[r];
       }
       float4 nxt = newn[0];  // the next layer's attention-branch input
-      if (NS > 1 && ln < p.L) {
+      if (NS > 1 && ln < p.L && !p.skip_next) {
         const HcCoef *cn = p.coef + ln;
         float4 sa = f4_scale(__ldg(&cn->pa[0]), newn[0]), sm = f4_scale(__ldg(&cn->pmra[0]), newn[0]);
 #pragma unroll
@@ -186,7 +187,7 @@ __global__ void __launch_bounds__(256, NS == 1 ? 4 : 2) k_correct(CorrParams p) 
 #pragma unroll
         for (int s = 1; s < NS; ++s) nxt = f4_add(nxt, newn[s]);
       }
-      if (p.xb != nullptr) {
+      if (p.xb != nullptr && !p.skip_next) {
         __nv_bfloat162 lo = __floats2bfloat162_rn(nxt.x, nxt.y), hi = __floats2bfloat162_rn(nxt.z, nxt.w);
         uint2 pk = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
         reinterpret_cast<uint2 *>(p.xb)[(size_t)ln * Md4 + bm_off] = pk;
@@ -195,7 +196,7 @@ __global__ void __launch_bounds__(256, NS == 1 ? 4 : 2) k_correct(CorrParams p) 
 #pragma unroll
       for (int r = 0; r < NS; ++r) { oldp[r] = oldn[r]; newp[r] = newn[r]; }
     }
-    if (p.xb != nullptr) {
+    if (p.xb != nullptr && !p.skip_next) {
       // d is a multiple of 128 here, so the 32 lanes of a warp hold 128 consecutive columns of one row
       xs = warp_sum(xs);
       if (lane == 0 && active) p.ssq_x[((size_t)ln * (d4 >> 5) + (c4 >> 5)) * p.M + row] = xs;

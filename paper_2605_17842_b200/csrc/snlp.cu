@@ -131,6 +131,7 @@ struct Fwd {
   const int *pos;       // device: first position of this call
   int pos_hi;           // host copy of *pos
   int kv_rows;          // rows per sequence in the key / value store
+  bool last_pass = false;   // no sweep follows this correction: it need not prepare the next sweep's branch inputs
   int implicit_state = -1;  // >= 0: states after this one are not materialised yet and equal it (first pass after Alg. 2 line 5)
   cudaStream_t st;
 };
@@ -479,6 +480,7 @@ static int correct(snlp_model *m, const Fwd &f, int l0, int nsteps, int lstep, i
   p.d = c.d_model;
   p.mode = mode;
   p.implicit_old = f.implicit_state >= 0 ? 1 : 0;
+  p.skip_next = f.last_pass && f.M > kDecodeRows ? 1 : 0;   // the decode regime's LM head reads slot L of xb
   p.coef = m->coef;
   p.xa = umma_path_ok(m) ? nullptr : m->xa;   // the tensor-core path reads the bf16 copy xb instead
   p.xm = m->xm;
@@ -836,7 +838,8 @@ static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *res
     // outputs they wrote in the previous pass.  Only chunks from `exact` on are evaluated; the correction still runs
     // over the whole suffix on the stored branch outputs, so trace, residual norms and next inputs are unchanged.
     const int b0 = exact < L ? exact : L;
-    const Fwd &fk = fresh ? first : f;
+    Fwd fk = fresh ? first : f;
+    fk.last_pass = k == sol.K - 1;
     if (b0 < L) TRY(run_blocks(m, fk, b0, L - b0, F));
     TRY(correct_range(m, fk, S, L - S, F, sol.mode, resnorm_out ? resnorm_out + (size_t)k * L * 2 : nullptr));
     fresh = false;
