@@ -323,9 +323,11 @@ __global__ void k_prep_lm(const float *__restrict__ h, size_t row_stride, int ns
 // Latency-oriented variant for the decode regime (a handful of rows): the per-thread loop over
 // layers above serialises ~7 dependent-latency loads per layer, which dominates when there are too
 // few threads to hide it.  Here a block owns 32 float4 columns of one row; its 8 warps first fetch
-// every layer's branch outputs and old states in parallel into shared memory, then warp 0 runs the
-// serial recurrence out of shared memory.  Same arithmetic, same summation order as k_correct.
-// grid (d/128, M), 256 threads; dynamic shared memory nl*32*(2+NS) float4 + nl*2 floats.
+// every layer's branch outputs and old states into shared memory (four layers per warp at a time, all loads
+// issued before the first is consumed), then warp 0 runs the serial recurrence out of shared memory, keeping the
+// per-layer sums of squares per lane; afterwards all warps reduce those, so the serial loop carries no shuffles.
+// Same arithmetic, same summation order as k_correct.
+// grid (d/128, M), 256 threads; dynamic shared memory nl*32*(2+NS) float4 + nl*2 floats + nl*3*32 floats.
 template <int NS>
 __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
   extern __shared__ float4 s_buf[];
@@ -340,107 +342,134 @@ __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
   float4 *tr4 = reinterpret_cast<float4 *>(p.trace);
   const size_t bm_off = row * d4 + c4, st_off = row * NS * d4 + c4;
   float4 *sa = s_buf, *sm = s_buf + (size_t)p.nl * 32, *so = s_buf + (size_t)p.nl * 64;  // so: [nl][NS][32]
-  float *snorm = reinterpret_cast<float *>(s_buf + (size_t)p.nl * 32 * (2 + NS));
+  float *snorm = reinterpret_cast<float *>(s_buf + (size_t)p.nl * 32 * (2 + NS));          // [nl][2]
+  float *sred = snorm + (size_t)p.nl * 2;                                                  // [nl][3][32]: per-lane xs, rs, hs
   const bool want_norm = p.partial != nullptr;
   if (active) {
-    for (int i = ll; i < p.nl; i += 8) {
-      const int l = p.l0 + i * p.lstep, ln = l + p.lstep;  // this step maps state l to state ln
-      float4 av = a4[(size_t)l * Md4 + bm_off];
-      for (int q = 1; q < p.a_splits; ++q) av = f4_add(av, a4[(size_t)q * (p.a_ss >> 2) + (size_t)l * Md4 + bm_off]);
-      float4 mv = m4[(size_t)l * Md4 + bm_off];
-      for (int q = 1; q < p.m_splits; ++q) mv = f4_add(mv, m4[(size_t)q * (p.m_ss >> 2) + (size_t)l * Md4 + bm_off]);
-      sa[i * 32 + c] = av;
-      sm[i * 32 + c] = mv;
+#pragma unroll 1
+    for (int i0 = ll; i0 < p.nl; i0 += 32) {
+      float4 av[4], mv[4], ov[4][NS];
 #pragma unroll
-      for (int r = 0; r < NS; ++r) so[(i * NS + r) * 32 + c] = tr4[(size_t)(p.implicit_old ? p.l0 : ln) * state4 + st_off + (size_t)r * d4];
+      for (int k = 0; k < 4; ++k) {
+        const int i = i0 + 8 * k;
+        if (i < p.nl) {
+          const int l = p.l0 + i * p.lstep, ln = l + p.lstep;  // this step maps state l to state ln
+          av[k] = a4[(size_t)l * Md4 + bm_off];
+          mv[k] = m4[(size_t)l * Md4 + bm_off];
+#pragma unroll
+          for (int r = 0; r < NS; ++r) ov[k][r] = tr4[(size_t)(p.implicit_old ? p.l0 : ln) * state4 + st_off + (size_t)r * d4];
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int i = i0 + 8 * k;
+        if (i < p.nl) {
+          const int l = p.l0 + i * p.lstep;
+          for (int q = 1; q < p.a_splits; ++q) av[k] = f4_add(av[k], a4[(size_t)q * (p.a_ss >> 2) + (size_t)l * Md4 + bm_off]);
+          for (int q = 1; q < p.m_splits; ++q) mv[k] = f4_add(mv[k], m4[(size_t)q * (p.m_ss >> 2) + (size_t)l * Md4 + bm_off]);
+          sa[i * 32 + c] = av[k];
+          sm[i * 32 + c] = mv[k];
+#pragma unroll
+          for (int r = 0; r < NS; ++r) so[(i * NS + r) * 32 + c] = ov[k][r];
+        }
+      }
     }
   }
   __syncthreads();
-  if (ll != 0) return;
-  const bool native = (NS == 1) ? (p.mode != 2) : (p.mode == 1);
-  float4 oldp[NS], newp[NS];
-  if (active) {
-#pragma unroll
-    for (int s = 0; s < NS; ++s) oldp[s] = newp[s] = tr4[(size_t)p.l0 * state4 + st_off + (size_t)s * d4];
-  }
-  for (int i = 0; i < p.nl; ++i) {
-    const int l = p.l0 + i * p.lstep, ln = l + p.lstep;  // this step maps state l to state ln
-    float rs = 0.f, hs = 0.f, xs = 0.f;
+  if (ll == 0) {
+    const bool native = (NS == 1) ? (p.mode != 2) : (p.mode == 1);
+    float4 oldp[NS], newp[NS];
     if (active) {
-      const float4 av = sa[i * 32 + c], mv = sm[i * 32 + c];
-      const HcCoef &cf = p.coef[l];
-      float4 oldn[NS], newn[NS], tilde[NS];
 #pragma unroll
-      for (int r = 0; r < NS; ++r) {
-        oldn[r] = so[(i * NS + r) * 32 + c];
-        if (NS == 1) {
-          tilde[r] = f4_add(f4_add(oldp[0], av), mv);
-        } else {
-          float4 t = f4_scale(cf.A[r * NS], oldp[0]);
-#pragma unroll
-          for (int s = 1; s < NS; ++s) t = f4_fma(cf.A[r * NS + s], oldp[s], t);
-          tilde[r] = f4_fma(cf.cm[r], mv, f4_fma(cf.ca[r], av, t));
-        }
-      }
-#pragma unroll
-      for (int r = 0; r < NS; ++r) {
-        if (p.mode == 2) {
-          newn[r] = tilde[r];
-        } else if (native) {
-          if (NS == 1) {
-            newn[r] = f4_add(f4_add(newp[0], av), mv);
-          } else {
-            float4 t = f4_scale(cf.A[r * NS], newp[0]);
-#pragma unroll
-            for (int s = 1; s < NS; ++s) t = f4_fma(cf.A[r * NS + s], newp[s], t);
-            newn[r] = f4_fma(cf.cm[r], mv, f4_fma(cf.ca[r], av, t));
-          }
-        } else {
-          newn[r] = f4_add(tilde[r], f4_sub(newp[r], oldp[r]));
-        }
-        const float4 rr = f4_sub(tilde[r], oldn[r]);
-        rs += f4_sq(rr);
-        hs += f4_sq(oldn[r]);
-        tr4[(size_t)ln * state4 + st_off + (size_t)r * d4] = newn[r];
-      }
-      float4 nxt = newn[0];
-      if (NS > 1 && ln < p.L) {
-        const HcCoef &cn = p.coef[ln];
-        float4 xa = f4_scale(cn.pa[0], newn[0]), xm = f4_scale(cn.pmra[0], newn[0]);
-#pragma unroll
-        for (int s = 1; s < NS; ++s) {
-          xa = f4_fma(cn.pa[s], newn[s], xa);
-          xm = f4_fma(cn.pmra[s], newn[s], xm);
-        }
-        if (p.xa != nullptr) reinterpret_cast<float4 *>(p.xa)[(size_t)ln * Md4 + bm_off] = xa;
-        reinterpret_cast<float4 *>(p.xm)[(size_t)ln * Md4 + bm_off] = xm;
-        nxt = xa;
-      }
-      if (NS > 1 && ln == p.L) {
-#pragma unroll
-        for (int s = 1; s < NS; ++s) nxt = f4_add(nxt, newn[s]);
-      }
-      if (p.xb != nullptr) {
-        __nv_bfloat162 lo = __floats2bfloat162_rn(nxt.x, nxt.y), hi = __floats2bfloat162_rn(nxt.z, nxt.w);
-        reinterpret_cast<uint2 *>(p.xb)[(size_t)ln * Md4 + bm_off] = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
-        xs = f4_sq(nxt);
-      }
-#pragma unroll
-      for (int r = 0; r < NS; ++r) { oldp[r] = oldn[r]; newp[r] = newn[r]; }
+      for (int s = 0; s < NS; ++s) oldp[s] = newp[s] = tr4[(size_t)p.l0 * state4 + st_off + (size_t)s * d4];
     }
-    if (p.xb != nullptr) {  // this warp holds 128 consecutive columns of the row: partial blockIdx.x
-      xs = warp_sum(xs);
+    for (int i = 0; i < p.nl; ++i) {
+      const int l = p.l0 + i * p.lstep, ln = l + p.lstep;  // this step maps state l to state ln
+      float rs = 0.f, hs = 0.f, xs = 0.f;
+      if (active) {
+        const float4 av = sa[i * 32 + c], mv = sm[i * 32 + c];
+        const HcCoef &cf = p.coef[l];
+        float4 oldn[NS], newn[NS], tilde[NS];
+#pragma unroll
+        for (int r = 0; r < NS; ++r) {
+          oldn[r] = so[(i * NS + r) * 32 + c];
+          if (NS == 1) {
+            tilde[r] = f4_add(f4_add(oldp[0], av), mv);
+          } else {
+            float4 t = f4_scale(cf.A[r * NS], oldp[0]);
+#pragma unroll
+            for (int s = 1; s < NS; ++s) t = f4_fma(cf.A[r * NS + s], oldp[s], t);
+            tilde[r] = f4_fma(cf.cm[r], mv, f4_fma(cf.ca[r], av, t));
+          }
+        }
+#pragma unroll
+        for (int r = 0; r < NS; ++r) {
+          if (p.mode == 2) {
+            newn[r] = tilde[r];
+          } else if (native) {
+            if (NS == 1) {
+              newn[r] = f4_add(f4_add(newp[0], av), mv);
+            } else {
+              float4 t = f4_scale(cf.A[r * NS], newp[0]);
+#pragma unroll
+              for (int s = 1; s < NS; ++s) t = f4_fma(cf.A[r * NS + s], newp[s], t);
+              newn[r] = f4_fma(cf.cm[r], mv, f4_fma(cf.ca[r], av, t));
+            }
+          } else {
+            newn[r] = f4_add(tilde[r], f4_sub(newp[r], oldp[r]));
+          }
+          const float4 rr = f4_sub(tilde[r], oldn[r]);
+          rs += f4_sq(rr);
+          hs += f4_sq(oldn[r]);
+          tr4[(size_t)ln * state4 + st_off + (size_t)r * d4] = newn[r];
+        }
+        float4 nxt = newn[0];
+        if (NS > 1 && ln < p.L) {
+          const HcCoef &cn = p.coef[ln];
+          float4 xa = f4_scale(cn.pa[0], newn[0]), xm = f4_scale(cn.pmra[0], newn[0]);
+#pragma unroll
+          for (int s = 1; s < NS; ++s) {
+            xa = f4_fma(cn.pa[s], newn[s], xa);
+            xm = f4_fma(cn.pmra[s], newn[s], xm);
+          }
+          if (p.xa != nullptr) reinterpret_cast<float4 *>(p.xa)[(size_t)ln * Md4 + bm_off] = xa;
+          reinterpret_cast<float4 *>(p.xm)[(size_t)ln * Md4 + bm_off] = xm;
+          nxt = xa;
+        }
+        if (NS > 1 && ln == p.L) {
+#pragma unroll
+          for (int s = 1; s < NS; ++s) nxt = f4_add(nxt, newn[s]);
+        }
+        if (p.xb != nullptr) {
+          __nv_bfloat162 lo = __floats2bfloat162_rn(nxt.x, nxt.y), hi = __floats2bfloat162_rn(nxt.z, nxt.w);
+          reinterpret_cast<uint2 *>(p.xb)[(size_t)ln * Md4 + bm_off] = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+          xs = f4_sq(nxt);
+        }
+#pragma unroll
+        for (int r = 0; r < NS; ++r) { oldp[r] = oldn[r]; newp[r] = newn[r]; }
+      }
+      sred[(i * 3 + 0) * 32 + c] = xs;
+      sred[(i * 3 + 1) * 32 + c] = rs;
+      sred[(i * 3 + 2) * 32 + c] = hs;
+    }
+  }
+  __syncthreads();
+  // every warp reduces the sums of some steps (this block's 32 lanes hold 128 consecutive columns of the row: partial blockIdx.x)
+  for (int i = ll; i < p.nl; i += 8) {
+    const int ln = p.l0 + (i + 1) * p.lstep;
+    if (p.xb != nullptr) {
+      const float xs = warp_sum(sred[(i * 3 + 0) * 32 + c]);
       if (c == 0) p.ssq_x[((size_t)ln * gridDim.x + blockIdx.x) * p.M + row] = xs;
     }
     if (want_norm) {
-      rs = warp_sum(rs);
-      hs = warp_sum(hs);
+      const float rs = warp_sum(sred[(i * 3 + 1) * 32 + c]), hs = warp_sum(sred[(i * 3 + 2) * 32 + c]);
       if (c == 0) { snorm[i * 2] = rs; snorm[i * 2 + 1] = hs; }
     }
   }
   if (!want_norm) return;
+  __syncthreads();
+  if (ll != 0) return;
   // warp 0 only from here on
-  __syncwarp();
   const unsigned nblk = gridDim.x * gridDim.y, blk = blockIdx.y * gridDim.x + blockIdx.x;
   for (int i = c; i < p.nl * 2; i += 32) p.partial[(size_t)blk * p.nl * 2 + i] = snorm[i];
   __threadfence();

@@ -494,7 +494,7 @@ static int correct(snlp_model *m, const Fwd &f, int l0, int nsteps, int lstep, i
   const unsigned blocks = (unsigned)((total + threads - 1) / threads);
   const size_t sm = corr_ring_bytes(c.n_streams, threads) + (resnorm ? (size_t)(threads / 32) * nl * 2 * sizeof(float) : 0);
   if (sm > corr_ring_bytes(c.n_streams, threads) + 16384) return fail(SNLP_ERR_UNSUPPORTED, "correction: more than 256 layers in one range");
-  const size_t sm_small = (size_t)nl * 32 * (2 + c.n_streams) * sizeof(float4) + (size_t)nl * 2 * sizeof(float);
+  const size_t sm_small = (size_t)nl * 32 * (2 + c.n_streams) * sizeof(float4) + (size_t)nl * 2 * sizeof(float) + (size_t)nl * 3 * 32 * sizeof(float);
   if (f.M <= kDecodeRows && c.n_streams <= 4 && sm_small <= kCorrSmallSmem) {
     dim3 grid((c.d_model / 4 + 31) / 32, f.M);
     TimedLaunch tl_(m, f.st, KC_CORRECT);
