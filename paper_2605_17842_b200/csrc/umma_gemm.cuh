@@ -226,33 +226,36 @@ __device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t
   }
   constexpr int kHalf = BN / 64;  // 32-column chunks per warp group
   if (EPI == UEPI_F32 || EPI == UEPI_RELU2_BF16) {
+    // Each 32 x 32 chunk goes through the warp's staging tile (float4 slots XOR-swizzled by row, conflict-free both
+    // ways) and is stored with 8 lanes per row, 4 rows per instruction: whole 128-byte (fp32) or 64-byte (bf16) runs
+    // instead of 16 bytes per row.
+    const int lane = threadIdx.x & 31, row0 = row - lane, rsub = lane >> 3, c4 = lane & 7;
 #pragma unroll 1
     for (int c = grp * kHalf; c < (grp + 1) * kHalf; ++c) {
       uint32_t r[32];
       tmem_ld32(tbase + c * 32, r);
-      if (live) {
-        const size_t off = (size_t)l * p.out_ls + (size_t)row * p.N + (size_t)n_tile * BN + c * 32;
-        if (EPI == UEPI_F32) {
-          float4 *dst = reinterpret_cast<float4 *>(p.c + (size_t)ks * p.out_ss + off);
 #pragma unroll
-          for (int j = 0; j < 8; ++j)
-            dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
-                                 __uint_as_float(r[4 * j + 3]));
-        } else {
-          uint4 *dst = reinterpret_cast<uint4 *>(p.z + off);
+      for (int j = 0; j < 8; ++j) {
+        float4 v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+        if (EPI == UEPI_RELU2_BF16) {   // the row scale belongs to this thread's row: apply it before the transposition
+          v.x = fmaxf(v.x * rstd, 0.f); v.y = fmaxf(v.y * rstd, 0.f); v.z = fmaxf(v.z * rstd, 0.f); v.w = fmaxf(v.w * rstd, 0.f);
+          v.x *= v.x; v.y *= v.y; v.z *= v.z; v.w *= v.w;
+        }
+        stg[lane * 8 + (j ^ (lane & 7))] = v;
+      }
+      __syncwarp();
+      const size_t col = (size_t)n_tile * BN + c * 32 + c4 * 4;
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            uint32_t w[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const float a = fmaxf(__uint_as_float(r[8 * j + 2 * q]) * rstd, 0.f);
-              const float b = fmaxf(__uint_as_float(r[8 * j + 2 * q + 1]) * rstd, 0.f);
-              w[q] = pack_bf16x2(a * a, b * b);
-            }
-            dst[j] = make_uint4(w[0], w[1], w[2], w[3]);
-          }
+      for (int it = 0; it < 8; ++it) {
+        const int rr = it * 4 + rsub, grow = row0 + rr;
+        if (grow < p.M) {
+          const float4 v = stg[rr * 8 + (c4 ^ (rr & 7))];
+          const size_t off = (size_t)l * p.out_ls + (size_t)grow * p.N + col;
+          if (EPI == UEPI_F32) *reinterpret_cast<float4 *>(p.c + (size_t)ks * p.out_ss + off) = v;
+          else *reinterpret_cast<uint2 *>(p.z + off) = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
         }
       }
+      __syncwarp();
     }
   } else if (EPI == UEPI_RESID) {
     // Ten bytes move per accumulator element here (x read, a and u written), so the accesses must be whole lines:
