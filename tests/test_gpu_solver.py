@@ -59,6 +59,27 @@ def test_solver_argument_errors():
         assert e.value.code == snlp.ERR_ARG
 
 
+@pytest.mark.parametrize("name", list(CASES))
+def test_zero_sweeps_return_the_initialisation(name):
+    """K = 0 with the h0 initialisation: states 0..S are the sequential ones and every later state is a copy of h_S
+    (Alg. 2 line 5 with nothing after it).  The tensor-core path does not write those copies when a sweep follows, so
+    this is the one call in which it has to."""
+    from paper_2605_17842_b200 import snlp
+    cfg, B, T = CASES[name]
+    W = synth.make_weights(cfg, seed=1234, std=0.05, embed_std=1.0)
+    h0 = synth.make_hidden(cfg, B, T, seed=7)
+    m = make_model(cfg, W, max_rows=B * T, max_batch=B)
+    mode = O.MODE_HCN if cfg.n_streams > 1 else O.MODE_IDN
+    seq = m.forward_sequential(dev(h0))
+    m.forward_solver(dev(h0), snlp.Solver(K=2, mode=mode))     # leave other values in the trace first
+    for S in (0, 2):
+        tr, _ = m.forward_solver(dev(h0), snlp.Solver(K=0, mode=mode, prefix=S))
+        assert torch.equal(tr[: S + 1], seq[: S + 1])
+        for l in range(S + 1, cfg.n_layer + 1):
+            assert torch.equal(tr[l], tr[S]), (S, l)
+    m.device_status()
+
+
 def test_decode_step_with_prefix_and_fwd_init():
     from paper_2605_17842_b200 import snlp
     cfg = synth.ModelConfig(5, 256, 2, 128, 512, 1024, 1, "bf16")
