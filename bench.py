@@ -101,18 +101,14 @@ def alg_bytes(cfg, B, ctx):
 # ----------------------------------------------------------------------------------------------
 def run_ours(args):
     import torch
-    import torch.distributed as dist
 
-    from paper_2605_17842_b200 import build
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2605_17842_b200 import build, replicas
+    rk = replicas.ranks_from_env()
+    rank, world, local = rk.rank, rk.world, rk.local
     if rank == 0:
         build.build()
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-        dist.barrier()
+    replicas.init(rk, "nccl", torch.device("cuda", local))
     from paper_2605_17842_b200 import snlp, synth
 
     cfg = d20()
@@ -126,8 +122,7 @@ def run_ours(args):
     hbm_peak, peak_src = peaks()
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        replicas.barrier(rk)
         torch.cuda.synchronize()
 
     def timed_decode(kv, first_tok, K, n_warm, n_steps):
@@ -143,11 +138,7 @@ def run_ours(args):
             model.decode_step(kv, tok, K, snlp.MODE_IDN, tok_out=tok)
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = replicas.max_over_ranks(rk, e0.elapsed_time(e1), "cuda")
         return ms / n_steps
 
     results = {}
@@ -178,7 +169,7 @@ def run_ours(args):
         if args.only_main:
             if rank == 0:
                 print(json.dumps({"metric": "d20 decode tokens/s SNLP(K) vs sequential; sweep HBM GB/s vs B200 peak",
-                                  "value": world * 1e3 / ms_main, "unit": "tokens/s", "ms_per_step": ms_main,
+                                  "value": replicas.whole_job_rate(rk, 1, ms_main), "unit": "tokens/s", "ms_per_step": ms_main,
                                   "steps": steps, "warmup": warmup, "note": "--only-main: headline point only"}))
             return
 
@@ -214,11 +205,7 @@ def run_ours(args):
             e2e_step()
         e1.record()
         barrier()
-        ms_e2e = e0.elapsed_time(e1) / e2e_steps
-        if world > 1:
-            t = torch.tensor([ms_e2e], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        ms_e2e = replicas.max_over_ranks(rk, e0.elapsed_time(e1) / e2e_steps, "cuda")
 
         # ---- per-kernel device time (CUDA events inside the library, on its launch stream) ----
         model.set_flag(2, 1)
@@ -237,7 +224,7 @@ def run_ours(args):
 
     if rank != 0:
         if world > 1:
-            dist.destroy_process_group()
+            replicas.finish(rk)
         return
 
     ctx_mid = CTX + warmup + steps / 2.0
@@ -268,14 +255,14 @@ def run_ours(args):
 
     table = {}
     for (B, K), ms in sorted(results.items()):
-        table[f"B{B}_" + ("seq" if K == 0 else f"K{K}")] = {"ms_per_step": ms, "tok_s": world * B * 1e3 / ms}
+        table[f"B{B}_" + ("seq" if K == 0 else f"K{K}")] = {"ms_per_step": ms, "tok_s": replicas.whole_job_rate(rk, B, ms)}
     speedups = {f"B{B}_K{K}": results[(B, 0)] / results[(B, K)] for (B, K) in results if K > 0 and (B, 0) in results}
 
     cpu = cpu_baseline_sample(cfg, W, seconds=8.0 if args.quick else 20.0)
 
     line = {
         "metric": "d20 decode tokens/s SNLP(K) vs sequential; sweep HBM GB/s vs B200 peak",
-        "value": world * 1e3 / ms_main,
+        "value": replicas.whole_job_rate(rk, 1, ms_main),
         "unit": "tokens/s",
         "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms_main,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -301,8 +288,7 @@ def run_ours(args):
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.finish(rk)
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch (all 20 layers) of k_umma_gemm in this workload, from the
