@@ -35,7 +35,9 @@ __device__ __forceinline__ float4 f4_fma(float s, float4 a, float4 b) {
   return make_float4(fmaf(s, a.x, b.x), fmaf(s, a.y, b.y), fmaf(s, a.z, b.z), fmaf(s, a.w, b.w));
 }
 __device__ __forceinline__ float4 f4_scale(float s, float4 a) { return make_float4(s * a.x, s * a.y, s * a.z, s * a.w); }
-__device__ __forceinline__ float f4_sq(float4 a) { return a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w; }
+// explicit fused multiply-adds: the same bits in every kernel that takes a row's sum of squares, whatever the compiler
+// would otherwise contract
+__device__ __forceinline__ float f4_sq(float4 a) { return fmaf(a.w, a.w, fmaf(a.z, a.z, fmaf(a.y, a.y, a.x * a.x))); }
 
 // Depth of the operand ring of k_correct (steps in flight per thread) and its shared-memory size.
 __host__ __device__ constexpr int corr_depth(int ns) { return ns <= 1 ? 4 : (ns <= 4 ? 3 : 2); }
@@ -267,15 +269,30 @@ __global__ void k_prep_rows(const float *__restrict__ trace, int l0, int M, int 
 // l0 .. L-1 get their bf16 attention-branch input, its sums of squares and (mHC) the fp32 MLP pre-map, all from one read
 // of the row.  Same values as k_bcast_trace followed by k_prep_rows.  grid (M), d/4 threads (d a multiple of 128).
 // write_trace == 0 leaves the copies out: the first pass then reads state l0 wherever it needs a later state.
+// ids != nullptr: state l0 itself is the embedding of the row's token (replicated into every stream) and is written
+// here too, so that a decode step needs no separate embedding kernel.
 template <int NS>
 __global__ void k_init_rows(float *__restrict__ trace, int l0, int L, int M, int d, const HcCoef *__restrict__ coef,
-                            __nv_bfloat16 *__restrict__ xb, float *__restrict__ ssq_x, float *__restrict__ xm, int write_trace) {
+                            __nv_bfloat16 *__restrict__ xb, float *__restrict__ ssq_x, float *__restrict__ xm, int write_trace,
+                            const int32_t *__restrict__ ids = nullptr, const __nv_bfloat16 *__restrict__ table = nullptr, int vocab = 0) {
   const int d4 = d >> 2, c4 = threadIdx.x;
   const size_t row = blockIdx.x, Md4 = (size_t)M * d4;
   float4 *tr4 = reinterpret_cast<float4 *>(trace);
   float4 x[NS];
+  if (ids != nullptr) {
+    int id = ids[row];
+    id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);
+    const uint2 e = reinterpret_cast<const uint2 *>(table + (size_t)id * d)[c4];
+    const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&e.x)), hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&e.y));
 #pragma unroll
-  for (int s = 0; s < NS; ++s) x[s] = tr4[(size_t)l0 * Md4 * NS + row * NS * d4 + (size_t)s * d4 + c4];
+    for (int s = 0; s < NS; ++s) {
+      x[s] = make_float4(lo.x, lo.y, hi.x, hi.y);
+      tr4[(size_t)l0 * Md4 * NS + row * NS * d4 + (size_t)s * d4 + c4] = x[s];
+    }
+  } else {
+#pragma unroll
+    for (int s = 0; s < NS; ++s) x[s] = tr4[(size_t)l0 * Md4 * NS + row * NS * d4 + (size_t)s * d4 + c4];
+  }
   float4 v = x[0];
   uint2 pk = make_uint2(0, 0);
   float ss = 0.f;

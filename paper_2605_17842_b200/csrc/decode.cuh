@@ -225,7 +225,9 @@ __global__ void __launch_bounds__(kGemvThreads) k_gemv_mma(GemvParams p) {
 }
 
 // Final argmax over the per-tile partials (ties -> lowest index).  One block per token.
-static __global__ void k_argmax_tiles(const float *__restrict__ pm_val, const int *__restrict__ pm_idx, int ntile, int32_t *__restrict__ out) {
+// bump (nullable): a device counter incremented by one once per launch (the cache position after a decode step).
+static __global__ void k_argmax_tiles(const float *__restrict__ pm_val, const int *__restrict__ pm_idx, int ntile, int32_t *__restrict__ out,
+                                      int *__restrict__ bump = nullptr) {
   __shared__ float sv[32];
   __shared__ int si[32];
   const int tok = blockIdx.x;
@@ -250,6 +252,7 @@ static __global__ void k_argmax_tiles(const float *__restrict__ pm_val, const in
     for (int i = 1; i < nw; ++i)
       if (sv[i] > bv || (sv[i] == bv && si[i] < bi)) { bv = sv[i]; bi = si[i]; }
     out[tok] = bi == 0x7fffffff ? 0 : bi;
+    if (bump != nullptr && tok == 0) *bump += 1;
   }
 }
 

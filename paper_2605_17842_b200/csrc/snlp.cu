@@ -131,6 +131,7 @@ struct Fwd {
   const int *pos;       // device: first position of this call
   int pos_hi;           // host copy of *pos
   int kv_rows;          // rows per sequence in the key / value store
+  const int32_t *embed_ids = nullptr;   // non-NULL: state 0 is the embedding of these tokens and has not been written yet
   bool last_pass = false;   // no sweep follows this correction: it need not prepare the next sweep's branch inputs
   int implicit_state = -1;  // >= 0: states after this one are not materialised yet and equal it (first pass after Alg. 2 line 5)
   cudaStream_t st;
@@ -776,13 +777,19 @@ static int check_solver(const snlp_model *m, const snlp_solver &sol, const char 
   return SNLP_OK;
 }
 
-// General Alg. 2 over the internal trace (trace[0] must hold h_0): sequential prefix, initialisation, K sweeps over the
+static int embed_impl(snlp_model *m, cudaStream_t st, const int32_t *ids, int rows, float *h0);
+
+// General Alg. 2 over the internal trace (trace[0] must hold h_0, or f.embed_ids the tokens it is the embedding of): sequential prefix, initialisation, K sweeps over the
 // suffix in chunks of `fuse` fused layers (Eq. 5 for fuse = 1, Eq. 11 otherwise).
 static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *resnorm_out) {
   const snlp_config &c = m->cfg;
   const int L = c.n_layer, F = sol.fuse;
   const bool seq = sol.mode == SNLP_MODE_SEQUENTIAL;
   const int S = (seq && F == 1) ? L : sol.prefix;
+  // a decode step hands over token ids instead of state 0: the initialisation kernel embeds them itself where it runs
+  // on state 0; every other path needs the embedding first
+  const bool fused_embed = f.embed_ids != nullptr && umma_path_ok(m) && S == 0 && !seq;
+  if (f.embed_ids != nullptr && !fused_embed) TRY(embed_impl(m, f.st, f.embed_ids, f.M, m->trace));
   if (resnorm_out && sol.K > 0 && !seq) CU(cudaMemsetAsync(resnorm_out, 0, (size_t)sol.K * L * 2 * sizeof(float), f.st));
   if (S > 0) {  // Alg. 2 lines 2-4
     if (umma_path_ok(m)) TRY(prep_rows(m, f, 0, 1));
@@ -804,7 +811,7 @@ static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *res
   // Alg. 2 line 5: every suffix state starts at h_S
   if (umma_path_ok(m)) {
     switch (c.n_streams) {   // one kernel: the copies and the layers' first branch inputs
-#define CASE(NS) case NS: KLAUNCH(m, f.st, KC_OTHER, k_init_rows<NS><<<f.M, c.d_model / 4, 0, f.st>>>(m->trace, S, L, f.M, c.d_model, m->coef, (__nv_bfloat16 *)m->xn, m->ssq_x, m->xm, 0)); break;
+#define CASE(NS) case NS: KLAUNCH(m, f.st, KC_OTHER, k_init_rows<NS><<<f.M, c.d_model / 4, 0, f.st>>>(m->trace, S, L, f.M, c.d_model, m->coef, (__nv_bfloat16 *)m->xn, m->ssq_x, m->xm, 0, fused_embed ? f.embed_ids : nullptr, (const __nv_bfloat16 *)m->embed, c.vocab)); break;
       CASE(1) CASE(2) CASE(3) CASE(4) CASE(5) CASE(6) CASE(7) CASE(8)
 #undef CASE
     }
@@ -861,7 +868,7 @@ static int parallel(snlp_model *m, const Fwd &f, int K, int mode, float *resnorm
 // LMHead on `rows` hidden states.  pre_xb / pre_ssq: the bf16 stream-summed rows and their sums of squares if the
 // caller already has them (slot L of the branch-input buffers after a decode-regime forward), else NULL.
 static int lm_head_impl(snlp_model *m, cudaStream_t st, const float *hL, size_t row_stride, int rows, float *logits, int32_t *argmax,
-                        const __nv_bfloat16 *pre_xb = nullptr, const float *pre_ssq = nullptr) {
+                        const __nv_bfloat16 *pre_xb = nullptr, const float *pre_ssq = nullptr, int *bump = nullptr) {
   const snlp_config &c = m->cfg;
   const int d = c.d_model, V = c.vocab, n = c.n_streams;
   if (umma_path_ok(m) && rows <= kDecodeRows) {
@@ -875,7 +882,8 @@ static int lm_head_impl(snlp_model *m, cudaStream_t st, const float *hL, size_t 
     p.ssq = pre_ssq; p.nparts = P; p.eps = c.rms_eps;
     p.logits = logits; p.pm_val = m->pm_val; p.pm_idx = m->pm_idx;
     TRY(umma_gemm<UEPI_LMHEAD>(m, st, KC_LMHEAD, pre_xb, 0, m->w_lm, 0, p, rows, V, d, 1, 1));
-    if (argmax) KLAUNCH(m, st, KC_LMHEAD, k_argmax_tiles<<<rows, 256, 0, st>>>(m->pm_val, m->pm_idx, V / m->w_lm.BN, argmax));
+    if (argmax) KLAUNCH(m, st, KC_LMHEAD, k_argmax_tiles<<<rows, 256, 0, st>>>(m->pm_val, m->pm_idx, V / m->w_lm.BN, argmax, bump));
+    else if (bump) KLAUNCH(m, st, KC_OTHER, k_add_int<<<1, 1, 0, st>>>(bump, 1));
     return SNLP_OK;
   }
   for (int r0 = 0; r0 < rows; r0 += m->logit_rows) {
@@ -1100,23 +1108,25 @@ extern "C" int snlp_prefill(snlp_model *m, snlp_kv *kv, const int32_t *ids, int 
 }
 
 // greedy tokens of all `rows` rows of the forward that just ran (rows <= 16)
-static int lm_head_tail(snlp_model *m, cudaStream_t st, int rows, int32_t *argmax) {
+// bump (nullable): device counter to advance by one after the tokens are out (fused into the arg-max kernel where there is one)
+static int lm_head_tail(snlp_model *m, cudaStream_t st, int rows, int32_t *argmax, int *bump = nullptr) {
   const snlp_config &c = m->cfg;
   const size_t nd = (size_t)c.n_streams * c.d_model, L = c.n_layer;
   if (umma_path_ok(m) && rows <= kDecodeRows)  // the correction left the LM-head input in slot L of xb / ssq_x
     return lm_head_impl(m, st, nullptr, 0, rows, nullptr, argmax, (const __nv_bfloat16 *)m->xn + L * rows * c.d_model,
-                        m->ssq_x + L * (c.d_model / 128) * rows);
-  return lm_head_impl(m, st, m->trace + L * rows * nd, nd, rows, nullptr, argmax);
+                        m->ssq_x + L * (c.d_model / 128) * rows, bump);
+  TRY(lm_head_impl(m, st, m->trace + L * rows * nd, nd, rows, nullptr, argmax));
+  if (bump) KLAUNCH(m, st, KC_OTHER, k_add_int<<<1, 1, 0, st>>>(bump, 1));
+  return SNLP_OK;
 }
 
 // enqueue one decode step (no graph handling, no host-side length update)
 static int decode_launches(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, const snlp_solver &sol, int32_t *tok_out, float *resnorm_out,
                            cudaStream_t st) {
-  TRY(embed_impl(m, st, tok_in, kv->B, m->trace));
   Fwd f = kv_fwd(m, kv, 1, st);
+  f.embed_ids = tok_in;
   TRY(solve(m, f, sol, resnorm_out));
-  TRY(lm_head_tail(m, st, kv->B, tok_out));
-  KLAUNCH(m, st, KC_OTHER, k_add_int<<<1, 1, 0, st>>>(kv->pos, 1));
+  TRY(lm_head_tail(m, st, kv->B, tok_out, kv->pos));   // also advances the cache position
   return SNLP_OK;
 }
 
