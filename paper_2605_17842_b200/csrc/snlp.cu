@@ -113,6 +113,7 @@ struct snlp_model {
   int n_sm = 148;
   EncodeTiledFn encode_tiled = nullptr;  // cuTensorMapEncodeTiled, looked up through the runtime
   int *dev_err = nullptr;                // raised by a kernel whose bounded wait expired
+  int lm_tiles = 0;                   // column tiles of the last LM-head launch (its arg-max partials)
   cudaStream_t cap_stream = nullptr;  // capture target: graphs are recorded here and replayed on the caller's stream
 };
 
@@ -608,14 +609,25 @@ static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat1
     KLAUNCH(m, st, cls, k_umma_gemm2<EPI><<<2 * pairs, kUmmaThreads, kU2Smem, st>>>(ta, w.tm_half, p));
     return SNLP_OK;
   }
+  // Decode regime: a CTA streams at most ~52 GB/s, so a launch that does not even occupy every SM (a sequential step's
+  // single layer: 15-20 items) lasts as long as one item.  The column tiling does not touch the numbers (every output
+  // column is its own dot product), so such launches take 128-wide tiles: twice the CTAs, half the bytes each.  With
+  // all SMs busy the 256-wide tile is the faster one (a 128-wide MMA costs as much as a 256-wide one).  The
+  // out-projection keeps its tile width whatever the launch: its epilogue emits per-tile partial sums of squares,
+  // which must not depend on how many layers a launch covers.
+  int bn = w.BN;
+  if (small && w.BN == 256 && EPI != UEPI_RESID && (N / 256) * ksplit * nl < m->n_sm) bn = 128;
+  const CUtensorMap &tmw = bn == w.BN ? w.tm : w.tm_half;
+  p.Nt = N / bn;
+  if (EPI == UEPI_LMHEAD) m->lm_tiles = p.Nt;
   const int items = p.Mt * p.Nt * ksplit * nl;
   const int grid = items < m->n_sm ? items : m->n_sm;
 #define SNLP_UMMA_LAUNCH(BN_, AM_)                                                                                                   \
   do {                                                                                                                               \
     p.nstages = UmmaCfg<BN_, AM_>::kStages;                                                                                          \
-    KLAUNCH(m, st, cls, k_umma_gemm<BN_, AM_, EPI><<<grid, kUmmaThreads, UmmaCfg<BN_, AM_>::kSmem, st>>>(ta, w.tm, p));              \
+    KLAUNCH(m, st, cls, k_umma_gemm<BN_, AM_, EPI><<<grid, kUmmaThreads, UmmaCfg<BN_, AM_>::kSmem, st>>>(ta, tmw, p));                \
   } while (0)
-  if (w.BN == 256) {
+  if (bn == 256) {
     if (small) SNLP_UMMA_LAUNCH(256, 16);
     else if (EPI != UEPI_LMHEAD) SNLP_UMMA_LAUNCH(256, 128);
   } else {
@@ -882,7 +894,7 @@ static int lm_head_impl(snlp_model *m, cudaStream_t st, const float *hL, size_t 
     p.ssq = pre_ssq; p.nparts = P; p.eps = c.rms_eps;
     p.logits = logits; p.pm_val = m->pm_val; p.pm_idx = m->pm_idx;
     TRY(umma_gemm<UEPI_LMHEAD>(m, st, KC_LMHEAD, pre_xb, 0, m->w_lm, 0, p, rows, V, d, 1, 1));
-    if (argmax) KLAUNCH(m, st, KC_LMHEAD, k_argmax_tiles<<<rows, 256, 0, st>>>(m->pm_val, m->pm_idx, V / m->w_lm.BN, argmax, bump));
+    if (argmax) KLAUNCH(m, st, KC_LMHEAD, k_argmax_tiles<<<rows, 256, 0, st>>>(m->pm_val, m->pm_idx, m->lm_tiles, argmax, bump));
     else if (bump) KLAUNCH(m, st, KC_OTHER, k_add_int<<<1, 1, 0, st>>>(bump, 1));
     return SNLP_OK;
   }
