@@ -447,62 +447,94 @@ def run_prefill_workload(args, name):
 
 
 def run_spec_workload(args):
-    """d20 self-speculative decoding: IDN K=2 drafter, 8-token blocks, batch 1, 4096-token random-prefill context."""
+    """d20 self-speculative decoding: IDN K=2 drafter, 8-token blocks, batch 1, 4096-token random-prefill context.
+
+    Two synthetic models: the benchmark's initialisation (every matrix N(0, 0.02)), whose branches are several times
+    larger than the embedded state, so that a K=2 drafter almost never agrees with the sequential model; and the same
+    weights with unit-scale embeddings (branches small against the state, the regime J ~ I the method is built for),
+    reported beside it and labelled as such.  Trained checkpoints are not available."""
     import torch
     from paper_2605_17842_b200 import build
     build.build()
-    from oracle import snlp_oracle as O
     from paper_2605_17842_b200 import snlp, synth
     torch.cuda.set_device(0)
     cfg = d20()
     ctx, block, K, n_gen = 4096, 8, 2, 512 if args.steps >= 256 else args.steps
-    W = synth.make_weights(cfg, seed=1234)
-    model = snlp.Model(cfg, max_rows=2048, max_batch=1, max_ctx=ctx + n_gen + 2 * block + 8)
-    model.load_weights(W)
     ids = torch.from_numpy(synth.make_ids(cfg, 1, ctx, seed=6)).cuda()
     stream = torch.cuda.Stream()
-    with torch.cuda.stream(stream):
-        kv = model.kv_cache(1, ctx + n_gen + 2 * block + 8)
-        first = model.prefill(kv, ids)
-        # plain sequential greedy decoding (the stream the verifier guarantees)
-        tok = first.clone()
-        for _ in range(8):
-            model.decode_step(kv, tok, 0, tok_out=tok)
-        kv.truncate(ctx)
-        tok = first.clone()
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        seq_tokens = []
-        for _ in range(n_gen):
-            model.decode_step(kv, tok, 0, tok_out=tok)
-            seq_tokens.append(tok.clone())
-        torch.cuda.synchronize()
-        seq_s = time.perf_counter() - t0
-        seq_tokens = torch.stack(seq_tokens).flatten().tolist()
-        # self-speculative decoding
-        kv.truncate(ctx)
-        last = first.clone()
-        model.draft_and_verify(kv, last, block, K)   # warm-up round (graphs)
-        kv.truncate(ctx)
-        last = first.clone()
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        got, acc, rounds = [], 0, 0
-        while len(got) < n_gen:
-            em, na = model.draft_and_verify(kv, last, block, K)
-            got += em
-            acc += na
-            rounds += 1
-        torch.cuda.synchronize()
-        spec_s = time.perf_counter() - t0
-    alpha = acc / (rounds * block)
-    same = got[:n_gen] == seq_tokens[:n_gen]
-    line = {"metric": "d20 self-speculative decode accepted tokens/s", "value": len(got) / spec_s, "unit": "tokens/s", "higher_is_better": True,
+
+    def measure(W):
+        model = snlp.Model(cfg, max_rows=2048, max_batch=1, max_ctx=ctx + n_gen + 2 * block + 8)
+        model.load_weights(W)
+        with torch.cuda.stream(stream):
+            kv = model.kv_cache(1, ctx + n_gen + 2 * block + 8)
+            first = model.prefill(kv, ids)
+            # plain sequential greedy decoding (the stream the verifier guarantees)
+            tok = first.clone()
+            for _ in range(8):
+                model.decode_step(kv, tok, 0, tok_out=tok)
+            kv.truncate(ctx)
+            tok = first.clone()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            seq_tokens = []
+            for _ in range(n_gen):
+                model.decode_step(kv, tok, 0, tok_out=tok)
+                seq_tokens.append(tok.clone())
+            torch.cuda.synchronize()
+            seq_s = time.perf_counter() - t0
+            seq_tokens = torch.stack(seq_tokens).flatten().tolist()
+            # the drafter alone (its speed relative to the sequential model enters the paper's estimator)
+            kv.truncate(ctx)
+            tok = first.clone()
+            for _ in range(8):
+                model.decode_step(kv, tok, K, tok_out=tok)
+            kv.truncate(ctx)
+            tok = first.clone()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for _ in range(n_gen):
+                model.decode_step(kv, tok, K, tok_out=tok)
+            torch.cuda.synchronize()
+            draft_s = time.perf_counter() - t0
+            # self-speculative decoding
+            kv.truncate(ctx)
+            last = first.clone()
+            model.draft_and_verify(kv, last, block, K)   # warm-up round (graphs)
+            kv.truncate(ctx)
+            last = first.clone()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            got, acc, rounds, rejects = [], 0, 0, 0
+            while len(got) < n_gen:
+                em, na = model.draft_and_verify(kv, last, block, K)
+                got += em
+                acc += na
+                rounds += 1
+                rejects += na < block
+            torch.cuda.synchronize()
+            spec_s = time.perf_counter() - t0
+        model.device_status()
+        kv.close()
+        model.close()
+        alpha = acc / (rounds * block)                               # accepted drafts / proposed drafts
+        a_tok = acc / max(acc + rejects, 1)                          # per-token acceptance: accepted / (accepted + first rejections)
+        s_rel = seq_s / draft_s                                      # drafter speed in units of the sequential model's
+        num = block + 1.0 if a_tok >= 1.0 else (1.0 - a_tok ** (block + 1)) / (1.0 - a_tok)
+        return {"accepted_tok_s": len(got) / spec_s, "generated": len(got), "rounds": rounds, "acceptance_rate": alpha,
+                "per_token_acceptance": a_tok, "tokens_per_round": len(got) / rounds, "sequential_tok_s": n_gen / seq_s, "drafter_tok_s": n_gen / draft_s,
+                "speedup_vs_own_sequential": (len(got) / spec_s) / (n_gen / seq_s),
+                "estimator_speedup": num / (block / s_rel + 1.0),      # ((1 - a^(B+1)) / (1 - a)) / (B / s + 1) with the per-token a, Sec. 5.1
+                "output_equals_sequential_greedy": bool(got[:n_gen] == seq_tokens[:n_gen])}
+
+    base = measure(synth.make_weights(cfg, seed=1234))
+    pert = measure(synth.make_weights(cfg, seed=1234, embed_std=1.0))
+    line = {"metric": "d20 self-speculative decode accepted tokens/s", "value": base["accepted_tok_s"], "unit": "tokens/s", "higher_is_better": True,
             "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": "d20 self-speculative decode: IDN K=2 drafter, block 8, batch 1, ctx 4096 random prefill, greedy"},
-            "generated": len(got), "rounds": rounds, "acceptance_rate": alpha, "tokens_per_round": len(got) / rounds,
-            "sequential_tok_s": n_gen / seq_s, "speedup_vs_own_sequential": (len(got) / spec_s) / (n_gen / seq_s),
-            "output_equals_sequential_greedy": bool(same),
+            **{k: v for k, v in base.items() if k != "accepted_tok_s"},
+            "unit_scale_embeddings": {"what": "same shapes and seeds, embedding rows N(0, 1) instead of N(0, 0.02): branches are small "
+                                              "against the residual state, so the solver's bias is small", **pert},
             "note": "timed with the host clock around the whole loop (each round synchronises once to learn the accepted count)"}
     print(json.dumps(line))
 
