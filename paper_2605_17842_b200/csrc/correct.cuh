@@ -29,12 +29,52 @@ struct CorrParams {
   unsigned *counter; // zero on entry, left zero on exit
 };
 
-__device__ __forceinline__ float4 f4_add(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
-__device__ __forceinline__ float4 f4_sub(float4 a, float4 b) { return make_float4(a.x - b.x, a.y - b.y, a.z - b.z, a.w - b.w); }
-__device__ __forceinline__ float4 f4_fma(float s, float4 a, float4 b) {
-  return make_float4(fmaf(s, a.x, b.x), fmaf(s, a.y, b.y), fmaf(s, a.z, b.z), fmaf(s, a.w, b.w));
+// float4 arithmetic on the packed fp32 pipe (two IEEE operations per instruction: same bits as the scalar forms, half
+// the issue slots; the correction is issue-limited for n > 1 streams)
+__device__ __forceinline__ unsigned long long pk2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
 }
-__device__ __forceinline__ float4 f4_scale(float s, float4 a) { return make_float4(s * a.x, s * a.y, s * a.z, s * a.w); }
+__device__ __forceinline__ void upk2(unsigned long long v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ float4 f4_add(float4 a, float4 b) {
+  unsigned long long d0, d1;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d0) : "l"(pk2(a.x, a.y)), "l"(pk2(b.x, b.y)));
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d1) : "l"(pk2(a.z, a.w)), "l"(pk2(b.z, b.w)));
+  float4 r;
+  upk2(d0, r.x, r.y);
+  upk2(d1, r.z, r.w);
+  return r;
+}
+__device__ __forceinline__ float4 f4_sub(float4 a, float4 b) {
+  unsigned long long d0, d1;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d0) : "l"(pk2(a.x, a.y)), "l"(pk2(b.x, b.y)));
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d1) : "l"(pk2(a.z, a.w)), "l"(pk2(b.z, b.w)));
+  float4 r;
+  upk2(d0, r.x, r.y);
+  upk2(d1, r.z, r.w);
+  return r;
+}
+__device__ __forceinline__ float4 f4_fma(float s, float4 a, float4 b) {
+  unsigned long long d0, d1;
+  const unsigned long long ss = pk2(s, s);
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d0) : "l"(ss), "l"(pk2(a.x, a.y)), "l"(pk2(b.x, b.y)));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d1) : "l"(ss), "l"(pk2(a.z, a.w)), "l"(pk2(b.z, b.w)));
+  float4 r;
+  upk2(d0, r.x, r.y);
+  upk2(d1, r.z, r.w);
+  return r;
+}
+__device__ __forceinline__ float4 f4_scale(float s, float4 a) {
+  unsigned long long d0, d1;
+  const unsigned long long ss = pk2(s, s);
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d0) : "l"(ss), "l"(pk2(a.x, a.y)));
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d1) : "l"(ss), "l"(pk2(a.z, a.w)));
+  float4 r;
+  upk2(d0, r.x, r.y);
+  upk2(d1, r.z, r.w);
+  return r;
+}
 // explicit fused multiply-adds: the same bits in every kernel that takes a row's sum of squares, whatever the compiler
 // would otherwise contract
 __device__ __forceinline__ float f4_sq(float4 a) { return fmaf(a.w, a.w, fmaf(a.z, a.z, fmaf(a.y, a.y, a.x * a.x))); }
