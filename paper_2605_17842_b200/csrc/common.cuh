@@ -56,6 +56,25 @@ __device__ __forceinline__ float block_sum(float v, float *red) {
   return s;
 }
 
+// Two fp32 values in one 64-bit register for the packed fp32 pipe (add / mul / fma .f32x2: two IEEE operations per
+// instruction, bit-identical to the scalar forms).
+__device__ __forceinline__ unsigned long long pk2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void upk2(unsigned long long v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned long long mul2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 // 16-byte asynchronous global -> shared copy (L2 only); valid == false zero-fills the destination instead.
 __device__ __forceinline__ void cp_async16(void *smem, const void *gmem, bool valid) {
   const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);

@@ -31,12 +31,6 @@ struct CorrParams {
 
 // float4 arithmetic on the packed fp32 pipe (two IEEE operations per instruction: same bits as the scalar forms, half
 // the issue slots; the correction is issue-limited for n > 1 streams)
-__device__ __forceinline__ unsigned long long pk2(float lo, float hi) {
-  unsigned long long r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void upk2(unsigned long long v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
 __device__ __forceinline__ float4 f4_add(float4 a, float4 b) {
   unsigned long long d0, d1;
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d0) : "l"(pk2(a.x, a.y)), "l"(pk2(b.x, b.y)));

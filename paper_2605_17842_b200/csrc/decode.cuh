@@ -299,10 +299,14 @@ static __global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat
       if (tid == 0) { dst[128] = -INFINITY; dst[129] = 0.f; }
       continue;
     }
-    float qv[8];
+    // query features and the output accumulator as fp32 pairs: the dot products and the value accumulation run on the
+    // packed fp32 pipe (the kernel is limited by instruction issue as much as by bandwidth)
+    unsigned long long qv2[4], acc2[4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) qv[i] = qs[t][li * 8 + i];
-    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int i = 0; i < 4; ++i) {
+      qv2[i] = pk2(qs[t][li * 8 + 2 * i], qs[t][li * 8 + 2 * i + 1]);
+      acc2[i] = pk2(0.f, 0.f);
+    }
     float mrun = -INFINITY, lrun = 0.f;
     // The chunk is walked in 32-key mini-blocks (4 keys per half-warp), software-pipelined through two register
     // buffers: the loads of the next mini-block are in flight while the current one is reduced.
@@ -323,13 +327,15 @@ static __global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat
       for (int j = 0; j < JM; ++j) {
         const int key = base + hw + 8 * j;
         const __nv_bfloat162 *k2 = reinterpret_cast<const __nv_bfloat162 *>(&kr[j]);
-        float dot = 0.f;
+        unsigned long long d2 = pk2(0.f, 0.f);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 f = __bfloat1622float2(k2[i]);
-          dot = fmaf(qv[2 * i], f.x, dot);
-          dot = fmaf(qv[2 * i + 1], f.y, dot);
+          d2 = fma2(qv2[i], pk2(f.x, f.y), d2);
         }
+        float dlo, dhi;
+        upk2(d2, dlo, dhi);
+        float dot = dlo + dhi;
         dot += __shfl_xor_sync(0xffffffffu, dot, 8);
         dot += __shfl_xor_sync(0xffffffffu, dot, 4);
         dot += __shfl_xor_sync(0xffffffffu, dot, 2);
@@ -342,7 +348,7 @@ static __global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat
       const float resc = mrun == -INFINITY ? 0.f : __expf(mrun - mnew);
       lrun *= resc;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) acc[i] *= resc;
+      for (int i = 0; i < 4; ++i) acc2[i] = mul2(acc2[i], pk2(resc, resc));
 #pragma unroll
       for (int j = 0; j < JM; ++j) {
         const float pj = s[j] == -INFINITY ? 0.f : __expf(s[j] - mnew);
@@ -351,8 +357,7 @@ static __global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 f = __bfloat1622float2(v2[i]);
-          acc[2 * i] = fmaf(pj, f.x, acc[2 * i]);
-          acc[2 * i + 1] = fmaf(pj, f.y, acc[2 * i + 1]);
+          acc2[i] = fma2(pk2(pj, pj), pk2(f.x, f.y), acc2[i]);
         }
       }
       mrun = mnew;
@@ -372,7 +377,7 @@ static __global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat
       }
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) hacc[hw][li * 8 + i] = acc[i];
+    for (int i = 0; i < 4; ++i) upk2(acc2[i], hacc[hw][li * 8 + 2 * i], hacc[hw][li * 8 + 2 * i + 1]);
     if (li == 0) { hm[hw] = mrun; hl[hw] = lrun; }
     __syncthreads();
     {  // merge the 8 half-warps in index order
