@@ -293,7 +293,7 @@ def run_ours(args):
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch (all 20 layers) of k_umma_gemm in this workload, from the
 # ncu capture summarised in profiles/k_umma_gemm_d20_decode.md
-NCU_TRAFFIC_BYTES: dict = {"qkv": 201.5e6, "out_proj": 65.9e6, "mlp_up": 265.9e6, "mlp_down": 266.4e6}
+NCU_TRAFFIC_BYTES: dict = {"qkv": 200.6e6, "out_proj": 65.9e6, "mlp_up": 265.8e6, "mlp_down": 266.3e6}
 
 
 # ----------------------------------------------------------------------------------------------
