@@ -373,14 +373,15 @@ __global__ void k_prep_lm(const float *__restrict__ h, size_t row_stride, int ns
 
 // Latency-oriented variant for the decode regime (a handful of rows): the per-thread loop over
 // layers above serialises ~7 dependent-latency loads per layer, which dominates when there are too
-// few threads to hide it.  Here a block owns 32 float4 columns of one row; its 8 warps first fetch
-// every layer's branch outputs and old states into shared memory (four layers per warp at a time, all loads
-// issued before the first is consumed), then warp 0 runs the serial recurrence out of shared memory, keeping the
-// per-layer sums of squares per lane; afterwards all warps reduce those, so the serial loop carries no shuffles.
-// Same arithmetic, same summation order as k_correct.
-// grid (d/128, M), 256 threads; dynamic shared memory nl*32*(2+NS) float4 + nl*2 floats + nl*3*32 floats.
+// few threads to hide it.  Here a block owns 32 float4 columns of one row; its 16 warps first fetch
+// every layer's branch outputs (with up to four K-split partial sums each) and old states into shared memory (two
+// layers per warp at a time, all loads issued before the first is consumed), then warp 0 runs the serial recurrence
+// out of shared memory, keeping the per-layer sums of squares per lane; afterwards all warps reduce those, so the
+// serial loop carries no shuffles.  Same arithmetic, same summation order as k_correct.
+// grid (d/128, M), 512 threads; dynamic shared memory nl*32*(2+NS) float4 + nl*2 floats + nl*3*32 floats.
+constexpr int kCorrSmallWarps = 16;
 template <int NS>
-__global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
+__global__ void __launch_bounds__(32 * kCorrSmallWarps) k_correct_small(CorrParams p) {
   extern __shared__ float4 s_buf[];
   const int d4 = p.d >> 2;
   const int c = threadIdx.x & 31, ll = threadIdx.x >> 5;
@@ -396,28 +397,44 @@ __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
   float *snorm = reinterpret_cast<float *>(s_buf + (size_t)p.nl * 32 * (2 + NS));          // [nl][2]
   float *sred = snorm + (size_t)p.nl * 2;                                                  // [nl][3][32]: per-lane xs, rs, hs
   const bool want_norm = p.partial != nullptr;
+  float4 first[NS];  // warp 0: the state the recurrence starts from
   if (active) {
-#pragma unroll 1
-    for (int i0 = ll; i0 < p.nl; i0 += 32) {
-      float4 av[4], mv[4], ov[4][NS];
+    if (ll == 0) {
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const int i = i0 + 8 * k;
+      for (int s = 0; s < NS; ++s) first[s] = tr4[(size_t)p.l0 * state4 + st_off + (size_t)s * d4];
+    }
+#pragma unroll 1
+    for (int i0 = ll; i0 < p.nl; i0 += 2 * kCorrSmallWarps) {
+      // every load of two steps (K-split partial sums included) is issued before the first is consumed
+      float4 av[2], mv[2], aq[2][3], mq[2][3], ov[2][NS];
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        const int i = i0 + kCorrSmallWarps * k;
         if (i < p.nl) {
           const int l = p.l0 + i * p.lstep, ln = l + p.lstep;  // this step maps state l to state ln
           av[k] = a4[(size_t)l * Md4 + bm_off];
           mv[k] = m4[(size_t)l * Md4 + bm_off];
 #pragma unroll
+          for (int q = 1; q < 4; ++q) {
+            if (q < p.a_splits) aq[k][q - 1] = a4[(size_t)q * (p.a_ss >> 2) + (size_t)l * Md4 + bm_off];
+            if (q < p.m_splits) mq[k][q - 1] = m4[(size_t)q * (p.m_ss >> 2) + (size_t)l * Md4 + bm_off];
+          }
+#pragma unroll
           for (int r = 0; r < NS; ++r) ov[k][r] = tr4[(size_t)(p.implicit_old ? p.l0 : ln) * state4 + st_off + (size_t)r * d4];
         }
       }
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const int i = i0 + 8 * k;
+      for (int k = 0; k < 2; ++k) {
+        const int i = i0 + kCorrSmallWarps * k;
         if (i < p.nl) {
+#pragma unroll
+          for (int q = 1; q < 4; ++q) {  // partial sums are added in slice order
+            if (q < p.a_splits) av[k] = f4_add(av[k], aq[k][q - 1]);
+            if (q < p.m_splits) mv[k] = f4_add(mv[k], mq[k][q - 1]);
+          }
           const int l = p.l0 + i * p.lstep;
-          for (int q = 1; q < p.a_splits; ++q) av[k] = f4_add(av[k], a4[(size_t)q * (p.a_ss >> 2) + (size_t)l * Md4 + bm_off]);
-          for (int q = 1; q < p.m_splits; ++q) mv[k] = f4_add(mv[k], m4[(size_t)q * (p.m_ss >> 2) + (size_t)l * Md4 + bm_off]);
+          for (int q = 4; q < p.a_splits; ++q) av[k] = f4_add(av[k], a4[(size_t)q * (p.a_ss >> 2) + (size_t)l * Md4 + bm_off]);
+          for (int q = 4; q < p.m_splits; ++q) mv[k] = f4_add(mv[k], m4[(size_t)q * (p.m_ss >> 2) + (size_t)l * Md4 + bm_off]);
           sa[i * 32 + c] = av[k];
           sm[i * 32 + c] = mv[k];
 #pragma unroll
@@ -432,7 +449,7 @@ __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
     float4 oldp[NS], newp[NS];
     if (active) {
 #pragma unroll
-      for (int s = 0; s < NS; ++s) oldp[s] = newp[s] = tr4[(size_t)p.l0 * state4 + st_off + (size_t)s * d4];
+      for (int s = 0; s < NS; ++s) oldp[s] = newp[s] = first[s];
     }
     for (int i = 0; i < p.nl; ++i) {
       const int l = p.l0 + i * p.lstep, ln = l + p.lstep;  // this step maps state l to state ln
@@ -506,7 +523,7 @@ __global__ void __launch_bounds__(256) k_correct_small(CorrParams p) {
   }
   __syncthreads();
   // every warp reduces the sums of some steps (this block's 32 lanes hold 128 consecutive columns of the row: partial blockIdx.x)
-  for (int i = ll; i < p.nl; i += 8) {
+  for (int i = ll; i < p.nl; i += kCorrSmallWarps) {
     const int ln = p.l0 + (i + 1) * p.lstep;
     if (p.xb != nullptr) {
       const float xs = warp_sum(sred[(i * 3 + 0) * 32 + c]);

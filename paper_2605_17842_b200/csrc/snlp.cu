@@ -501,7 +501,7 @@ static int correct(snlp_model *m, const Fwd &f, int l0, int nsteps, int lstep, i
     dim3 grid((c.d_model / 4 + 31) / 32, f.M);
     TimedLaunch tl_(m, f.st, KC_CORRECT);
     switch (c.n_streams) {
-#define CASE(NS) case NS: k_correct_small<NS><<<grid, 256, sm_small, f.st>>>(p); break;
+#define CASE(NS) case NS: k_correct_small<NS><<<grid, 32 * kCorrSmallWarps, sm_small, f.st>>>(p); break;
       CASE(1) CASE(2) CASE(3) CASE(4)
 #undef CASE
     }
