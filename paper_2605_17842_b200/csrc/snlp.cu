@@ -609,14 +609,14 @@ static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat1
     KLAUNCH(m, st, cls, k_umma_gemm2<EPI><<<2 * pairs, kUmmaThreads, kU2Smem, st>>>(ta, w.tm_half, p));
     return SNLP_OK;
   }
-  // Decode regime: a CTA streams at most ~52 GB/s, so a launch that does not even occupy every SM (a sequential step's
-  // single layer: 15-20 items) lasts as long as one item.  The column tiling does not touch the numbers (every output
-  // column is its own dot product), so such launches take 128-wide tiles: twice the CTAs, half the bytes each.  With
-  // all SMs busy the 256-wide tile is the faster one (a 128-wide MMA costs as much as a 256-wide one).  The
-  // out-projection keeps its tile width whatever the launch: its epilogue emits per-tile partial sums of squares,
-  // which must not depend on how many layers a launch covers.
+  // Decode regime: a launch that does not occupy every SM (a sequential step's single layer: 5-20 items) lasts as long
+  // as one item.  The column tiling does not touch the numbers (every output column is its own dot product), so a
+  // launch whose 128-wide items still fit one round over the SMs takes those: twice the CTAs, half the bytes each.
+  // Beyond that the 256-wide tile is the faster one (a 128-wide MMA costs as much as a 256-wide one, which caps a
+  // CTA streaming 128-wide tiles at ~50 GB/s).  The
+  // out-projection's partial sums of squares are per 128 columns in this regime, whatever the tile width.
   int bn = w.BN;
-  if (small && w.BN == 256 && EPI != UEPI_RESID && (N / 256) * ksplit * nl < m->n_sm) bn = 128;
+  if (small && w.BN == 256 && (N / 128) * ksplit * nl <= m->n_sm) bn = 128;
   const CUtensorMap &tmw = bn == w.BN ? w.tm : w.tm_half;
   p.Nt = N / bn;
   if (EPI == UEPI_LMHEAD) m->lm_tiles = p.Nt;
@@ -659,7 +659,7 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
   T *z = (T *)m->z + (size_t)l0 * M * ff;
   float *a = m->a + l0 * Md, *mb = m->mb + l0 * Md;
   T *kc = (T *)f.kc + (size_t)l0 * f.kv_ls, *vc = (T *)f.vc + (size_t)l0 * f.kv_ls;
-  const int Pu = 2 * (d / m->w_o.BN);  // partials of sum u^2: two per column tile of the out-projection
+  const int Pu = small ? d / 128 : 2 * (d / m->w_o.BN);  // partials of sum u^2: one per 128 columns (decode regime), two per column tile of the out-projection
   const int sd = down_splits(m, M);
   {
     UmmaParams p{};

@@ -53,7 +53,7 @@ struct UmmaParams {
   __nv_bfloat16 *kc, *vc; size_t kv_ls, kv_bs;
   int T, d; const int *pos_base; const float2 *rope; float qk_eps;
   const float2 *rope_t; int rope_ld;  // rope transposed [hd/2][rope_ld], read by the prefill-regime epilogue (thread = row)
-  const float *xm; size_t xm_ls; const HcCoef *coef; float *ssq_out;   // UEPI_RESID; ssq_out [nl][Nt][M]
+  const float *xm; size_t xm_ls; const HcCoef *coef; float *ssq_out;   // UEPI_RESID; ssq_out [nl][partials][M]
   float *logits; float *pm_val; int *pm_idx;                            // UEPI_LMHEAD
 };
 
@@ -415,19 +415,20 @@ __device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const f
       const float *xs = p.xm + (size_t)l * p.xm_ls + (size_t)tok * p.N + n0;
       float *adst = p.c + (size_t)l * p.out_ls + (size_t)tok * p.N + n0;
       __nv_bfloat16 *udst = p.z + (size_t)l * p.out_ls + (size_t)tok * p.N + n0;
-      float ss = 0.f;
+      // one partial sum of u^2 per 128 columns, so that 128- and 256-wide tiles leave the same numbers behind
 #pragma unroll
-      for (int j = 0; j < BN / 32; ++j) {
-        const float a = y[lane + 32 * j];
-        const float u = fmaf(kappa, a, xs[lane + 32 * j]);
-        adst[lane + 32 * j] = a;
-        udst[lane + 32 * j] = __float2bfloat16_rn(u);
-        ss = fmaf(u, u, ss);
-      }
-      ss = warp_sum(ss);
-      if (lane == 0) {  // two partials per tile, as in the prefill regime (the second is zero here)
-        p.ssq_out[(((size_t)l * p.Nt + n_tile) * 2) * p.M + tok] = ss;
-        p.ssq_out[(((size_t)l * p.Nt + n_tile) * 2 + 1) * p.M + tok] = 0.f;
+      for (int h = 0; h < BN / 128; ++h) {
+        float ss = 0.f;
+#pragma unroll
+        for (int j = 4 * h; j < 4 * h + 4; ++j) {
+          const float a = y[lane + 32 * j];
+          const float u = fmaf(kappa, a, xs[lane + 32 * j]);
+          adst[lane + 32 * j] = a;
+          udst[lane + 32 * j] = __float2bfloat16_rn(u);
+          ss = fmaf(u, u, ss);
+        }
+        ss = warp_sum(ss);
+        if (lane == 0) p.ssq_out[((size_t)l * p.Nt * (BN / 128) + n_tile * (BN / 128) + h) * p.M + tok] = ss;
       }
     } else if (EPI == UEPI_QKV) {
       const int b = tok / p.T, pos = *p.pos_base + (tok % p.T);
