@@ -22,6 +22,10 @@ CASES = {
     "bf16_decode_hc4": (synth.ModelConfig(3, 256, 2, 128, 512, 1024, 4, "bf16"), 3, 4),    # decode-regime + mHC
     "bf16_prefill": (synth.ModelConfig(2, 256, 2, 128, 512, 1024, 1, "bf16"), 2, 150),     # prefill-regime, ragged M = 300
     "bf16_prefill_hc4": (synth.ModelConfig(2, 256, 2, 128, 512, 1024, 4, "bf16"), 1, 130),
+    # widths that are multiples of 128 but not of 256 (the paper's d = 640 is one): 128-wide weight tiles in every
+    # projection, an odd number of heads
+    "bf16_decode_d384": (synth.ModelConfig(3, 384, 3, 128, 896, 1152, 1, "bf16"), 2, 6),
+    "bf16_prefill_d384": (synth.ModelConfig(2, 384, 3, 128, 896, 1152, 1, "bf16"), 1, 200),
 }
 
 
@@ -70,7 +74,8 @@ def test_parallel_sweeps_match_oracle(name):
     m.device_status()
 
 
-@pytest.mark.parametrize("name", ["tiny", "f32_hc4", "bf16_decode_nt2", "bf16_decode_hc4", "bf16_generic", "bf16_prefill"])
+@pytest.mark.parametrize("name", ["tiny", "f32_hc4", "bf16_decode_nt2", "bf16_decode_hc4", "bf16_generic", "bf16_prefill", "bf16_decode_d384",
+                                  "bf16_prefill_d384"])
 def test_K_equal_L_reproduces_the_librarys_sequential_trace_bitwise(name):
     """Finite-step exactness on the GPU: the correction adds (h + a) + m in layer order, so after L
     sweeps the trace is bit-identical to the library's own sequential forward."""
