@@ -186,14 +186,10 @@ def run_ours(args):
         host_in = torch.empty((1,), dtype=torch.int32).pin_memory()
         host_out = torch.empty((1,), dtype=torch.int32).pin_memory()
         host_in.copy_(first.cpu())
-        dev_tok = torch.empty((1,), dtype=torch.int32, device="cuda")
         e2e_steps = min(steps, 128)
 
-        def e2e_step():
-            dev_tok.copy_(host_in, non_blocking=True)
-            model.decode_step(kv, dev_tok, K_MAIN, snlp.MODE_IDN, tok_out=dev_tok)
-            host_out.copy_(dev_tok, non_blocking=True)
-            stream.synchronize()
+        def e2e_step():   # the C-ABI call with host buffers: token in, the step, next token out, stream sync
+            model.decode_step_host(kv, host_in, K_MAIN, snlp.MODE_IDN, tok_out=host_out)
             host_in.copy_(host_out)
 
         for _ in range(warmup):
@@ -271,7 +267,7 @@ def run_ours(args):
                    "l2": "no flush: each step streams 2.2 GB of weights + KV (> 126 MB L2)"},
         "clocks": clocks,
         "e2e": {"value": world * 1e3 / ms_e2e, "unit": "tokens/s", "h2d_bytes_per_step": 4, "d2h_bytes_per_step": 4,
-                "steps": e2e_steps, "note": "host token in pinned memory -> H2D, snlp_decode_step, D2H, stream sync, every step"},
+                "steps": e2e_steps, "note": "snlp_decode_step_host every step: host token -> pinned staging, read across the bus by the step's first kernel; next token written back by its last kernel; stream sync"},
         "gpu_launches": launches_timed,
         "roofline": {"bound": "hbm", "kernel": f"k_umma_gemm<BN=256, AM=16> ({dom} projection, all 20 layers in one launch)", "achieved": achieved,
                      "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak, "peak_source": peak_src,

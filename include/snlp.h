@@ -178,6 +178,13 @@ int snlp_prefill(snlp_model *m, snlp_kv *kv, const int32_t *ids, int B, int T, i
 int snlp_decode_step(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, int K, int mode, int32_t *tok_out,
                      float *resnorm_out, void *stream);
 
+/* snlp_decode_step for a caller that keeps its tokens on the host: tok_in_host and tok_out_host are HOST int32 [B]
+ * (pageable or pinned; they may alias).  The tokens go through the library's own mapped pinned staging buffer, which
+ * the step's kernels read and write across the bus; the call synchronises `stream` before returning, so tok_out_host
+ * is valid on return.  Errors as snlp_decode_step, plus CUDA. */
+int snlp_decode_step_host(snlp_model *m, snlp_kv *kv, const int32_t *tok_in_host, int K, int mode, int32_t *tok_out_host,
+                          void *stream);
+
 /* One round of greedy self-speculative decoding (Sec. 5.1), batch 1: the SNLP(K, mode) drafter proposes
  * `block` tokens x_1..x_block from *last_tok by decode steps; one sequential forward over
  * [last_tok, x_1..x_block] (block+1 rows) verifies them and overwrites the drafter's cache entries;

@@ -95,6 +95,7 @@ struct snlp_model {
   unsigned *counter = nullptr, *attn_counters = nullptr;
   int *zero = nullptr;
   int32_t *spec = nullptr;  // [2 * (max_rows + 1)] ids / verifier tokens for draft-and-verify
+  int32_t *tok_pin = nullptr, *tok_dev = nullptr;   // [2][max_batch] mapped pinned host memory (tokens in, tokens out) and its device address (snlp_decode_step_host)
   int logit_rows = 0;
   std::vector<void *> allocs;
   // flags / stats
@@ -281,6 +282,11 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
   A(&m->attn_counters, L * (size_t)kDecodeRows * c.n_head * 4);
   A(&m->zero, 16);
   A(&m->spec, 2 * (R + 1) * 4);
+  if (rc == SNLP_OK && (cudaHostAlloc((void **)&m->tok_pin, (size_t)2 * c.max_batch * 4, cudaHostAllocMapped) != cudaSuccess ||
+                        cudaHostGetDevicePointer((void **)&m->tok_dev, m->tok_pin, 0) != cudaSuccess)) {
+    cudaGetLastError();
+    rc = fail(SNLP_ERR_OOM, "cudaHostAlloc of the token staging buffer failed");
+  }
   if (rc == SNLP_OK) {
     if (cudaMemset(m->dev_err, 0, 16) != cudaSuccess || cudaMemset(m->attn_counters, 0, L * (size_t)kDecodeRows * c.n_head * 4) != cudaSuccess || cudaMemset(m->counter, 0, 16) != cudaSuccess || cudaMemset(m->zero, 0, 16) != cudaSuccess)
       rc = fail(SNLP_ERR_CUDA, "cudaMemset failed");
@@ -318,6 +324,7 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
     rc = fail(SNLP_ERR_CUDA, "cudaStreamCreateWithFlags failed");
   if (rc != SNLP_OK) {
     for (void *p : m->allocs) cudaFree(p);
+    if (m->tok_pin) cudaFreeHost(m->tok_pin);
     delete m;
     return rc;
   }
@@ -334,6 +341,7 @@ extern "C" int snlp_destroy(snlp_model *m) {
   for (const PendingTime &t : m->pending) { cudaEventDestroy(t.e0); cudaEventDestroy(t.e1); }
   for (cudaEvent_t e : m->free_events) cudaEventDestroy(e);
   for (void *p : m->allocs) cudaFree(p);
+  if (m->tok_pin) cudaFreeHost(m->tok_pin);
   delete m;
   return SNLP_OK;
 }
@@ -1193,6 +1201,20 @@ extern "C" int snlp_decode_step(snlp_model *m, snlp_kv *kv, const int32_t *tok_i
   if (kv->len + 1 > kv->max_ctx) return fail(SNLP_ERR_SHAPE, "snlp_decode_step: cache is full (len %d, max_ctx %d)", kv->len, kv->max_ctx);
   const snlp_solver sol = K == 0 ? snlp_solver{0, SNLP_MODE_SEQUENTIAL, m->cfg.n_layer, SNLP_INIT_H0, 1} : snlp_solver{K, mode, 0, SNLP_INIT_H0, 1};
   return decode_step_impl(m, kv, tok_in, sol, tok_out, K > 0 ? resnorm_out : nullptr, (cudaStream_t)stream);
+}
+
+extern "C" int snlp_decode_step_host(snlp_model *m, snlp_kv *kv, const int32_t *tok_in_host, int K, int mode, int32_t *tok_out_host, void *stream) {
+  TRY(check_model(m, "snlp_decode_step_host"));
+  if (!kv || !tok_in_host || !tok_out_host) return fail(SNLP_ERR_ARG, "snlp_decode_step_host: NULL pointer");
+  if (kv->m != m) return fail(SNLP_ERR_ARG, "snlp_decode_step_host: cache belongs to another model");
+  // The step's kernels read the tokens from, and write the next ones to, mapped pinned host memory: the embedding
+  // gather fetches B ids across the bus and the arg-max kernel posts B ids back, with no copy operations around the graph.
+  const size_t bytes = (size_t)kv->B * sizeof(int32_t);
+  memcpy(m->tok_pin, tok_in_host, bytes);
+  TRY(snlp_decode_step(m, kv, m->tok_dev, K, mode, m->tok_dev + m->cfg.max_batch, nullptr, stream));
+  CU(cudaStreamSynchronize((cudaStream_t)stream));
+  memcpy(tok_out_host, m->tok_pin + m->cfg.max_batch, bytes);
+  return SNLP_OK;
 }
 
 extern "C" int snlp_decode_step_solver(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, const snlp_solver *solver, int32_t *tok_out,

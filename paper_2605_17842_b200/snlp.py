@@ -23,7 +23,7 @@ INIT_H0, INIT_FWD = 0, 1
 EXPORTS = [
     "snlp_create", "snlp_destroy", "snlp_load_weights", "snlp_embed", "snlp_forward_sequential",
     "snlp_forward_parallel", "snlp_forward_solver", "snlp_decode_step_solver", "snlp_lm_head", "snlp_kv_create", "snlp_kv_destroy", "snlp_kv_len",
-    "snlp_kv_truncate", "snlp_prefill", "snlp_decode_step", "snlp_draft_and_verify", "snlp_set_flag",
+    "snlp_kv_truncate", "snlp_prefill", "snlp_decode_step", "snlp_decode_step_host", "snlp_draft_and_verify", "snlp_set_flag",
     "snlp_launch_count", "snlp_kernel_times", "snlp_device_status", "snlp_lm_head_greedy_static", "snlp_last_error",
 ]
 
@@ -217,6 +217,15 @@ class Model:
             tok_out = torch.empty_like(tok_in)
         _check(_lib.snlp_decode_step(self._h, kv._h, _ptr(tok_in), C.c_int(K), C.c_int(mode), _ptr(tok_out),
                                      _ptr(resnorm), _stream()))
+        return tok_out
+
+    def decode_step_host(self, kv: KVCache, tok_in, K: int, mode: int = MODE_IDN, tok_out=None):
+        """decode_step on HOST int32 tensors (CPU, pinned or not): copies in, step, copies out, synchronises."""
+        if tok_out is None:
+            tok_out = torch.empty_like(tok_in)
+        assert tok_in.device.type == "cpu" and tok_out.device.type == "cpu" and tok_in.dtype == torch.int32 and tok_out.dtype == torch.int32
+        _check(_lib.snlp_decode_step_host(self._h, kv._h, C.c_void_p(tok_in.data_ptr()), C.c_int(K), C.c_int(mode),
+                                          C.c_void_p(tok_out.data_ptr()), _stream()))
         return tok_out
 
     def draft_and_verify(self, kv: KVCache, last_tok: torch.Tensor, block: int, K: int, mode: int = MODE_IDN):

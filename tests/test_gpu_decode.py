@@ -210,3 +210,34 @@ def test_kv_truncate_rewinds_decoding():
     b = [m.decode_step(kv, t0, 0).clone()]
     b.append(m.decode_step(kv, b[-1], 0).clone())
     assert torch.equal(torch.stack(a), torch.stack(b))
+
+
+@pytest.mark.parametrize("cfg,B", [(F32, 1), (BF16, 2)])
+def test_decode_through_host_buffers_gives_the_same_tokens(cfg, B):
+    """snlp_decode_step_host (tokens in host memory, copies and synchronisation inside the call) against the
+    device-pointer entry point, token for token; pageable and pinned host tensors."""
+    W = weights(cfg)
+    m = make_model(cfg, W, max_rows=8 * B, max_batch=B, max_ctx=32)
+    ids = dev(synth.make_ids(cfg, B, 8, seed=10))
+    kv = m.kv_cache(B, 32)
+    t0 = m.prefill(kv, ids)
+    want, t = [], t0
+    for _ in range(6):
+        t = m.decode_step(kv, t, 2)
+        want.append(t.cpu())
+    kv.truncate(8)
+    got, th = [], t0.cpu()
+    out_pinned = torch.empty_like(th).pin_memory()
+    for i in range(6):
+        th = m.decode_step_host(kv, th, 2, tok_out=out_pinned if i % 2 else None).clone()   # in/out may also alias (below)
+        got.append(th)
+    assert all(torch.equal(a, b) for a, b in zip(want, got))
+    assert len(kv) == 14
+    kv.truncate(8)
+    th = t0.cpu().clone()
+    m.decode_step_host(kv, th, 2, tok_out=th)
+    assert torch.equal(th, want[0])
+    from paper_2605_17842_b200 import snlp
+    with pytest.raises(snlp.SnlpError) as e:
+        m.decode_step_host(kv, th, -1)
+    assert e.value.code == snlp.ERR_ARG
