@@ -181,7 +181,8 @@ int snlp_decode_step(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, int K, i
 /* snlp_decode_step for a caller that keeps its tokens on the host: tok_in_host and tok_out_host are HOST int32 [B]
  * (pageable or pinned; they may alias).  The tokens go through the library's own mapped pinned staging buffer, which
  * the step's kernels read and write across the bus; the call synchronises `stream` before returning, so tok_out_host
- * is valid on return.  Errors as snlp_decode_step, plus CUDA. */
+ * is valid on return.  One staging buffer per model: calls on the same model must not overlap.  Errors as
+ * snlp_decode_step, plus CUDA. */
 int snlp_decode_step_host(snlp_model *m, snlp_kv *kv, const int32_t *tok_in_host, int K, int mode, int32_t *tok_out_host,
                           void *stream);
 
