@@ -94,6 +94,7 @@ struct snlp_model {
   int *pm_idx = nullptr;
   unsigned *counter = nullptr, *attn_counters = nullptr;
   int *zero = nullptr;
+  unsigned *lm_counter = nullptr;   // arrival counter of the LM-head launch (zero between launches)
   int32_t *spec = nullptr;  // [2 * (max_rows + 1)] ids / verifier tokens for draft-and-verify
   int32_t *tok_pin = nullptr, *tok_dev = nullptr;   // [2][max_batch] mapped pinned host memory (tokens in, tokens out) and its device address (snlp_decode_step_host)
   int logit_rows = 0;
@@ -114,7 +115,6 @@ struct snlp_model {
   int n_sm = 148;
   EncodeTiledFn encode_tiled = nullptr;  // cuTensorMapEncodeTiled, looked up through the runtime
   int *dev_err = nullptr;                // raised by a kernel whose bounded wait expired
-  int lm_tiles = 0;                   // column tiles of the last LM-head launch (its arg-max partials)
   cudaStream_t cap_stream = nullptr;  // capture target: graphs are recorded here and replayed on the caller's stream
 };
 
@@ -281,6 +281,7 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
   A(&m->dev_err, 16);
   A(&m->attn_counters, L * (size_t)kDecodeRows * c.n_head * 4);
   A(&m->zero, 16);
+  A(&m->lm_counter, 16);
   A(&m->spec, 2 * (R + 1) * 4);
   if (rc == SNLP_OK && (cudaHostAlloc((void **)&m->tok_pin, (size_t)2 * c.max_batch * 4, cudaHostAllocMapped) != cudaSuccess ||
                         cudaHostGetDevicePointer((void **)&m->tok_dev, m->tok_pin, 0) != cudaSuccess)) {
@@ -288,7 +289,7 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
     rc = fail(SNLP_ERR_OOM, "cudaHostAlloc of the token staging buffer failed");
   }
   if (rc == SNLP_OK) {
-    if (cudaMemset(m->dev_err, 0, 16) != cudaSuccess || cudaMemset(m->attn_counters, 0, L * (size_t)kDecodeRows * c.n_head * 4) != cudaSuccess || cudaMemset(m->counter, 0, 16) != cudaSuccess || cudaMemset(m->zero, 0, 16) != cudaSuccess)
+    if (cudaMemset(m->dev_err, 0, 16) != cudaSuccess || cudaMemset(m->attn_counters, 0, L * (size_t)kDecodeRows * c.n_head * 4) != cudaSuccess || cudaMemset(m->counter, 0, 16) != cudaSuccess || cudaMemset(m->zero, 0, 16) != cudaSuccess || cudaMemset(m->lm_counter, 0, 16) != cudaSuccess)
       rc = fail(SNLP_ERR_CUDA, "cudaMemset failed");
   }
   if (rc == SNLP_OK) {
@@ -627,7 +628,6 @@ static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat1
   if (small && w.BN == 256 && (N / 128) * ksplit * nl <= m->n_sm) bn = 128;
   const CUtensorMap &tmw = bn == w.BN ? w.tm : w.tm_half;
   p.Nt = N / bn;
-  if (EPI == UEPI_LMHEAD) m->lm_tiles = p.Nt;
   const int items = p.Mt * p.Nt * ksplit * nl;
   const int grid = items < m->n_sm ? items : m->n_sm;
 #define SNLP_UMMA_LAUNCH(BN_, AM_)                                                                                                   \
@@ -901,9 +901,9 @@ static int lm_head_impl(snlp_model *m, cudaStream_t st, const float *hL, size_t 
     UmmaParams p{};
     p.ssq = pre_ssq; p.nparts = P; p.eps = c.rms_eps;
     p.logits = logits; p.pm_val = m->pm_val; p.pm_idx = m->pm_idx;
+    p.argmax = argmax; p.bump = argmax ? bump : nullptr; p.lm_counter = m->lm_counter;   // the last CTA merges the tiles' maxima
     TRY(umma_gemm<UEPI_LMHEAD>(m, st, KC_LMHEAD, pre_xb, 0, m->w_lm, 0, p, rows, V, d, 1, 1));
-    if (argmax) KLAUNCH(m, st, KC_LMHEAD, k_argmax_tiles<<<rows, 256, 0, st>>>(m->pm_val, m->pm_idx, m->lm_tiles, argmax, bump));
-    else if (bump) KLAUNCH(m, st, KC_OTHER, k_add_int<<<1, 1, 0, st>>>(bump, 1));
+    if (!argmax && bump) KLAUNCH(m, st, KC_OTHER, k_add_int<<<1, 1, 0, st>>>(bump, 1));
     return SNLP_OK;
   }
   for (int r0 = 0; r0 < rows; r0 += m->logit_rows) {
@@ -1128,7 +1128,7 @@ extern "C" int snlp_prefill(snlp_model *m, snlp_kv *kv, const int32_t *ids, int 
 }
 
 // greedy tokens of all `rows` rows of the forward that just ran (rows <= 16)
-// bump (nullable): device counter to advance by one after the tokens are out (fused into the arg-max kernel where there is one)
+// bump (nullable): device counter to advance by one after the tokens are out (done by the LM-head kernel itself on the tensor-core path)
 static int lm_head_tail(snlp_model *m, cudaStream_t st, int rows, int32_t *argmax, int *bump = nullptr) {
   const snlp_config &c = m->cfg;
   const size_t nd = (size_t)c.n_streams * c.d_model, L = c.n_layer;
@@ -1208,7 +1208,7 @@ extern "C" int snlp_decode_step_host(snlp_model *m, snlp_kv *kv, const int32_t *
   if (!kv || !tok_in_host || !tok_out_host) return fail(SNLP_ERR_ARG, "snlp_decode_step_host: NULL pointer");
   if (kv->m != m) return fail(SNLP_ERR_ARG, "snlp_decode_step_host: cache belongs to another model");
   // The step's kernels read the tokens from, and write the next ones to, mapped pinned host memory: the embedding
-  // gather fetches B ids across the bus and the arg-max kernel posts B ids back, with no copy operations around the graph.
+  // gather fetches B ids across the bus and the LM-head kernel posts B ids back, with no copy operations around the graph.
   const size_t bytes = (size_t)kv->B * sizeof(int32_t);
   memcpy(m->tok_pin, tok_in_host, bytes);
   TRY(snlp_decode_step(m, kv, m->tok_dev, K, mode, m->tok_dev + m->cfg.max_batch, nullptr, stream));

@@ -55,6 +55,9 @@ struct UmmaParams {
   const float2 *rope_t; int rope_ld;  // rope transposed [hd/2][rope_ld], read by the prefill-regime epilogue (thread = row)
   const float *xm; size_t xm_ls; const HcCoef *coef; float *ssq_out;   // UEPI_RESID; ssq_out [nl][partials][M]
   float *logits; float *pm_val; int *pm_idx;                            // UEPI_LMHEAD
+  // UEPI_LMHEAD, optional: the CTA that finishes last merges the per-tile maxima into argmax[M] (ties -> lowest
+  // index) and then adds one to *bump (nullable).  lm_counter: zero on entry, left zero.
+  int32_t *argmax; int *bump; unsigned *lm_counter;
 };
 
 constexpr int kUmmaThreads = 320;   // warp 0: TMA, warp 1: MMA + TMEM allocation, warps 2-9: epilogue (two per TMEM lane quarter)
@@ -627,6 +630,38 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
         if (et == 0) mbar_arrive(&accempty[b]);
         umma_epilogue_small<BN, EPI>(p, outs, ew, lane, n_tile, ks, l, la);
         epi_bar_sync();  // outs is reused by the next item
+      }
+    }
+    if (EPI == UEPI_LMHEAD && AM != kUmmaBM && p.argmax != nullptr) {
+      // Greedy token: every CTA counts itself in once its partial maxima are out (also after a wait that ran out,
+      // so that the counter always returns to zero); the last one merges the tiles.
+      int *s_last = reinterpret_cast<int *>(outs);
+      __threadfence();
+      epi_bar_sync();
+      if (et == 0) *s_last = atomicAdd(p.lm_counter, 1u) == gridDim.x - 1 ? 1 : 0;
+      epi_bar_sync();
+      if (*s_last) {
+        __threadfence();
+        for (int tok = ew; tok < p.M; tok += 8) {
+          float bv = -INFINITY;
+          int bi = 0x7fffffff;
+          for (int j = lane; j < p.Nt; j += 32) {
+            const float v = __ldcg(&p.pm_val[(size_t)tok * p.Nt + j]);
+            const int ix = __ldcg(&p.pm_idx[(size_t)tok * p.Nt + j]);
+            if (v > bv || (v == bv && ix < bi)) { bv = v; bi = ix; }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+          }
+          if (lane == 0) p.argmax[tok] = (unsigned)bi < (unsigned)p.N ? bi : 0;
+        }
+        if (et == 0) {
+          if (p.bump != nullptr) *p.bump += 1;
+          *p.lm_counter = 0u;
+        }
       }
     }
   }
