@@ -75,6 +75,8 @@ __device__ __forceinline__ float f4_sq(float4 a) { return fmaf(a.w, a.w, fmaf(a.
 
 // Depth of the operand ring of k_correct (steps in flight per thread) and its shared-memory size.
 __host__ __device__ constexpr int corr_depth(int ns) { return ns <= 1 ? 4 : (ns <= 4 ? 3 : 2); }
+// floats per step of the staged mixing coefficients (A, c^a, c^m, next pre-maps), rounded up to whole float4
+__host__ __device__ constexpr int corr_coef_stride(int ns) { return (ns * (ns + 4) + 3) / 4 * 4; }
 __host__ __device__ constexpr size_t corr_ring_bytes(int ns, int threads) { return (size_t)corr_depth(ns) * (2 + ns) * threads * sizeof(float4); }
 
 // NS = number of residual streams (compile time so the per-thread state stays in registers).
@@ -82,13 +84,13 @@ __host__ __device__ constexpr size_t corr_ring_bytes(int ns, int threads) { retu
 // operands of the next corr_depth(NS)-1 steps are kept in flight with cp.async into a per-thread ring in shared memory
 // (a thread only ever reads its own slots, so no block barrier is involved).  With K-split branch outputs (a_splits or
 // m_splits > 1) the operands are summed from global memory directly, one step ahead.
-// Dynamic shared memory: corr_ring_bytes(NS, blockDim.x) + [warps][nl][2] floats.
+// Dynamic shared memory: corr_ring_bytes(NS, blockDim.x) + [warps][nl][2] floats (with norms) + [nl][corr_coef_stride(NS)] floats (NS > 1).
 // NATIVE: the surrogate is the block's own affine map (IDN on a single stream, HCN on n streams), known at compile time.
 template <int NS, bool NATIVE>
 __global__ void __launch_bounds__(256, NS == 1 ? 4 : 2) k_correct(CorrParams p) {
   extern __shared__ float4 s_ring[];  // [depth][2 + NS][blockDim.x]
   constexpr int D = corr_depth(NS);
-  float *s_norm = reinterpret_cast<float *>(s_ring + (size_t)D * (2 + NS) * blockDim.x);  // [warps][nl][2]
+  float *s_norm = reinterpret_cast<float *>(s_ring + (size_t)D * (2 + NS) * blockDim.x);  // [warps][nl][2] (only with norms)
   const int d4 = p.d >> 2;
   const size_t total = (size_t)p.M * d4;
   const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -107,6 +109,25 @@ __global__ void __launch_bounds__(256, NS == 1 ? 4 : 2) k_correct(CorrParams p) 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
   const bool ring = p.a_splits == 1 && p.m_splits == 1;
   const bool need_old = (want_norm || !native) && !p.implicit_old;   // the old next state enters only the residual norm and the surrogate forms
+  // Mixing coefficients of every step in shared memory, [nl][kCoefStride]: A, c^a, c^m of the step's layer, then the
+  // pre-maps of the layer after it (zero past the last layer).  Read back as broadcast vector loads: per step a
+  // thread would otherwise issue one global load per coefficient.
+  constexpr int kCoefStride = corr_coef_stride(NS);
+  float *s_coef = s_norm + (want_norm ? (size_t)nwarp * p.nl * 2 : 0);
+  if (NS > 1) {
+    for (int idx = threadIdx.x; idx < p.nl * kCoefStride; idx += blockDim.x) {
+      const int i = idx / kCoefStride, j = idx % kCoefStride;
+      const int l = p.l0 + i * p.lstep, ln = l + p.lstep;
+      float v = 0.f;
+      if (j < NS * NS) v = p.coef[l].A[j];
+      else if (j < NS * NS + NS) v = p.coef[l].ca[j - NS * NS];
+      else if (j < NS * NS + 2 * NS) v = p.coef[l].cm[j - NS * NS - NS];
+      else if (j < NS * NS + 3 * NS) v = ln < p.L ? p.coef[ln].pa[j - NS * NS - 2 * NS] : 0.f;
+      else if (j < NS * NS + 4 * NS) v = ln < p.L ? p.coef[ln].pmra[j - NS * NS - 3 * NS] : 0.f;
+      s_coef[idx] = v;
+    }
+    __syncthreads();
+  }
 
   float4 oldp[NS], newp[NS];
   // operands of one step: branch outputs and the old next state
@@ -157,17 +178,32 @@ __global__ void __launch_bounds__(256, NS == 1 ? 4 : 2) k_correct(CorrParams p) 
     }
     if (active) {
       const float4 av = av_n, mv = mv_n;
-      // this layer's coefficients into registers once (read through the non-coherent path: a reference into global
-      // memory would have to be re-read after every store of the step, which may alias it for all the compiler knows)
-      const HcCoef *cp = p.coef + l;
-      float cA[NS * NS], cca[NS], ccm[NS];
+      // this step's coefficients into registers once
+      float cA[NS * NS], cca[NS], ccm[NS], cpa[NS], cpm[NS];
       if (NS > 1) {
+        const float *sc = s_coef + (size_t)i * kCoefStride;
+        if (NS % 4 == 0) {
+          const float4 *sc4 = reinterpret_cast<const float4 *>(sc);
 #pragma unroll
-        for (int r = 0; r < NS; ++r) {
+          for (int k = 0; k < NS * NS / 4; ++k) { const float4 t = sc4[k]; cA[4 * k] = t.x; cA[4 * k + 1] = t.y; cA[4 * k + 2] = t.z; cA[4 * k + 3] = t.w; }
 #pragma unroll
-          for (int s = 0; s < NS; ++s) cA[r * NS + s] = __ldg(&cp->A[r * NS + s]);
-          cca[r] = __ldg(&cp->ca[r]);
-          ccm[r] = __ldg(&cp->cm[r]);
+          for (int k = 0; k < NS / 4; ++k) {
+            const float4 t0 = sc4[NS * NS / 4 + k], t1 = sc4[NS * NS / 4 + NS / 4 + k], t2 = sc4[NS * NS / 4 + 2 * (NS / 4) + k], t3 = sc4[NS * NS / 4 + 3 * (NS / 4) + k];
+            cca[4 * k] = t0.x; cca[4 * k + 1] = t0.y; cca[4 * k + 2] = t0.z; cca[4 * k + 3] = t0.w;
+            ccm[4 * k] = t1.x; ccm[4 * k + 1] = t1.y; ccm[4 * k + 2] = t1.z; ccm[4 * k + 3] = t1.w;
+            cpa[4 * k] = t2.x; cpa[4 * k + 1] = t2.y; cpa[4 * k + 2] = t2.z; cpa[4 * k + 3] = t2.w;
+            cpm[4 * k] = t3.x; cpm[4 * k + 1] = t3.y; cpm[4 * k + 2] = t3.z; cpm[4 * k + 3] = t3.w;
+          }
+        } else {
+#pragma unroll
+          for (int k = 0; k < NS * NS; ++k) cA[k] = sc[k];
+#pragma unroll
+          for (int k = 0; k < NS; ++k) {
+            cca[k] = sc[NS * NS + k];
+            ccm[k] = sc[NS * NS + NS + k];
+            cpa[k] = sc[NS * NS + 2 * NS + k];
+            cpm[k] = sc[NS * NS + 3 * NS + k];
+          }
         }
       }
       float4 oldn[NS], newn[NS], tilde[NS];
@@ -208,12 +244,11 @@ __global__ void __launch_bounds__(256, NS == 1 ? 4 : 2) k_correct(CorrParams p) 
       }
       float4 nxt = newn[0];  // the next layer's attention-branch input
       if (NS > 1 && ln < p.L && !p.skip_next) {
-        const HcCoef *cn = p.coef + ln;
-        float4 sa = f4_scale(__ldg(&cn->pa[0]), newn[0]), sm = f4_scale(__ldg(&cn->pmra[0]), newn[0]);
+        float4 sa = f4_scale(cpa[0], newn[0]), sm = f4_scale(cpm[0], newn[0]);
 #pragma unroll
         for (int s = 1; s < NS; ++s) {
-          sa = f4_fma(__ldg(&cn->pa[s]), newn[s], sa);
-          sm = f4_fma(__ldg(&cn->pmra[s]), newn[s], sm);
+          sa = f4_fma(cpa[s], newn[s], sa);
+          sm = f4_fma(cpm[s], newn[s], sm);
         }
         if (p.xa != nullptr) reinterpret_cast<float4 *>(p.xa)[(size_t)ln * Md4 + bm_off] = sa;
         reinterpret_cast<float4 *>(p.xm)[(size_t)ln * Md4 + bm_off] = sm;
@@ -238,9 +273,16 @@ __global__ void __launch_bounds__(256, NS == 1 ? 4 : 2) k_correct(CorrParams p) 
       if (lane == 0 && active) p.ssq_x[((size_t)ln * (d4 >> 5) + (c4 >> 5)) * p.M + row] = xs;
     }
     if (want_norm) {
-      rs = warp_sum(rs);
-      hs = warp_sum(hs);
-      if (lane == 0) { s_norm[(warp * p.nl + i) * 2] = rs; s_norm[(warp * p.nl + i) * 2 + 1] = hs; }
+      // both sums in one butterfly: the upper half-warp hands its residual part to the lower one and takes the
+      // state part in return, then each half reduces one quantity (lane 0: sum r^2, lane 16: sum h^2)
+      const bool up = (lane & 16) != 0;
+      float keep = up ? hs : rs;
+      keep += __shfl_xor_sync(0xffffffffu, up ? rs : hs, 16);
+      keep += __shfl_xor_sync(0xffffffffu, keep, 8);
+      keep += __shfl_xor_sync(0xffffffffu, keep, 4);
+      keep += __shfl_xor_sync(0xffffffffu, keep, 2);
+      keep += __shfl_xor_sync(0xffffffffu, keep, 1);
+      if ((lane & 15) == 0) s_norm[(warp * p.nl + i) * 2 + (up ? 1 : 0)] = keep;
     }
   }
   if (!want_norm) return;

@@ -56,6 +56,7 @@ void set_last_error(const char *msg) { g_err = msg; }  // for the library's othe
 
 // ------------------------------------------------------------------------------------------------
 // handles
+constexpr size_t kCorrExtraSmem = 32768;   // k_correct: shared memory beyond the operand ring (norm partials, staged coefficients)
 constexpr int kMaxSplits = 4;    // K-splits of the partial-sum GEMV outputs
 constexpr int kDecodeRows = 16;  // largest row count served by the decode-regime kernels
 constexpr size_t kCorrSmallSmem = 160 * 1024;
@@ -503,8 +504,9 @@ static int correct(snlp_model *m, const Fwd &f, int l0, int nsteps, int lstep, i
   const size_t total = (size_t)f.M * (c.d_model / 4);
   const int threads = 256;
   const unsigned blocks = (unsigned)((total + threads - 1) / threads);
-  const size_t sm = corr_ring_bytes(c.n_streams, threads) + (resnorm ? (size_t)(threads / 32) * nl * 2 * sizeof(float) : 0);
-  if (sm > corr_ring_bytes(c.n_streams, threads) + 16384) return fail(SNLP_ERR_UNSUPPORTED, "correction: more than 256 layers in one range");
+  const size_t sm = corr_ring_bytes(c.n_streams, threads) + (resnorm ? (size_t)(threads / 32) * nl * 2 * sizeof(float) : 0) +
+                    (c.n_streams > 1 ? (size_t)nl * corr_coef_stride(c.n_streams) * sizeof(float) : 0);
+  if (sm > corr_ring_bytes(c.n_streams, threads) + kCorrExtraSmem) return fail(SNLP_ERR_UNSUPPORTED, "correction: too many layers in one range");
   const size_t sm_small = (size_t)nl * 32 * (2 + c.n_streams) * sizeof(float4) + (size_t)nl * 2 * sizeof(float) + (size_t)nl * 3 * 32 * sizeof(float);
   if (f.M <= kDecodeRows && c.n_streams <= 4 && sm_small <= kCorrSmallSmem) {
     dim3 grid((c.d_model / 4 + 31) / 32, f.M);
@@ -746,8 +748,8 @@ static int init_kernel_attributes() {
   CU((umma_attr<128, 16, UEPI_LMHEAD>()));
   CU((umma_attr<256, 16, UEPI_LMHEAD>()));
   CU(cudaFuncSetAttribute(k_attn_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, kFuSmem));
-#define ATTR(NS) CU(cudaFuncSetAttribute(k_correct<NS, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(corr_ring_bytes(NS, 256) + 16384))); \
-  CU(cudaFuncSetAttribute(k_correct<NS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(corr_ring_bytes(NS, 256) + 16384)));
+#define ATTR(NS) CU(cudaFuncSetAttribute(k_correct<NS, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(corr_ring_bytes(NS, 256) + kCorrExtraSmem))); \
+  CU(cudaFuncSetAttribute(k_correct<NS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(corr_ring_bytes(NS, 256) + kCorrExtraSmem)));
   ATTR(1) ATTR(2) ATTR(3) ATTR(4) ATTR(5) ATTR(6) ATTR(7) ATTR(8)
 #undef ATTR
   CU(cudaFuncSetAttribute(k_correct_small<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCorrSmallSmem));
