@@ -420,11 +420,10 @@ def run_prefill_workload(args, name):
             if k in flops:
                 classes[k]["TFLOPs"] = flops[k] / (ms / nrep * 1e-3) / 1e12
                 classes[k]["frac_of_bf16_peak"] = classes[k]["TFLOPs"] / burst
-    # the correction is HBM-bound: new states written, a and m read, bf16 inputs (and the mHC MLP pre-map) written; the
-    # sweep timed here is the first one after initialisation, which does not read old states (they all equal h_0); later
-    # sweeps read them too (n * 4 more bytes per element)
+    # the correction timed here is that of a K = 1 forward: the first sweep after initialisation (old states all equal h_0:
+    # not read) and at the same time the last one (no operands for a next sweep): it reads a and m and writes the new states
     n = cfg.n_streams
-    corr_bytes = L * M * d * (n * 4 + 2 * 4 + 2 + (4 if n > 1 else 0))
+    corr_bytes = L * M * d * (n * 4 + 2 * 4)
     if "correction" in classes:
         hbm = peaks()[0]
         classes["correction"]["alg_GBs"] = corr_bytes / (classes["correction"]["ms_per_sweep"] * 1e-3) / 1e9
