@@ -153,3 +153,36 @@ class NaiveModel:
                 new.append(nxt)
             old = new
         return old
+
+    # ---- model entry and exit (Alg. 1 lines 1 and 5) ---------------------------
+    def embed(self, ids):
+        """ids: list of T token ids -> list[t][s][j]; the embedding row goes into every stream."""
+        c = self.cfg
+        out = []
+        for tok in ids:
+            row = [float(self.W.embed[tok][j]) for j in range(c.d_model)]
+            out.append([list(row) for _ in range(c.n_streams)])
+        return out
+
+    def lm_head(self, X):
+        """X: list[t][s][j] -> logits list[t][v]: streams summed, weight-free RMSNorm (eps inside the root),
+        one dot product per vocabulary row."""
+        c = self.cfg
+        out = []
+        for t in range(len(X)):
+            summed = [0.0] * c.d_model
+            for s in range(c.n_streams):
+                for j in range(c.d_model):
+                    summed[j] += X[t][s][j]
+            ms = 0.0
+            for j in range(c.d_model):
+                ms += summed[j] * summed[j]
+            r = 1.0 / math.sqrt(ms / c.d_model + c.rms_eps)
+            logits = []
+            for v in range(c.vocab):
+                acc = 0.0
+                for j in range(c.d_model):
+                    acc += float(self.W.lm_head[v][j]) * (summed[j] * r)
+                logits.append(acc)
+            out.append(logits)
+        return out

@@ -495,3 +495,96 @@ def test_fused_chunks():
     # without correction information moves one chunk per sweep
     a = O.forward_chunked(cfg, W, h0, 1, 2, correct=False)
     assert relerr(a[-1], O.fused_chunk(cfg, W, [2, 3], h0, kv, 0, np.float64)[0]) < 1e-13
+
+
+# ------------------------------------------------------------------ model entry / exit (Alg. 1 lines 1 and 5)
+@pytest.mark.parametrize("n_streams", [1, 3])
+def test_embed_and_lm_head_match_scalar_brute_force(n_streams):
+    cfg = small_cfg(n_streams)
+    W = big_weights(cfg)
+    ids = synth.make_ids(cfg, 1, 6, seed=40)
+    nv = NaiveModel(cfg, W)
+    h0 = O.embed(cfg, W, ids)
+    assert h0.shape == (1, 6, n_streams, cfg.d_model)
+    assert np.array_equal(h0[0], np.array(nv.embed(ids[0].tolist())))
+    # every stream carries the token's own embedding row (not a scaled or split copy)
+    for s in range(n_streams):
+        assert np.array_equal(h0[0, :, s, :], W.embed[ids[0]].astype(np.float64))
+    hL = synth.make_hidden(cfg, 1, 6, seed=41).astype(np.float64)   # streams differ from one another
+    want = np.array(nv.lm_head(to_lists(hL)))
+    got = O.lm_head(cfg, W, hL)
+    assert got.shape == (1, 6, cfg.vocab)
+    assert relerr(got[0], want) < 1e-13
+
+
+def test_lm_head_closed_forms():
+    # a one-hot row of the head reads one feature of the normalised stream sum: logit = sum_s h[s][j] / rms(sum_s h[s])
+    cfg = small_cfg(3)
+    W = big_weights(cfg)
+    W.lm_head = np.zeros_like(W.lm_head)
+    W.lm_head[7, 5] = 1.0
+    W.lm_head[9, 2] = -2.0
+    hL = synth.make_hidden(cfg, 1, 4, seed=42).astype(np.float64)
+    s = hL.sum(axis=2)                                   # [1, T, d]
+    rms = np.sqrt((s * s).mean(-1) + cfg.rms_eps)
+    lg = O.lm_head(cfg, W, hL)
+    assert np.allclose(lg[..., 7], s[..., 5] / rms, rtol=1e-14, atol=0)
+    assert np.allclose(lg[..., 9], -2.0 * s[..., 2] / rms, rtol=1e-14, atol=0)
+    assert np.count_nonzero(np.delete(lg, [7, 9], axis=-1)) == 0
+    # the final norm makes the logits invariant to the scale of h_L (up to eps) ...
+    assert relerr(O.lm_head(cfg, W, 3.0 * hL), lg) < 1e-6
+    # ... and the streams enter through their SUM: a mean would not change the logits either, but moving mass
+    # between streams must not, while changing one stream alone must
+    moved = hL.copy(); moved[:, :, 0] += 0.25; moved[:, :, 1] -= 0.25
+    assert relerr(O.lm_head(cfg, W, moved), lg) < 1e-12
+    bumped = hL.copy(); bumped[:, :, 2, 5] += 1.0
+    assert relerr(O.lm_head(cfg, W, bumped), lg) > 1e-3
+
+
+# ------------------------------------------------------------------ chunkwise form with a prefix / fwd initialisation
+@pytest.mark.parametrize("init", [O.INIT_H0, O.INIT_FWD])
+def test_forward_chunked_prefix_and_fwd(init):
+    cfg = small_cfg(1, L=6)
+    W = big_weights(cfg)
+    h0 = synth.make_hidden(cfg, 1, 4, seed=43).astype(np.float64)
+    L = cfg.n_layer
+    extra = 1 if init == O.INIT_FWD else 0
+    # fuse = 1 is Algorithm 2 with the same prefix and initialisation, state for state
+    for S in (0, 2):
+        for K in (0, 1, 2) if (init == O.INIT_FWD or S > 0) else (1, 2):
+            st = O.forward_chunked(cfg, W, h0, K, 1, S=S, init=init)
+            ref = O.forward_snlp(cfg, W, h0, K, O.MODE_IDN, S=S, init=init)[0]
+            assert len(st) == L - S + 1
+            for i, l in enumerate(range(S, L + 1)):
+                assert relerr(st[i], ref[l]) < 1e-13, (S, K, l)
+    # fuse = 2 behind a prefix of 2: chunkwise finite-step exactness against sequential execution of the SAME fused
+    # model -- after K sweeps the first K (+1 with fwd) chunk outputs are final and the next one is not
+    S, F = 2, 2
+    fseq = O.forward_chunked(cfg, W, h0, None, F, S=S)
+    seq = O.forward_sequential(cfg, W, h0)
+    assert relerr(fseq[0], seq[S]) < 1e-13          # the prefix is Algorithm 1 up to h_S
+    N = (L - S) // F
+    for K in (0, 1) if init == O.INIT_FWD else (1,):
+        st = O.forward_chunked(cfg, W, h0, K, F, S=S, init=init)
+        assert len(st) == N + 1
+        exact = min(N, K + extra)
+        for c in range(exact + 1):
+            assert relerr(st[c], fseq[c]) < 1e-12, (K, c)
+        if exact + 1 <= N:
+            assert relerr(st[exact + 1], fseq[exact + 1]) > 1e-8, (K, exact)
+    # fwd initialisation alone (K = 0) is one evaluation of every chunk on the prefix state
+    if init == O.INIT_FWD:
+        st = O.forward_chunked(cfg, W, h0, 0, F, S=S, init=O.INIT_FWD)
+        kv = O.LayerKV(L, 1, 4, cfg.n_head, cfg.head_dim)
+        for c in range(N):
+            layers = [S + c * F, S + c * F + 1]
+            assert relerr(st[c + 1], O.fused_chunk(cfg, W, layers, seq[S], kv, 0, np.float64)[0]) < 1e-13
+    else:
+        # h0 initialisation, K = 1: h_S plus every chunk's branches evaluated on h_S (App. C.1 form, chunkwise)
+        st = O.forward_chunked(cfg, W, h0, 1, F, S=S)
+        kv = O.LayerKV(L, 1, 4, cfg.n_head, cfg.head_dim)
+        acc = seq[S].copy()
+        for c in range(N):
+            _, a, m = O.fused_chunk(cfg, W, [S + c * F, S + c * F + 1], seq[S], kv, 0, np.float64)
+            acc = acc + (a + m)[:, :, None, :]
+            assert relerr(st[c + 1], acc) < 1e-13
