@@ -5,7 +5,8 @@
  * Conventions
  *   - Every function returns 0 (SNLP_OK) or a negative SNLP_ERR_* code; snlp_last_error() gives a
  *     thread-local message for the last failure.  No exception or abort crosses this boundary and
- *     all arguments are validated before anything is launched.
+ *     all arguments are validated before anything is launched.  Hidden-state pointers (h0, hL, trace_out)
+ *     must be 16-byte aligned and int32 / fp32 scalar arrays 4-byte aligned (whole cudaMalloc'd buffers are); a misaligned pointer is rejected with SNLP_ERR_ARG.
  *   - "host" pointers are read during the call only (the caller keeps ownership and may free them
  *     on return).  "device" pointers are CUDA device memory owned by the caller; the library owns
  *     only its handles, weights, workspace and KV caches.
@@ -146,6 +147,17 @@ int snlp_forward_solver(snlp_model *m, const float *h0, int B, int T, const snlp
 int snlp_decode_step_solver(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, const snlp_solver *solver, int32_t *tok_out,
                             float *resnorm_out, void *stream);
 
+/* Copy the states the handle's last forward left behind (introspection; Alg. 1 / Alg. 2 define the trace, this call
+ * only exposes it where the entry point has no trace_out of its own).  Every forward, prefill, decode step and
+ * draft-and-verify round runs on the handle's internal trace [L+1][rows][n][d]; after
+ *   snlp_decode_step*          rows = batch size: the states of the new position of every sequence,
+ *   snlp_prefill               rows = B * (tokens of the last chunk), sequence-major,
+ *   snlp_draft_and_verify*     rows = block + 1: the verifier's sequential forward over [last_tok, x_1..x_block],
+ *   snlp_forward_*             rows = B * T
+ * this copies it to trace_out (device fp32, (L+1)*rows*n*d values).  With fused chunks only chunk-boundary states are
+ * defined.  Errors: ARG, STATE (nothing has run yet), SHAPE (rows differs from the last call's row count). */
+int snlp_copy_trace(snlp_model *m, int rows, float *trace_out, void *stream);
+
 /* LMHead (Alg. 1 line 5 / Alg. 2 line 14): sum the streams of hL (device fp32 [rows][n][d]), RMSNorm,
  * project with lm_head.  logits (device fp32 [rows][vocab], nullable) and argmax (device int32 [rows],
  * nullable; ties -> lowest index); at least one of them must be given.
@@ -158,7 +170,10 @@ int snlp_lm_head(snlp_model *m, const float *hL, int rows, float *logits, int32_
  * Errors: ARG, SHAPE (B > max_batch, max_ctx > config.max_ctx), OOM. */
 int snlp_kv_create(snlp_model *m, int B, int max_ctx, snlp_kv **out);
 int snlp_kv_destroy(snlp_kv *kv);
-int snlp_kv_len(const snlp_kv *kv, int32_t *len);            /* host out                          */
+/* The length is kept on the device and mirrored on the host.  After snlp_draft_and_verify_async the host knows only an
+ * upper bound; snlp_kv_len (and snlp_kv_truncate) then wait for the device (cudaDeviceSynchronize) and read the length
+ * back.  In every other situation they return at once. */
+int snlp_kv_len(snlp_kv *kv, int32_t *len);                   /* host out                          */
 int snlp_kv_truncate(snlp_kv *kv, int new_len, void *stream); /* 0 <= new_len <= len, else ARG     */
 
 /* Sequential forward (Alg. 1) over ids (device int32 [B][T]) at positions len .. len+T-1; fills the
@@ -174,6 +189,10 @@ int snlp_prefill(snlp_model *m, snlp_kv *kv, const int32_t *ids, int B, int T, i
  * Each sweep recomputes the new position's keys/values from its current iterate and overwrites the
  * cache slot, so the cache keeps the last sweep's values.  resnorm_out as in snlp_forward_parallel
  * (ignored for K = 0).  tok_in and tok_out may alias.
+ * With CUDA graphs on (the default) a step is captured once per (batch, solver, attention grid size, resnorm_out, cache)
+ * and replayed; the token buffers are not baked into the graph (the step's kernels find them through a device slot
+ * that a one-thread kernel re-points when a call brings other buffers than the previous call did), so callers may
+ * pass fresh buffers every step.
  * Errors: ARG (K < 0, mode), SHAPE (len + 1 > max_ctx), STATE. */
 int snlp_decode_step(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, int K, int mode, int32_t *tok_out,
                      float *resnorm_out, void *stream);
@@ -191,17 +210,28 @@ int snlp_decode_step_host(snlp_model *m, snlp_kv *kv, const int32_t *tok_in_host
  * [last_tok, x_1..x_block] (block+1 rows) verifies them and overwrites the drafter's cache entries;
  * the longest prefix with x_i == verifier token y_{i-1} is accepted.  Writes emitted (device int32
  * [block+1]) = x_1..x_n, y_n; n_emitted = n+1; n_accepted = n (device int32 each); *last_tok <- y_n;
- * cache length = len_before + n + 1.  The call synchronises `stream` before returning (the host needs
- * n to track the cache length).  The emitted stream equals the model's sequential greedy stream.
+ * cache length = len_before + n + 1.  This form synchronises `stream` before returning and brings the
+ * cache length back to the host.  The emitted stream equals the model's sequential greedy stream.
  * Errors: ARG (block < 1, K < 1, mode, NULLs), SHAPE (kv batch != 1, len + block + 1 > max_ctx,
  * block + 1 > max_rows), STATE. */
 int snlp_draft_and_verify(snlp_model *m, snlp_kv *kv, int32_t *last_tok, int block, int K, int mode,
                           int32_t *emitted, int32_t *n_emitted, int32_t *n_accepted, void *stream);
+/* The same round (Sec. 5.1) without any host synchronisation: everything is enqueued on `stream`; n_accepted,
+ * n_emitted, the emitted tokens, *last_tok and the new cache length stay on the device, so rounds can be issued
+ * back to back.  Until snlp_kv_len is called the host tracks the cache length by its upper bound (every draft
+ * accepted): capacity checks use that bound -- a call that would not fit under it first fetches the true length --
+ * and the decode attention sizes its grid by it (chunks beyond the true length add exact zeros, so no result bit
+ * changes).  Errors as snlp_draft_and_verify. */
+int snlp_draft_and_verify_async(snlp_model *m, snlp_kv *kv, int32_t *last_tok, int block, int K, int mode,
+                                int32_t *emitted, int32_t *n_emitted, int32_t *n_accepted, void *stream);
 
 /* Tuning / introspection (no effect on results).  flag 0: use CUDA graphs for decode steps (default 1).
  * flag 1: force the generic SIMT kernels even where a specialised kernel exists (default 0; testing).
  * flag 2: time every launch with CUDA events on its stream, accumulated per kernel class (default 0;
- *         while on, decode steps are launched directly instead of replaying graphs). */
+ *         while on, decode steps are launched directly instead of replaying graphs).
+ * flag 3: failure-detection test hook: waits for the device, then writes `value != 0` into the error word that a
+ *         kernel raises when one of its bounded waits expires; snlp_device_status then reports it exactly as it
+ *         would report a real expiry (no kernel is made to wait). */
 int snlp_set_flag(snlp_model *m, int flag, int value);
 
 /* Kernel classes of snlp_kernel_times, in order: QKV projection, attention, out-projection, MLP up,
@@ -216,16 +246,19 @@ int snlp_device_status(snlp_model *m, void *stream);
 
 /* Number of kernel launches this handle has enqueued since creation (graph replays count their nodes). */
 int snlp_launch_count(const snlp_model *m, int64_t *count);
+/* Number of decode-step graphs this handle has captured since creation. */
+int snlp_graph_count(const snlp_model *m, int64_t *captured);
 
 /* Greedy LM head that allocates nothing (the paper has no counterpart: this entry point exists for
- * callers that cannot obtain device memory at call time -- for example code running between the
- * begin and end of a CUDA stream capture, a serving loop whose memory budget has been handed entirely to
- * another allocator, or a latency-critical path where the implicit device synchronisation of an
+ * callers that cannot obtain device memory at call time -- for example a serving loop whose memory budget
+ * has been handed entirely to another allocator, a plug-in running inside a host application that forbids
+ * allocation after start-up, or a latency-critical path where the implicit device synchronisation of an
  * allocation is not acceptable).  Same computation as snlp_lm_head restricted to the argmax:
  *     argmax[r] = argmax_v  lm_head[v] . RMSNorm(sum_s hL[r][s][:])        (ties -> lowest index)
- * but without a model handle and without a cudaMalloc'd workspace: the per-tile argmax partials go to a
- * fixed 256 KiB array inside the library image (each GPU that loads the library holds one copy until the
- * process exits).
+ * by a kernel of its own (the two entry points add a logit's terms in different orders, so they can disagree
+ * where two logits are closer than bf16 rounding noise), without a model handle and without a cudaMalloc'd
+ * workspace: the per-tile argmax partials go to a fixed 256 KiB array inside the library image (each GPU that
+ * loads the library holds one copy until the process exits).
  *   hL           device fp32 [rows][n_streams][d_model]
  *   lm_head_bf16 device bf16 bit patterns [vocab][d_model], caller-owned (inputs and outputs are still yours)
  *   argmax       device int32 [rows]
@@ -237,7 +270,9 @@ int snlp_launch_count(const snlp_model *m, int64_t *count);
  * All calls on a device share the one array, which keeps whatever the previous call left in it (nothing
  * needs to start at zero: every slot a call reads, it has written first).  Two calls that overlap on the
  * GPU -- different streams without ordering, or two host threads -- race on it: serialise them.
- * Errors: ARG (NULL, non-positive sizes), SHAPE (beyond the limits), UNSUPPORTED (vocab % 128, d_model % 32), CUDA. */
+ * hL and lm_head_bf16 must be 16-byte aligned, argmax 4-byte aligned.
+ * Errors: ARG (NULL, misaligned pointer, non-positive sizes), SHAPE (beyond the limits), UNSUPPORTED (vocab % 128,
+ * d_model % 32), CUDA. */
 #define SNLP_STATIC_LM_HEAD_MAX_VOCAB 262144
 #define SNLP_STATIC_LM_HEAD_MAX_D_MODEL 4096
 int snlp_lm_head_greedy_static(const float *hL, const void *lm_head_bf16, int rows, int n_streams, int d_model, int vocab,

@@ -350,7 +350,9 @@ __global__ void k_prep_rows(const float *__restrict__ trace, int l0, int M, int 
 template <int NS>
 __global__ void k_init_rows(float *__restrict__ trace, int l0, int L, int M, int d, const HcCoef *__restrict__ coef,
                             __nv_bfloat16 *__restrict__ xb, float *__restrict__ ssq_x, float *__restrict__ xm, int write_trace,
-                            const int32_t *__restrict__ ids = nullptr, const __nv_bfloat16 *__restrict__ table = nullptr, int vocab = 0) {
+                            const int32_t *__restrict__ ids = nullptr, const __nv_bfloat16 *__restrict__ table = nullptr, int vocab = 0,
+                            const int32_t *const *__restrict__ ids_pp = nullptr) {
+  if (ids_pp != nullptr) ids = *ids_pp;   // the ids' address is read from a device slot (replayed decode graphs)
   const int d4 = d >> 2, c4 = threadIdx.x;
   const size_t row = blockIdx.x, Md4 = (size_t)M * d4;
   float4 *tr4 = reinterpret_cast<float4 *>(trace);

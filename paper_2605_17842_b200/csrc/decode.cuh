@@ -1,259 +1,14 @@
-// Decode-regime kernels (at most 16 rows per layer, bf16 operands, head_dim 128): the sweep is bound by
-// streaming every layer's weights and keys/values from HBM once.
-//
-//  k_gemv_mma   layer-batched weight-streaming "GEMV": y[l][tok][n] = sum_k x[l][tok][k] W[l][n][k].
-//               The weights are the 16-row MMA operand (read once, 16-byte loads straight from global
-//               memory into the fragment registers), the <= 16 tokens are the 8-wide operand staged in
-//               shared memory, so the ALU cost is independent of the token count and a token's result
-//               does not depend on how many other tokens are in the call (batch invariance).
-//               Fused prologues: RMSNorm of the fp32 input row, residual add of the attention branch.
-//               Fused epilogues: rotary + QK-norm + KV-cache append; ReLU^2 + bf16 cast; per-tile argmax.
-//  k_attn_decode / k_attn_combine   split-KV causal attention over the (chunk, batch x head, layer) grid.
+// Decode-regime attention (at most 16 query rows per sequence, bf16 operands, head_dim 128): split-KV causal
+// attention over the (chunk, batch x head, layer) grid; a sweep streams every layer's keys/values from HBM once.
 #pragma once
 #include "common.cuh"
 
 namespace snlp {
 
-enum { PRO_BF16 = 0, PRO_NORM = 1, PRO_RESID_NORM = 2 };
-enum { EPI_PARTIAL = 0, EPI_QKV = 1, EPI_RELU2 = 2, EPI_LMHEAD = 3 };
-
-struct GemvParams {
-  const __nv_bfloat16 *W; size_t w_ls;  // [nl][N][Kd]
-  int N, Kd, kslice, M;
-  // prologue
-  const __nv_bfloat16 *xb; size_t xb_ls;            // PRO_BF16: [nl][M][Kd]
-  const float *xf; size_t xf_ls, xf_rs; int nsum;   // PRO_NORM / PRO_RESID_NORM: fp32 rows (sum of nsum streams)
-  const float *ap; size_t ap_ls, ap_ss; int ap_splits;  // PRO_RESID_NORM: attention-branch partials [S][nl][M][Kd]
-  const HcCoef *coef;                               // indexed by blockIdx.z (already offset to the first layer)
-  float eps;
-  // epilogue
-  float *out; size_t out_ls, out_ss;                // EPI_PARTIAL: [ksplit][nl][M][N]
-  __nv_bfloat16 *zout; size_t z_ls;                 // EPI_RELU2:   [nl][M][N]
-  __nv_bfloat16 *q; size_t q_ls;                    // EPI_QKV
-  __nv_bfloat16 *kc, *vc; size_t kv_ls, kv_bs;
-  int T, H; const int *pos_base; const float2 *rope; float qk_eps;
-  float *logits; float *pm_val; int *pm_idx; int ntile;  // EPI_LMHEAD: logits [M][N] nullable, partial argmax [M][ntile]
-};
-
 __device__ __forceinline__ uint4 ldg_stream(const void *p) {
   uint4 v;
   asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
   return v;
-}
-
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                               uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t *>(&v);
-}
-
-constexpr int kGemvThreads = 256;
-constexpr int kGemvRows = 128;   // weight rows per CTA: 8 warps x 16
-constexpr int kGemvPad = 32;     // bf16 elements of padding per staged token row (64 B: conflict-free 16 B reads)
-constexpr int kGemvUnroll = 8;   // 32-wide k steps kept in flight per thread (16 x 16 B loads)
-
-// grid (N/128, ksplit, nl), 256 threads.  NT = number of 8-token tiles (1 or 2).
-// Dynamic shared memory: NT*8*(kslice+32) bf16 + NT*8*129 floats + 16 floats.
-template <int NT, int PRO, int EPI>
-__global__ void __launch_bounds__(kGemvThreads) k_gemv_mma(GemvParams p) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int xstride = p.kslice + kGemvPad;
-  __nv_bfloat16 *xs = reinterpret_cast<__nv_bfloat16 *>(smem_raw);
-  float *outs = reinterpret_cast<float *>(smem_raw + (size_t)NT * 8 * xstride * sizeof(__nv_bfloat16));
-  float *rstd = outs + NT * 8 * (kGemvRows + 1);
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int tile = blockIdx.x, ks = blockIdx.y, l = blockIdx.z;
-  const int kbase = ks * p.kslice;
-  const int g = lane >> 2, t = lane & 3;
-
-  // ---- prologue: stage the token operand as bf16 ------------------------------------------------
-  if (PRO == PRO_BF16) {
-    const int vec_per_row = p.kslice >> 3;
-    for (int i = tid; i < NT * 8 * vec_per_row; i += kGemvThreads) {
-      const int tok = i / vec_per_row, v = i % vec_per_row;
-      uint4 val = make_uint4(0, 0, 0, 0);
-      if (tok < p.M) val = *reinterpret_cast<const uint4 *>(p.xb + (size_t)l * p.xb_ls + (size_t)tok * p.Kd + kbase + v * 8);
-      *reinterpret_cast<uint4 *>(xs + (size_t)tok * xstride + v * 8) = val;
-    }
-    if (tid < NT * 8) rstd[tid] = 1.f;
-  } else {
-    // one warp per token; kslice == Kd here
-    for (int tok = warp; tok < NT * 8; tok += kGemvThreads / 32) {
-      float ss = 0.f;
-      if (tok < p.M) {
-        const float *x = p.xf + (size_t)l * p.xf_ls + (size_t)tok * p.xf_rs;
-        const float kappa = PRO == PRO_RESID_NORM ? p.coef[l].kappa : 0.f;
-        for (int j = lane * 4; j < p.Kd; j += 128) {
-          float4 v = *reinterpret_cast<const float4 *>(x + j);
-          for (int s = 1; s < p.nsum; ++s) {
-            const float4 w = *reinterpret_cast<const float4 *>(x + (size_t)s * p.Kd + j);
-            v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
-          }
-          if (PRO == PRO_RESID_NORM) {
-            const float *a = p.ap + (size_t)l * p.ap_ls + (size_t)tok * p.Kd + j;
-            float4 as = *reinterpret_cast<const float4 *>(a);
-            for (int s = 1; s < p.ap_splits; ++s) {
-              const float4 w = *reinterpret_cast<const float4 *>(a + (size_t)s * p.ap_ss);
-              as.x += w.x; as.y += w.y; as.z += w.z; as.w += w.w;
-            }
-            v.x += kappa * as.x; v.y += kappa * as.y; v.z += kappa * as.z; v.w += kappa * as.w;
-          }
-          ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-          uint2 pk = make_uint2(pack_bf16(v.x, v.y), pack_bf16(v.z, v.w));
-          *reinterpret_cast<uint2 *>(xs + (size_t)tok * xstride + j) = pk;
-        }
-        ss = warp_sum(ss);
-        if (lane == 0) rstd[tok] = rsqrtf(ss / (float)p.Kd + p.eps);
-      } else {
-        for (int j = lane * 4; j < p.Kd; j += 128) *reinterpret_cast<uint2 *>(xs + (size_t)tok * xstride + j) = make_uint2(0, 0);
-        if (lane == 0) rstd[tok] = 0.f;
-      }
-    }
-  }
-  __syncthreads();
-
-  // ---- main loop: stream 16 weight rows per warp -------------------------------------------------
-  float acc[NT][4];
-#pragma unroll
-  for (int i = 0; i < NT; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
-  const int r0 = tile * kGemvRows + warp * 16;
-  const __nv_bfloat16 *w0 = p.W + (size_t)l * p.w_ls + (size_t)(r0 + g) * p.Kd + kbase + t * 8;
-  const __nv_bfloat16 *w1 = w0 + (size_t)8 * p.Kd;
-  const __nv_bfloat16 *x0 = xs + (size_t)g * xstride + t * 8;
-  for (int kk = 0; kk < p.kslice; kk += 32 * kGemvUnroll) {
-    uint4 wa[kGemvUnroll], wb[kGemvUnroll];
-#pragma unroll
-    for (int u = 0; u < kGemvUnroll; ++u) {
-      const int k = kk + 32 * u;
-      if (k < p.kslice) {
-        wa[u] = ldg_stream(w0 + k);
-        wb[u] = ldg_stream(w1 + k);
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < kGemvUnroll; ++u) {
-      const int k = kk + 32 * u;
-      if (k < p.kslice) {
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          const uint4 xv = *reinterpret_cast<const uint4 *>(x0 + (size_t)nt * 8 * xstride + k);
-          mma_bf16_16816(acc[nt], wa[u].x, wb[u].x, wa[u].y, wb[u].y, xv.x, xv.y);
-          mma_bf16_16816(acc[nt], wa[u].z, wb[u].z, wa[u].w, wb[u].w, xv.z, xv.w);
-        }
-      }
-    }
-  }
-  // accumulator (row g / g+8, token 2t / 2t+1) -> outs[token][row in tile]
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt) {
-    const int tk = nt * 8 + 2 * t, rr = warp * 16 + g;
-    outs[(tk) * (kGemvRows + 1) + rr] = acc[nt][0];
-    outs[(tk + 1) * (kGemvRows + 1) + rr] = acc[nt][1];
-    outs[(tk) * (kGemvRows + 1) + rr + 8] = acc[nt][2];
-    outs[(tk + 1) * (kGemvRows + 1) + rr + 8] = acc[nt][3];
-  }
-  __syncthreads();
-
-  // ---- epilogues -----------------------------------------------------------------------------------
-  const int n0 = tile * kGemvRows;
-  if (EPI == EPI_PARTIAL) {
-    for (int i = tid; i < p.M * kGemvRows; i += kGemvThreads) {
-      const int tok = i >> 7, r = i & 127;
-      p.out[(size_t)ks * p.out_ss + (size_t)l * p.out_ls + (size_t)tok * p.N + n0 + r] = outs[tok * (kGemvRows + 1) + r] * rstd[tok];
-    }
-  } else if (EPI == EPI_RELU2) {
-    for (int i = tid; i < p.M * kGemvRows; i += kGemvThreads) {
-      const int tok = i >> 7, r = i & 127;
-      const float v = fmaxf(outs[tok * (kGemvRows + 1) + r] * rstd[tok], 0.f);
-      p.zout[(size_t)l * p.z_ls + (size_t)tok * p.N + n0 + r] = __float2bfloat16_rn(v * v);
-    }
-  } else if (EPI == EPI_QKV) {
-    // the tile is exactly one 128-wide head of q, k or v
-    const int kind = tile / p.H, head = tile % p.H, d = p.H * 128;
-    for (int tok = warp; tok < p.M; tok += kGemvThreads / 32) {
-      const int b = tok / p.T, pos = *p.pos_base + (tok % p.T);
-      const float *y = outs + tok * (kGemvRows + 1);
-      const float rs = rstd[tok];
-      __nv_bfloat16 *dst;
-      if (kind == 0) dst = p.q + (size_t)l * p.q_ls + (size_t)tok * d + head * 128;
-      else dst = (kind == 1 ? p.kc : p.vc) + (size_t)l * p.kv_ls + (size_t)b * p.kv_bs + (size_t)pos * d + head * 128;
-      if (kind == 2) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) dst[lane + 32 * j] = __float2bfloat16_rn(y[lane + 32 * j] * rs);
-      } else {
-        const float2 c0 = p.rope[(size_t)pos * 64 + lane], c1 = p.rope[(size_t)pos * 64 + lane + 32];
-        const float a1 = y[lane] * rs, a2 = y[lane + 64] * rs, b1 = y[lane + 32] * rs, b2 = y[lane + 96] * rs;
-        const float ya1 = a1 * c0.x - a2 * c0.y, ya2 = a1 * c0.y + a2 * c0.x;
-        const float yb1 = b1 * c1.x - b2 * c1.y, yb2 = b1 * c1.y + b2 * c1.x;
-        const float ss = warp_sum(ya1 * ya1 + ya2 * ya2 + yb1 * yb1 + yb2 * yb2);
-        const float r = rsqrtf(ss * (1.f / 128.f) + p.qk_eps);
-        dst[lane] = __float2bfloat16_rn(ya1 * r);
-        dst[lane + 64] = __float2bfloat16_rn(ya2 * r);
-        dst[lane + 32] = __float2bfloat16_rn(yb1 * r);
-        dst[lane + 96] = __float2bfloat16_rn(yb2 * r);
-      }
-    }
-  } else {  // EPI_LMHEAD
-    for (int tok = warp; tok < p.M; tok += kGemvThreads / 32) {
-      const float *y = outs + tok * (kGemvRows + 1);
-      const float rs = rstd[tok];
-      float bv = -INFINITY;
-      int bi = 0x7fffffff;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int r = lane + 32 * j;
-        const float v = y[r] * rs;
-        if (p.logits) p.logits[(size_t)tok * p.N + n0 + r] = v;
-        if (v > bv) { bv = v; bi = n0 + r; }
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-        if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-      }
-      if (lane == 0) { p.pm_val[(size_t)tok * p.ntile + tile] = bv; p.pm_idx[(size_t)tok * p.ntile + tile] = bi; }
-    }
-  }
-}
-
-// Final argmax over the per-tile partials (ties -> lowest index).  One block per token.
-// bump (nullable): a device counter incremented by one once per launch (the cache position after a decode step).
-static __global__ void k_argmax_tiles(const float *__restrict__ pm_val, const int *__restrict__ pm_idx, int ntile, int32_t *__restrict__ out,
-                                      int *__restrict__ bump = nullptr) {
-  __shared__ float sv[32];
-  __shared__ int si[32];
-  const int tok = blockIdx.x;
-  float bv = -INFINITY;
-  int bi = 0x7fffffff;
-  for (int j = threadIdx.x; j < ntile; j += blockDim.x) {
-    const float v = pm_val[(size_t)tok * ntile + j];
-    const int ix = pm_idx[(size_t)tok * ntile + j];
-    if (v > bv || (v == bv && ix < bi)) { bv = v; bi = ix; }
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-  }
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  if (lane == 0) { sv[w] = bv; si[w] = bi; }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const int nw = (blockDim.x + 31) >> 5;
-    for (int i = 1; i < nw; ++i)
-      if (sv[i] > bv || (sv[i] == bv && si[i] < bi)) { bv = sv[i]; bi = si[i]; }
-    out[tok] = bi == 0x7fffffff ? 0 : bi;
-    if (bump != nullptr && tok == 0) *bump += 1;
-  }
 }
 
 // ---------------------------------------------------------------------------------------------------

@@ -9,8 +9,9 @@ namespace snlp {
 // h_0 = Embed(ids): one block per row; the embedding row is replicated into each stream.
 template <typename T>
 __global__ void k_embed(const int32_t *__restrict__ ids, const T *__restrict__ table, float *__restrict__ h0,
-                        int d, int n, int vocab) {
+                        int d, int n, int vocab, const int32_t *const *__restrict__ ids_pp = nullptr) {
   const int row = blockIdx.x;
+  if (ids_pp != nullptr) ids = *ids_pp;   // the ids' address is read from a device slot (replayed decode graphs)
   int id = ids[row];
   id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);
   const T *src = table + (size_t)id * d;
@@ -232,7 +233,10 @@ __global__ void k_attn_generic(const T *__restrict__ q, size_t q_ls, const T *__
 
 // ---------------------------------------------------------------------------------------------
 // Per-row argmax over `vocab` logits, ties to the lowest index.  One block per row.
-__global__ void k_argmax_rows(const float *__restrict__ logits, int vocab, int32_t *__restrict__ out) {
+// out_pp (nullable): the output's address is read from a device slot and `out_off` added (replayed decode graphs).
+__global__ void k_argmax_rows(const float *__restrict__ logits, int vocab, int32_t *__restrict__ out, int32_t *const *__restrict__ out_pp = nullptr,
+                              int out_off = 0) {
+  if (out_pp != nullptr) out = *out_pp + out_off;
   __shared__ float sv[32];
   __shared__ int si[32];
   const float *x = logits + (size_t)blockIdx.x * vocab;
@@ -282,11 +286,15 @@ __global__ void k_premix(const float *__restrict__ trace, size_t t_ls, int n, in
 // Small helpers for the decoding policies -------------------------------------------------------
 __global__ void k_set_int(int *p, int v) { *p = v; }
 __global__ void k_add_int(int *p, int v) { *p += v; }
+__global__ void k_copy_int(int *dst, const int *src) { *dst = *src; }
+// The device slot through which replayed decode graphs find the caller's token buffers.
+__global__ void k_set_ptrs(const void **slot, const void *a, const void *b) { slot[0] = a; slot[1] = b; }
 
 // Greedy acceptance (Sec. 5.1): n = longest prefix with draft[i] == y[i]; emit drafts[0..n), y[n].
 __global__ void k_accept(const int32_t *__restrict__ drafts, const int32_t *__restrict__ y, int block, int32_t *emitted,
-                         int32_t *n_emitted, int32_t *n_accepted, int32_t *last_tok, int *pos, int len0) {
+                         int32_t *n_emitted, int32_t *n_accepted, int32_t *last_tok, int *pos, const int *len0_p) {
   if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  const int len0 = *len0_p;   // cache length when the round began (kept on the device: the host need not know it)
   int n = 0;
   while (n < block && drafts[n] == y[n]) ++n;
   for (int i = 0; i < n; ++i) emitted[i] = drafts[i];

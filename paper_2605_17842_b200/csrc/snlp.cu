@@ -61,13 +61,14 @@ constexpr int kMaxSplits = 4;    // K-splits of the partial-sum GEMV outputs
 constexpr int kDecodeRows = 16;  // largest row count served by the decode-regime kernels
 constexpr size_t kCorrSmallSmem = 160 * 1024;
 
+// A captured decode step.  The token buffers are not part of the key: the step's kernels find them through the
+// handle's device slot (tok_slot), so one graph serves every caller buffer.
 struct GraphKey {
   int B, K, mode, prefix, init, fuse, nchunk;
-  const void *tin, *tout, *res;
+  const void *res;
   const void *kv;
   bool operator<(const GraphKey &o) const {
-    return std::tie(B, K, mode, prefix, init, fuse, nchunk, tin, tout, res, kv) <
-           std::tie(o.B, o.K, o.mode, o.prefix, o.init, o.fuse, o.nchunk, o.tin, o.tout, o.res, o.kv);
+    return std::tie(B, K, mode, prefix, init, fuse, nchunk, res, kv) < std::tie(o.B, o.K, o.mode, o.prefix, o.init, o.fuse, o.nchunk, o.res, o.kv);
   }
 };
 struct GraphEntry { cudaGraphExec_t exec; int64_t nodes; };
@@ -116,14 +117,22 @@ struct snlp_model {
   int n_sm = 148;
   EncodeTiledFn encode_tiled = nullptr;  // cuTensorMapEncodeTiled, looked up through the runtime
   int *dev_err = nullptr;                // raised by a kernel whose bounded wait expired
+  int last_rows = 0;                     // rows of the forward whose states the internal trace holds (snlp_copy_trace)
+  const void **tok_slot = nullptr;       // device: addresses of the decode step's {tok_in, tok_out}, read by its kernels
+  const void *slot_in = nullptr, *slot_out = nullptr;   // what tok_slot holds, in the order the calls were issued
+  int64_t graph_captures = 0;            // decode graphs captured so far
   cudaStream_t cap_stream = nullptr;  // capture target: graphs are recorded here and replayed on the caller's stream
 };
 
 struct snlp_kv {
   snlp_model *m = nullptr;
-  int B = 0, max_ctx = 0, len = 0;
+  int B = 0, max_ctx = 0;
+  // The cache length lives on the device (pos[0]); the host mirrors it.  After an asynchronous draft-and-verify
+  // round only an upper bound is known here (len_known == false, len_hi) until snlp_kv_len reads the device value.
+  int len = 0, len_hi = 0;
+  bool len_known = true;
   void *k = nullptr, *v = nullptr;
-  int *pos = nullptr;
+  int *pos = nullptr;   // device int[4]: [0] the length, [1] the length saved at the start of a draft-and-verify round
 };
 
 // a forward call's geometry and key/value store
@@ -135,6 +144,7 @@ struct Fwd {
   int pos_hi;           // host copy of *pos
   int kv_rows;          // rows per sequence in the key / value store
   const int32_t *embed_ids = nullptr;   // non-NULL: state 0 is the embedding of these tokens and has not been written yet
+  const int32_t *const *embed_ids_pp = nullptr;   // the same, with the tokens' address read from a device slot
   bool last_pass = false;   // no sweep follows this correction: it need not prepare the next sweep's branch inputs
   int implicit_state = -1;  // >= 0: states after this one are not materialised yet and equal it (first pass after Alg. 2 line 5)
   cudaStream_t st;
@@ -284,6 +294,7 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
   A(&m->zero, 16);
   A(&m->lm_counter, 16);
   A(&m->spec, 2 * (R + 1) * 4);
+  A(&m->tok_slot, 2 * sizeof(void *));
   if (rc == SNLP_OK && (cudaHostAlloc((void **)&m->tok_pin, (size_t)2 * c.max_batch * 4, cudaHostAllocMapped) != cudaSuccess ||
                         cudaHostGetDevicePointer((void **)&m->tok_dev, m->tok_pin, 0) != cudaSuccess)) {
     cudaGetLastError();
@@ -413,6 +424,11 @@ extern "C" int snlp_set_flag(snlp_model *m, int flag, int value) {
   if (flag == 0) m->use_graphs = value != 0;
   else if (flag == 1) m->force_generic = value != 0;
   else if (flag == 2) m->timing = value != 0;
+  else if (flag == 3) {   // host-side injection of the error word a kernel raises when a bounded wait expires
+    const int v = value != 0;
+    CU(cudaDeviceSynchronize());
+    CU(cudaMemcpy(m->dev_err, &v, sizeof v, cudaMemcpyHostToDevice));
+  }
   else return fail(SNLP_ERR_ARG, "snlp_set_flag: unknown flag %d", flag);
   return SNLP_OK;
 }
@@ -799,7 +815,7 @@ static int check_solver(const snlp_model *m, const snlp_solver &sol, const char 
   return SNLP_OK;
 }
 
-static int embed_impl(snlp_model *m, cudaStream_t st, const int32_t *ids, int rows, float *h0);
+static int embed_impl(snlp_model *m, cudaStream_t st, const int32_t *ids, int rows, float *h0, const int32_t *const *ids_pp = nullptr);
 
 // General Alg. 2 over the internal trace (trace[0] must hold h_0, or f.embed_ids the tokens it is the embedding of): sequential prefix, initialisation, K sweeps over the
 // suffix in chunks of `fuse` fused layers (Eq. 5 for fuse = 1, Eq. 11 otherwise).
@@ -810,8 +826,9 @@ static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *res
   const int S = (seq && F == 1) ? L : sol.prefix;
   // a decode step hands over token ids instead of state 0: the initialisation kernel embeds them itself where it runs
   // on state 0; every other path needs the embedding first
-  const bool fused_embed = f.embed_ids != nullptr && umma_path_ok(m) && S == 0 && !seq;
-  if (f.embed_ids != nullptr && !fused_embed) TRY(embed_impl(m, f.st, f.embed_ids, f.M, m->trace));
+  const bool have_ids = f.embed_ids != nullptr || f.embed_ids_pp != nullptr;
+  const bool fused_embed = have_ids && umma_path_ok(m) && S == 0 && !seq;
+  if (have_ids && !fused_embed) TRY(embed_impl(m, f.st, f.embed_ids, f.M, m->trace, f.embed_ids_pp));
   if (resnorm_out && sol.K > 0 && !seq) CU(cudaMemsetAsync(resnorm_out, 0, (size_t)sol.K * L * 2 * sizeof(float), f.st));
   if (S > 0) {  // Alg. 2 lines 2-4
     if (umma_path_ok(m)) TRY(prep_rows(m, f, 0, 1));
@@ -833,7 +850,7 @@ static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *res
   // Alg. 2 line 5: every suffix state starts at h_S
   if (umma_path_ok(m)) {
     switch (c.n_streams) {   // one kernel: the copies and the layers' first branch inputs
-#define CASE(NS) case NS: KLAUNCH(m, f.st, KC_OTHER, k_init_rows<NS><<<f.M, c.d_model / 4, 0, f.st>>>(m->trace, S, L, f.M, c.d_model, m->coef, (__nv_bfloat16 *)m->xn, m->ssq_x, m->xm, 0, fused_embed ? f.embed_ids : nullptr, (const __nv_bfloat16 *)m->embed, c.vocab)); break;
+#define CASE(NS) case NS: KLAUNCH(m, f.st, KC_OTHER, k_init_rows<NS><<<f.M, c.d_model / 4, 0, f.st>>>(m->trace, S, L, f.M, c.d_model, m->coef, (__nv_bfloat16 *)m->xn, m->ssq_x, m->xm, 0, fused_embed ? f.embed_ids : nullptr, (const __nv_bfloat16 *)m->embed, c.vocab, fused_embed ? f.embed_ids_pp : nullptr)); break;
       CASE(1) CASE(2) CASE(3) CASE(4) CASE(5) CASE(6) CASE(7) CASE(8)
 #undef CASE
     }
@@ -890,7 +907,9 @@ static int parallel(snlp_model *m, const Fwd &f, int K, int mode, float *resnorm
 // LMHead on `rows` hidden states.  pre_xb / pre_ssq: the bf16 stream-summed rows and their sums of squares if the
 // caller already has them (slot L of the branch-input buffers after a decode-regime forward), else NULL.
 static int lm_head_impl(snlp_model *m, cudaStream_t st, const float *hL, size_t row_stride, int rows, float *logits, int32_t *argmax,
-                        const __nv_bfloat16 *pre_xb = nullptr, const float *pre_ssq = nullptr, int *bump = nullptr) {
+                        const __nv_bfloat16 *pre_xb = nullptr, const float *pre_ssq = nullptr, int *bump = nullptr,
+                        int32_t *const *argmax_pp = nullptr) {
+  const bool want_argmax = argmax != nullptr || argmax_pp != nullptr;
   const snlp_config &c = m->cfg;
   const int d = c.d_model, V = c.vocab, n = c.n_streams;
   if (umma_path_ok(m) && rows <= kDecodeRows) {
@@ -903,9 +922,9 @@ static int lm_head_impl(snlp_model *m, cudaStream_t st, const float *hL, size_t 
     UmmaParams p{};
     p.ssq = pre_ssq; p.nparts = P; p.eps = c.rms_eps;
     p.logits = logits; p.pm_val = m->pm_val; p.pm_idx = m->pm_idx;
-    p.argmax = argmax; p.bump = argmax ? bump : nullptr; p.lm_counter = m->lm_counter;   // the last CTA merges the tiles' maxima
+    p.argmax = argmax; p.argmax_pp = argmax_pp; p.bump = want_argmax ? bump : nullptr; p.lm_counter = m->lm_counter;   // the last CTA merges the tiles' maxima
     TRY(umma_gemm<UEPI_LMHEAD>(m, st, KC_LMHEAD, pre_xb, 0, m->w_lm, 0, p, rows, V, d, 1, 1));
-    if (!argmax && bump) KLAUNCH(m, st, KC_OTHER, k_add_int<<<1, 1, 0, st>>>(bump, 1));
+    if (!want_argmax && bump) KLAUNCH(m, st, KC_OTHER, k_add_int<<<1, 1, 0, st>>>(bump, 1));
     return SNLP_OK;
   }
   for (int r0 = 0; r0 < rows; r0 += m->logit_rows) {
@@ -921,19 +940,19 @@ static int lm_head_impl(snlp_model *m, cudaStream_t st, const float *hL, size_t 
       KLAUNCH(m, st, KC_OTHER, k_rmsnorm_cast<T><<<dim3(nr, 1), 256, 0, st>>>(src, 0, row_stride, n, (T *)m->xlm, 0, d, c.rms_eps));
       TRY(gemm<T>(m, st, KC_LMHEAD, (const T *)m->xlm, 0, (const T *)m->lm_head, 0, lg, 0, nr, V, d, 1));
     }
-    if (argmax) {
-      KLAUNCH(m, st, KC_LMHEAD, k_argmax_rows<<<nr, 256, 0, st>>>(lg, V, argmax + r0));
+    if (want_argmax) {
+      KLAUNCH(m, st, KC_LMHEAD, k_argmax_rows<<<nr, 256, 0, st>>>(lg, V, argmax ? argmax + r0 : nullptr, argmax_pp, r0));
     }
   }
   return SNLP_OK;
 }
 
-static int embed_impl(snlp_model *m, cudaStream_t st, const int32_t *ids, int rows, float *h0) {
+static int embed_impl(snlp_model *m, cudaStream_t st, const int32_t *ids, int rows, float *h0, const int32_t *const *ids_pp) {
   const snlp_config &c = m->cfg;
   if (c.dtype == SNLP_DTYPE_BF16)
-    KLAUNCH(m, st, KC_OTHER, k_embed<__nv_bfloat16><<<rows, 128, 0, st>>>(ids, (const __nv_bfloat16 *)m->embed, h0, c.d_model, c.n_streams, c.vocab));
+    KLAUNCH(m, st, KC_OTHER, k_embed<__nv_bfloat16><<<rows, 128, 0, st>>>(ids, (const __nv_bfloat16 *)m->embed, h0, c.d_model, c.n_streams, c.vocab, ids_pp));
   else
-    KLAUNCH(m, st, KC_OTHER, k_embed<float><<<rows, 128, 0, st>>>(ids, (const float *)m->embed, h0, c.d_model, c.n_streams, c.vocab));
+    KLAUNCH(m, st, KC_OTHER, k_embed<float><<<rows, 128, 0, st>>>(ids, (const float *)m->embed, h0, c.d_model, c.n_streams, c.vocab, ids_pp));
   return SNLP_OK;
 }
 
@@ -942,6 +961,12 @@ static int embed_impl(snlp_model *m, cudaStream_t st, const int32_t *ids, int ro
 static int check_model(const snlp_model *m, const char *who) {
   if (!m) return fail(SNLP_ERR_ARG, "%s: NULL model handle", who);
   if (!m->loaded) return fail(SNLP_ERR_STATE, "%s: weights not loaded", who);
+  return SNLP_OK;
+}
+
+// The kernels read and write hidden states with 16-byte accesses; a misaligned pointer is turned away on the host.
+static int check_align16(const void *h0, const void *trace_out, const char *who) {
+  if ((uintptr_t)h0 % 16 || (uintptr_t)trace_out % 16) return fail(SNLP_ERR_ARG, "%s: hidden-state pointers must be 16-byte aligned", who);
   return SNLP_OK;
 }
 
@@ -957,6 +982,7 @@ static int check_shape(const snlp_model *m, int B, int T, const char *who) {
 extern "C" int snlp_embed(snlp_model *m, const int32_t *ids, int B, int T, float *h0, void *stream) {
   TRY(check_model(m, "snlp_embed"));
   if (!ids || !h0) return fail(SNLP_ERR_ARG, "snlp_embed: NULL pointer");
+  if ((uintptr_t)ids % 4 || (uintptr_t)h0 % 16) return fail(SNLP_ERR_ARG, "snlp_embed: ids must be 4-byte aligned, h0 16-byte aligned");
   TRY(check_shape(m, B, T, "snlp_embed"));
   return embed_impl(m, (cudaStream_t)stream, ids, B * T, h0);
 }
@@ -975,12 +1001,14 @@ static Fwd scratch_fwd(snlp_model *m, int B, int T, cudaStream_t st) {
 extern "C" int snlp_forward_sequential(snlp_model *m, const float *h0, int B, int T, float *trace_out, void *stream) {
   TRY(check_model(m, "snlp_forward_sequential"));
   if (!h0) return fail(SNLP_ERR_ARG, "snlp_forward_sequential: NULL h0");
+  TRY(check_align16(h0, trace_out, "snlp_forward_sequential"));
   TRY(check_shape(m, B, T, "snlp_forward_sequential"));
   cudaStream_t st = (cudaStream_t)stream;
   const size_t state = (size_t)B * T * m->cfg.n_streams * m->cfg.d_model;
   CU(cudaMemcpyAsync(m->trace, h0, state * 4, cudaMemcpyDeviceToDevice, st));
   Fwd f = scratch_fwd(m, B, T, st);
   TRY(sequential(m, f));
+  m->last_rows = B * T;
   if (trace_out) CU(cudaMemcpyAsync(trace_out, m->trace, (m->cfg.n_layer + 1) * state * 4, cudaMemcpyDeviceToDevice, st));
   return SNLP_OK;
 }
@@ -994,6 +1022,8 @@ extern "C" int snlp_forward_parallel(snlp_model *m, const float *h0, int B, int 
                                      void *stream) {
   TRY(check_model(m, "snlp_forward_parallel"));
   if (!h0) return fail(SNLP_ERR_ARG, "snlp_forward_parallel: NULL h0");
+  TRY(check_align16(h0, trace_out, "snlp_forward_parallel"));
+  if (resnorm_out && (uintptr_t)resnorm_out % 4) return fail(SNLP_ERR_ARG, "snlp_forward_parallel: resnorm_out must be 4-byte aligned");
   if (K < 1) return fail(SNLP_ERR_ARG, "snlp_forward_parallel: K must be >= 1 (got %d)", K);
   TRY(check_mode(mode, "snlp_forward_parallel"));
   TRY(check_shape(m, B, T, "snlp_forward_parallel"));
@@ -1002,6 +1032,7 @@ extern "C" int snlp_forward_parallel(snlp_model *m, const float *h0, int B, int 
   CU(cudaMemcpyAsync(m->trace, h0, state * 4, cudaMemcpyDeviceToDevice, st));
   Fwd f = scratch_fwd(m, B, T, st);
   TRY(parallel(m, f, K, mode, resnorm_out));
+  m->last_rows = B * T;
   if (trace_out) CU(cudaMemcpyAsync(trace_out, m->trace, (m->cfg.n_layer + 1) * state * 4, cudaMemcpyDeviceToDevice, st));
   return SNLP_OK;
 }
@@ -1010,6 +1041,7 @@ extern "C" int snlp_forward_solver(snlp_model *m, const float *h0, int B, int T,
                                    float *resnorm_out, void *stream) {
   TRY(check_model(m, "snlp_forward_solver"));
   if (!h0 || !solver) return fail(SNLP_ERR_ARG, "snlp_forward_solver: NULL pointer");
+  TRY(check_align16(h0, trace_out, "snlp_forward_solver"));
   TRY(check_solver(m, *solver, "snlp_forward_solver"));
   TRY(check_shape(m, B, T, "snlp_forward_solver"));
   cudaStream_t st = (cudaStream_t)stream;
@@ -1017,6 +1049,7 @@ extern "C" int snlp_forward_solver(snlp_model *m, const float *h0, int B, int T,
   CU(cudaMemcpyAsync(m->trace, h0, state * 4, cudaMemcpyDeviceToDevice, st));
   Fwd f = scratch_fwd(m, B, T, st);
   TRY(solve(m, f, *solver, resnorm_out));
+  m->last_rows = B * T;
   if (trace_out) CU(cudaMemcpyAsync(trace_out, m->trace, (m->cfg.n_layer + 1) * state * 4, cudaMemcpyDeviceToDevice, st));
   return SNLP_OK;
 }
@@ -1024,9 +1057,21 @@ extern "C" int snlp_forward_solver(snlp_model *m, const float *h0, int B, int T,
 extern "C" int snlp_lm_head(snlp_model *m, const float *hL, int rows, float *logits, int32_t *argmax, void *stream) {
   TRY(check_model(m, "snlp_lm_head"));
   if (!hL || (!logits && !argmax)) return fail(SNLP_ERR_ARG, "snlp_lm_head: NULL pointer");
+  if ((uintptr_t)hL % 16 || (uintptr_t)logits % 4 || (uintptr_t)argmax % 4) return fail(SNLP_ERR_ARG, "snlp_lm_head: hL must be 16-byte aligned, logits and argmax 4-byte aligned");
   if (rows < 1) return fail(SNLP_ERR_ARG, "snlp_lm_head: rows must be >= 1");
   if (rows > m->cfg.max_rows) return fail(SNLP_ERR_SHAPE, "snlp_lm_head: rows = %d exceeds max_rows = %d", rows, m->cfg.max_rows);
   return lm_head_impl(m, (cudaStream_t)stream, hL, (size_t)m->cfg.n_streams * m->cfg.d_model, rows, logits, argmax);
+}
+
+extern "C" int snlp_copy_trace(snlp_model *m, int rows, float *trace_out, void *stream) {
+  TRY(check_model(m, "snlp_copy_trace"));
+  if (!trace_out) return fail(SNLP_ERR_ARG, "snlp_copy_trace: NULL trace_out");
+  if ((uintptr_t)trace_out % 16) return fail(SNLP_ERR_ARG, "snlp_copy_trace: trace_out must be 16-byte aligned");
+  if (m->last_rows == 0) return fail(SNLP_ERR_STATE, "snlp_copy_trace: no forward, prefill or decode call has run on this handle yet");
+  if (rows != m->last_rows) return fail(SNLP_ERR_SHAPE, "snlp_copy_trace: rows = %d but the last call ran %d rows", rows, m->last_rows);
+  const size_t bytes = (size_t)(m->cfg.n_layer + 1) * rows * m->cfg.n_streams * m->cfg.d_model * sizeof(float);
+  CU(cudaMemcpyAsync(trace_out, m->trace, bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  return SNLP_OK;
 }
 
 extern "C" int snlp_kv_create(snlp_model *m, int B, int max_ctx, snlp_kv **out) {
@@ -1069,8 +1114,35 @@ extern "C" int snlp_kv_destroy(snlp_kv *kv) {
   return SNLP_OK;
 }
 
-extern "C" int snlp_kv_len(const snlp_kv *kv, int32_t *len) {
+// Make the host's mirror of the cache length exact again (it is only an upper bound after an asynchronous
+// draft-and-verify round): wait for the device and read the length it holds.
+static int kv_resolve(snlp_kv *kv) {
+  if (kv->len_known) return SNLP_OK;
+  CU(cudaDeviceSynchronize());
+  int len = 0;
+  CU(cudaMemcpy(&len, kv->pos, sizeof len, cudaMemcpyDeviceToHost));
+  kv->len = kv->len_hi = len;
+  kv->len_known = true;
+  return SNLP_OK;
+}
+
+// Room for `need` more positions?  Decided on the host's upper bound; when that bound is not exact and says no,
+// the exact length is fetched first.
+static int kv_room(snlp_kv *kv, int need, const char *who) {
+  if (kv->len_hi + need > kv->max_ctx && !kv->len_known) TRY(kv_resolve(kv));
+  if (kv->len_hi + need > kv->max_ctx)
+    return fail(SNLP_ERR_SHAPE, "%s: cache length %d + %d exceeds max_ctx %d", who, kv->len_hi, need, kv->max_ctx);
+  return SNLP_OK;
+}
+
+static void kv_advance(snlp_kv *kv, int n) {
+  kv->len_hi += n;
+  if (kv->len_known) kv->len = kv->len_hi;
+}
+
+extern "C" int snlp_kv_len(snlp_kv *kv, int32_t *len) {
   if (!kv || !len) return fail(SNLP_ERR_ARG, "snlp_kv_len: NULL argument");
+  TRY(kv_resolve(kv));
   *len = kv->len;
   return SNLP_OK;
 }
@@ -1078,12 +1150,16 @@ extern "C" int snlp_kv_len(const snlp_kv *kv, int32_t *len) {
 extern "C" int snlp_kv_truncate(snlp_kv *kv, int new_len, void *stream) {
   if (!kv) return fail(SNLP_ERR_ARG, "snlp_kv_truncate: NULL handle");
   if (!kv->m) return fail(SNLP_ERR_STATE, "snlp_kv_truncate: the model of this cache has been destroyed");
+  TRY(kv_resolve(kv));
   if (new_len < 0 || new_len > kv->len) return fail(SNLP_ERR_ARG, "snlp_kv_truncate: new_len = %d outside 0..%d", new_len, kv->len);
   KLAUNCH(kv->m, (cudaStream_t)stream, KC_OTHER, k_set_int<<<1, 1, 0, (cudaStream_t)stream>>>(kv->pos, new_len));
-  kv->len = new_len;
+  kv->len = kv->len_hi = new_len;
   return SNLP_OK;
 }
 
+// Geometry of a forward over T new positions per sequence against the cache.  pos_hi (which only sizes the split-KV
+// grid of the decode-regime attention) is the host's upper bound of the length: chunks that lie wholly beyond the
+// true length contribute exact zeros to the merge, so an overestimate changes no output bit.
 static Fwd kv_fwd(snlp_model *m, snlp_kv *kv, int T, cudaStream_t st) {
   Fwd f{};
   f.M = kv->B * T; f.B = kv->B; f.T = T;
@@ -1091,7 +1167,7 @@ static Fwd kv_fwd(snlp_model *m, snlp_kv *kv, int T, cudaStream_t st) {
   f.kv_bs = (size_t)kv->max_ctx * m->cfg.d_model;
   f.kv_ls = (size_t)kv->B * f.kv_bs;
   f.kv_rows = kv->max_ctx;
-  f.pos = kv->pos; f.pos_hi = kv->len; f.st = st;
+  f.pos = kv->pos; f.pos_hi = kv->len_hi; f.st = st;
   return f;
 }
 
@@ -1106,7 +1182,7 @@ extern "C" int snlp_prefill(snlp_model *m, snlp_kv *kv, const int32_t *ids, int 
   if (kv->m != m) return fail(SNLP_ERR_ARG, "snlp_prefill: cache belongs to another model");
   if (B < 1 || T < 1) return fail(SNLP_ERR_ARG, "snlp_prefill: B and T must be >= 1");
   if (B != kv->B) return fail(SNLP_ERR_SHAPE, "snlp_prefill: B = %d but the cache holds %d sequences", B, kv->B);
-  if (kv->len + T > kv->max_ctx) return fail(SNLP_ERR_SHAPE, "snlp_prefill: len %d + T %d exceeds max_ctx %d", kv->len, T, kv->max_ctx);
+  TRY(kv_room(kv, T, "snlp_prefill"));
   cudaStream_t st = (cudaStream_t)stream;
   const snlp_config &c = m->cfg;
   const int tc_max = c.max_rows / B;
@@ -1120,7 +1196,8 @@ extern "C" int snlp_prefill(snlp_model *m, snlp_kv *kv, const int32_t *ids, int 
     Fwd f = kv_fwd(m, kv, Tc, st);
     TRY(sequential(m, f));
     KLAUNCH(m, st, KC_OTHER, k_add_int<<<1, 1, 0, st>>>(kv->pos, Tc));
-    kv->len += Tc;
+    kv_advance(kv, Tc);
+    m->last_rows = B * Tc;
   }
   if (last_argmax) {
     const float *hL = m->trace + (size_t)c.n_layer * B * Tc * nd + (size_t)(Tc - 1) * nd;
@@ -1131,37 +1208,44 @@ extern "C" int snlp_prefill(snlp_model *m, snlp_kv *kv, const int32_t *ids, int 
 
 // greedy tokens of all `rows` rows of the forward that just ran (rows <= 16)
 // bump (nullable): device counter to advance by one after the tokens are out (done by the LM-head kernel itself on the tensor-core path)
-static int lm_head_tail(snlp_model *m, cudaStream_t st, int rows, int32_t *argmax, int *bump = nullptr) {
+static int lm_head_tail(snlp_model *m, cudaStream_t st, int rows, int32_t *argmax, int *bump = nullptr, int32_t *const *argmax_pp = nullptr) {
   const snlp_config &c = m->cfg;
   const size_t nd = (size_t)c.n_streams * c.d_model, L = c.n_layer;
   if (umma_path_ok(m) && rows <= kDecodeRows)  // the correction left the LM-head input in slot L of xb / ssq_x
     return lm_head_impl(m, st, nullptr, 0, rows, nullptr, argmax, (const __nv_bfloat16 *)m->xn + L * rows * c.d_model,
-                        m->ssq_x + L * (c.d_model / 128) * rows, bump);
-  TRY(lm_head_impl(m, st, m->trace + L * rows * nd, nd, rows, nullptr, argmax));
+                        m->ssq_x + L * (c.d_model / 128) * rows, bump, argmax_pp);
+  TRY(lm_head_impl(m, st, m->trace + L * rows * nd, nd, rows, nullptr, argmax, nullptr, nullptr, nullptr, argmax_pp));
   if (bump) KLAUNCH(m, st, KC_OTHER, k_add_int<<<1, 1, 0, st>>>(bump, 1));
   return SNLP_OK;
 }
 
-// enqueue one decode step (no graph handling, no host-side length update)
-static int decode_launches(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, const snlp_solver &sol, int32_t *tok_out, float *resnorm_out,
-                           cudaStream_t st) {
+// Enqueue one decode step (no graph handling, no host-side length update).  The step reads its input tokens and
+// writes its output tokens through the handle's device slot, so the launches -- and a graph captured from them --
+// do not depend on where the caller keeps its tokens.
+static int decode_launches(snlp_model *m, snlp_kv *kv, const snlp_solver &sol, float *resnorm_out, cudaStream_t st) {
   Fwd f = kv_fwd(m, kv, 1, st);
-  f.embed_ids = tok_in;
+  f.embed_ids_pp = (const int32_t *const *)m->tok_slot;
   TRY(solve(m, f, sol, resnorm_out));
-  TRY(lm_head_tail(m, st, kv->B, tok_out, kv->pos));   // also advances the cache position
+  TRY(lm_head_tail(m, st, kv->B, nullptr, kv->pos, (int32_t *const *)(m->tok_slot + 1)));   // also advances the cache position
   return SNLP_OK;
 }
 
 static int decode_step_impl(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, const snlp_solver &sol, int32_t *tok_out, float *resnorm_out,
                             cudaStream_t st) {
+  if (m->slot_in != tok_in || m->slot_out != tok_out) {   // point the slot at this call's buffers (stream-ordered)
+    KLAUNCH(m, st, KC_OTHER, k_set_ptrs<<<1, 1, 0, st>>>(m->tok_slot, tok_in, tok_out));
+    m->slot_in = tok_in;
+    m->slot_out = tok_out;
+  }
+  m->last_rows = kv->B;
   if (!m->use_graphs || m->timing) {
-    TRY(decode_launches(m, kv, tok_in, sol, tok_out, resnorm_out, st));
-    kv->len += 1;
+    TRY(decode_launches(m, kv, sol, resnorm_out, st));
+    kv_advance(kv, 1);
     return SNLP_OK;
   }
   const bool fast = fast_decode_ok(m, kv->B);
   const int chunk_len = attn_csub(kv->B * m->cfg.n_head) * kAttnSub;
-  GraphKey key{kv->B, sol.K, sol.mode, sol.prefix, sol.init, sol.fuse, fast ? kv->len / chunk_len + 1 : 0, tok_in, tok_out, resnorm_out, kv};
+  GraphKey key{kv->B, sol.K, sol.mode, sol.prefix, sol.init, sol.fuse, fast ? kv->len_hi / chunk_len + 1 : 0, resnorm_out, kv};
   auto it = m->graphs.find(key);
   if (it == m->graphs.end()) {
     if (m->graphs.size() >= 256) {
@@ -1172,7 +1256,7 @@ static int decode_step_impl(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, c
     CU(cudaStreamBeginCapture(m->cap_stream, cudaStreamCaptureModeThreadLocal));
     m->capturing = true;
     m->cap_nodes = 0;
-    const int rc = decode_launches(m, kv, tok_in, sol, tok_out, resnorm_out, m->cap_stream);
+    const int rc = decode_launches(m, kv, sol, resnorm_out, m->cap_stream);
     m->capturing = false;
     cudaError_t e = cudaStreamEndCapture(m->cap_stream, &graph);
     if (rc != SNLP_OK) {
@@ -1186,21 +1270,29 @@ static int decode_step_impl(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, c
     cudaGraphDestroy(graph);
     if (e != cudaSuccess) return fail(SNLP_ERR_CUDA, "cudaGraphInstantiate failed: %s", cudaGetErrorString(e));
     it = m->graphs.emplace(key, ge).first;
+    m->graph_captures += 1;
   }
   CU(cudaGraphLaunch(it->second.exec, st));
   m->launches += it->second.nodes;
-  kv->len += 1;
+  kv_advance(kv, 1);
+  return SNLP_OK;
+}
+
+static int check_token_ptrs(const int32_t *tok_in, const int32_t *tok_out, const char *who) {
+  if (!tok_in || !tok_out) return fail(SNLP_ERR_ARG, "%s: NULL pointer", who);
+  if ((uintptr_t)tok_in % 4 || (uintptr_t)tok_out % 4) return fail(SNLP_ERR_ARG, "%s: token pointers must be 4-byte aligned", who);
   return SNLP_OK;
 }
 
 extern "C" int snlp_decode_step(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, int K, int mode, int32_t *tok_out, float *resnorm_out,
                                 void *stream) {
   TRY(check_model(m, "snlp_decode_step"));
-  if (!kv || !tok_in || !tok_out) return fail(SNLP_ERR_ARG, "snlp_decode_step: NULL pointer");
+  if (!kv) return fail(SNLP_ERR_ARG, "snlp_decode_step: NULL pointer");
+  TRY(check_token_ptrs(tok_in, tok_out, "snlp_decode_step"));
   if (kv->m != m) return fail(SNLP_ERR_ARG, "snlp_decode_step: cache belongs to another model");
   if (K < 0) return fail(SNLP_ERR_ARG, "snlp_decode_step: K must be >= 0 (got %d)", K);
   TRY(check_mode(mode, "snlp_decode_step"));
-  if (kv->len + 1 > kv->max_ctx) return fail(SNLP_ERR_SHAPE, "snlp_decode_step: cache is full (len %d, max_ctx %d)", kv->len, kv->max_ctx);
+  TRY(kv_room(kv, 1, "snlp_decode_step"));
   const snlp_solver sol = K == 0 ? snlp_solver{0, SNLP_MODE_SEQUENTIAL, m->cfg.n_layer, SNLP_INIT_H0, 1} : snlp_solver{K, mode, 0, SNLP_INIT_H0, 1};
   return decode_step_impl(m, kv, tok_in, sol, tok_out, K > 0 ? resnorm_out : nullptr, (cudaStream_t)stream);
 }
@@ -1222,43 +1314,71 @@ extern "C" int snlp_decode_step_host(snlp_model *m, snlp_kv *kv, const int32_t *
 extern "C" int snlp_decode_step_solver(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, const snlp_solver *solver, int32_t *tok_out,
                                        float *resnorm_out, void *stream) {
   TRY(check_model(m, "snlp_decode_step_solver"));
-  if (!kv || !tok_in || !tok_out || !solver) return fail(SNLP_ERR_ARG, "snlp_decode_step_solver: NULL pointer");
+  if (!kv || !solver) return fail(SNLP_ERR_ARG, "snlp_decode_step_solver: NULL pointer");
+  TRY(check_token_ptrs(tok_in, tok_out, "snlp_decode_step_solver"));
   if (kv->m != m) return fail(SNLP_ERR_ARG, "snlp_decode_step_solver: cache belongs to another model");
   TRY(check_solver(m, *solver, "snlp_decode_step_solver"));
-  if (kv->len + 1 > kv->max_ctx) return fail(SNLP_ERR_SHAPE, "snlp_decode_step_solver: cache is full (len %d, max_ctx %d)", kv->len, kv->max_ctx);
+  TRY(kv_room(kv, 1, "snlp_decode_step_solver"));
   return decode_step_impl(m, kv, tok_in, *solver, tok_out, solver->K > 0 ? resnorm_out : nullptr, (cudaStream_t)stream);
+}
+
+// One draft-and-verify round, everything enqueued on the stream; the round's first position and the number of accepted
+// drafts stay on the device.  On return the host knows the cache length only up to len_hi (every draft accepted).
+static int draft_and_verify_launches(snlp_model *m, snlp_kv *kv, int32_t *last_tok, int block, int K, int mode, int32_t *emitted,
+                                     int32_t *n_emitted, int32_t *n_accepted, cudaStream_t st, const char *who) {
+  TRY(check_model(m, who));
+  if (!kv || !last_tok || !emitted || !n_emitted || !n_accepted) return fail(SNLP_ERR_ARG, "%s: NULL pointer", who);
+  if ((uintptr_t)last_tok % 4 || (uintptr_t)emitted % 4 || (uintptr_t)n_emitted % 4 || (uintptr_t)n_accepted % 4)
+    return fail(SNLP_ERR_ARG, "%s: int32 pointers must be 4-byte aligned", who);
+  if (kv->m != m) return fail(SNLP_ERR_ARG, "%s: cache belongs to another model", who);
+  if (block < 1) return fail(SNLP_ERR_ARG, "%s: block must be >= 1", who);
+  if (K < 1) return fail(SNLP_ERR_ARG, "%s: K must be >= 1", who);
+  TRY(check_mode(mode, who));
+  if (kv->B != 1) return fail(SNLP_ERR_SHAPE, "%s: batch must be 1 (cache holds %d)", who, kv->B);
+  if (block + 1 > m->cfg.max_rows) return fail(SNLP_ERR_SHAPE, "%s: block+1 exceeds max_rows", who);
+  TRY(kv_room(kv, block + 1, who));
+  const snlp_config &c = m->cfg;
+  const int hi0 = kv->len_hi;
+  int32_t *ids = m->spec;                          // [block+1]: last_tok, x_1..x_block
+  int32_t *y = m->spec + (c.max_rows + 1);         // [block+1]: verifier tokens
+  CU(cudaMemcpyAsync(ids, last_tok, 4, cudaMemcpyDeviceToDevice, st));
+  KLAUNCH(m, st, KC_OTHER, k_copy_int<<<1, 1, 0, st>>>(kv->pos + 1, kv->pos));   // remember where the round began
+  const snlp_solver draft{K, mode, 0, SNLP_INIT_H0, 1};
+  for (int i = 0; i < block; ++i) TRY(decode_step_impl(m, kv, ids + i, draft, ids + i + 1, nullptr, st));
+  KLAUNCH(m, st, KC_OTHER, k_copy_int<<<1, 1, 0, st>>>(kv->pos, kv->pos + 1));   // back to the round's first position
+  kv->len_hi = hi0;
+  if (kv->len_known) kv->len = hi0;
+  TRY(embed_impl(m, st, ids, block + 1, m->trace));
+  Fwd f = kv_fwd(m, kv, block + 1, st);
+  f.pos_hi = hi0;
+  TRY(sequential(m, f));
+  m->last_rows = block + 1;
+  TRY(lm_head_tail(m, st, block + 1, y));
+  KLAUNCH(m, st, KC_OTHER, k_accept<<<1, 32, 0, st>>>(ids + 1, y, block, emitted, n_emitted, n_accepted, last_tok, kv->pos, kv->pos + 1));
+  kv->len_hi = hi0 + block + 1;   // the most the round can have kept
+  kv->len_known = false;
+  return SNLP_OK;
+}
+
+extern "C" int snlp_draft_and_verify_async(snlp_model *m, snlp_kv *kv, int32_t *last_tok, int block, int K, int mode, int32_t *emitted,
+                                           int32_t *n_emitted, int32_t *n_accepted, void *stream) {
+  return draft_and_verify_launches(m, kv, last_tok, block, K, mode, emitted, n_emitted, n_accepted, (cudaStream_t)stream,
+                                   "snlp_draft_and_verify_async");
 }
 
 extern "C" int snlp_draft_and_verify(snlp_model *m, snlp_kv *kv, int32_t *last_tok, int block, int K, int mode, int32_t *emitted,
                                      int32_t *n_emitted, int32_t *n_accepted, void *stream) {
-  TRY(check_model(m, "snlp_draft_and_verify"));
-  if (!kv || !last_tok || !emitted || !n_emitted || !n_accepted) return fail(SNLP_ERR_ARG, "snlp_draft_and_verify: NULL pointer");
-  if (kv->m != m) return fail(SNLP_ERR_ARG, "snlp_draft_and_verify: cache belongs to another model");
-  if (block < 1) return fail(SNLP_ERR_ARG, "snlp_draft_and_verify: block must be >= 1");
-  if (K < 1) return fail(SNLP_ERR_ARG, "snlp_draft_and_verify: K must be >= 1");
-  TRY(check_mode(mode, "snlp_draft_and_verify"));
-  if (kv->B != 1) return fail(SNLP_ERR_SHAPE, "snlp_draft_and_verify: batch must be 1 (cache holds %d)", kv->B);
-  if (block + 1 > m->cfg.max_rows) return fail(SNLP_ERR_SHAPE, "snlp_draft_and_verify: block+1 exceeds max_rows");
-  if (kv->len + block + 1 > kv->max_ctx) return fail(SNLP_ERR_SHAPE, "snlp_draft_and_verify: len %d + block+1 exceeds max_ctx %d", kv->len, kv->max_ctx);
-  cudaStream_t st = (cudaStream_t)stream;
-  const snlp_config &c = m->cfg;
-  const int len0 = kv->len;
-  int32_t *ids = m->spec;                          // [block+1]: last_tok, x_1..x_block
-  int32_t *y = m->spec + (c.max_rows + 1);         // [block+1]: verifier tokens
-  CU(cudaMemcpyAsync(ids, last_tok, 4, cudaMemcpyDeviceToDevice, st));
-  const snlp_solver draft{K, mode, 0, SNLP_INIT_H0, 1};
-  for (int i = 0; i < block; ++i) TRY(decode_step_impl(m, kv, ids + i, draft, ids + i + 1, nullptr, st));
-  KLAUNCH(m, st, KC_OTHER, k_set_int<<<1, 1, 0, st>>>(kv->pos, len0));
-  kv->len = len0;
-  TRY(embed_impl(m, st, ids, block + 1, m->trace));
-  Fwd f = kv_fwd(m, kv, block + 1, st);
-  TRY(sequential(m, f));
-  const size_t nd = (size_t)c.n_streams * c.d_model;
-  TRY(lm_head_tail(m, st, block + 1, y));
-  KLAUNCH(m, st, KC_OTHER, k_accept<<<1, 32, 0, st>>>(ids + 1, y, block, emitted, n_emitted, n_accepted, last_tok, kv->pos, len0));
-  int32_t n = 0;
-  CU(cudaMemcpyAsync(&n, n_accepted, 4, cudaMemcpyDeviceToHost, st));
-  CU(cudaStreamSynchronize(st));
-  kv->len = len0 + n + 1;
+  TRY(draft_and_verify_launches(m, kv, last_tok, block, K, mode, emitted, n_emitted, n_accepted, (cudaStream_t)stream, "snlp_draft_and_verify"));
+  int len = 0;   // the convenience form: wait for the round and bring the cache length back to the host
+  CU(cudaMemcpyAsync(&len, kv->pos, sizeof len, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+  CU(cudaStreamSynchronize((cudaStream_t)stream));
+  kv->len = kv->len_hi = len;
+  kv->len_known = true;
+  return SNLP_OK;
+}
+
+extern "C" int snlp_graph_count(const snlp_model *m, int64_t *captured) {
+  if (!m || !captured) return fail(SNLP_ERR_ARG, "snlp_graph_count: NULL argument");
+  *captured = m->graph_captures;
   return SNLP_OK;
 }

@@ -57,7 +57,8 @@ struct UmmaParams {
   float *logits; float *pm_val; int *pm_idx;                            // UEPI_LMHEAD
   // UEPI_LMHEAD, optional: the CTA that finishes last merges the per-tile maxima into argmax[M] (ties -> lowest
   // index) and then adds one to *bump (nullable).  lm_counter: zero on entry, left zero.
-  int32_t *argmax; int *bump; unsigned *lm_counter;
+  // argmax_pp (nullable): the address of argmax is read from a device slot instead (replayed decode graphs).
+  int32_t *argmax; int *bump; unsigned *lm_counter; int32_t *const *argmax_pp;
 };
 
 constexpr int kUmmaThreads = 320;   // warp 0: TMA, warp 1: MMA + TMEM allocation, warps 2-9: epilogue (two per TMEM lane quarter)
@@ -632,7 +633,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
         epi_bar_sync();  // outs is reused by the next item
       }
     }
-    if (EPI == UEPI_LMHEAD && AM != kUmmaBM && p.argmax != nullptr) {
+    if (EPI == UEPI_LMHEAD && AM != kUmmaBM && (p.argmax != nullptr || p.argmax_pp != nullptr)) {
       // Greedy token: every CTA counts itself in once its partial maxima are out (also after a wait that ran out,
       // so that the counter always returns to zero); the last one merges the tiles.
       int *s_last = reinterpret_cast<int *>(outs);
@@ -642,6 +643,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
       epi_bar_sync();
       if (*s_last) {
         __threadfence();
+        int32_t *amax = p.argmax_pp != nullptr ? *p.argmax_pp : p.argmax;
         for (int tok = ew; tok < p.M; tok += 8) {
           float bv = -INFINITY;
           int bi = 0x7fffffff;
@@ -656,7 +658,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
             const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
             if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
           }
-          if (lane == 0) p.argmax[tok] = (unsigned)bi < (unsigned)p.N ? bi : 0;
+          if (lane == 0) amax[tok] = (unsigned)bi < (unsigned)p.N ? bi : 0;
         }
         if (et == 0) {
           if (p.bump != nullptr) *p.bump += 1;

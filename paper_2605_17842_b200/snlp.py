@@ -25,6 +25,7 @@ EXPORTS = [
     "snlp_forward_parallel", "snlp_forward_solver", "snlp_decode_step_solver", "snlp_lm_head", "snlp_kv_create", "snlp_kv_destroy", "snlp_kv_len",
     "snlp_kv_truncate", "snlp_prefill", "snlp_decode_step", "snlp_decode_step_host", "snlp_draft_and_verify", "snlp_set_flag",
     "snlp_launch_count", "snlp_kernel_times", "snlp_device_status", "snlp_lm_head_greedy_static", "snlp_last_error",
+    "snlp_copy_trace", "snlp_draft_and_verify_async", "snlp_graph_count",
 ]
 
 
@@ -238,6 +239,31 @@ class Model:
                                           _stream()))
         n_emit, n_acc = counts.tolist()
         return emitted[:n_emit].tolist(), n_acc
+
+    def draft_and_verify_async(self, kv: KVCache, last_tok: torch.Tensor, block: int, K: int, mode: int = MODE_IDN,
+                               emitted: torch.Tensor | None = None, counts: torch.Tensor | None = None):
+        """One round with no host synchronisation.  Returns (emitted [block+1] int32, counts [2] int32 =
+        (n_emitted, n_accepted)), both still on the device; last_tok is updated in place."""
+        dev = last_tok.device
+        if emitted is None:
+            emitted = torch.empty((block + 1,), dtype=torch.int32, device=dev)
+        if counts is None:
+            counts = torch.zeros((2,), dtype=torch.int32, device=dev)
+        _check(_lib.snlp_draft_and_verify_async(self._h, kv._h, _ptr(last_tok), C.c_int(block), C.c_int(K), C.c_int(mode),
+                                                _ptr(emitted), C.c_void_p(counts.data_ptr()), C.c_void_p(counts.data_ptr() + 4),
+                                                _stream()))
+        return emitted, counts
+
+    def copy_trace(self, rows: int) -> torch.Tensor:
+        """The states [L+1, rows, n, d] of the handle's last forward / prefill chunk / decode step / verify block."""
+        tr = torch.empty((self.n_layer + 1, rows, self.n_streams, self.d_model), dtype=torch.float32, device="cuda")
+        _check(_lib.snlp_copy_trace(self._h, C.c_int(rows), _ptr(tr), _stream()))
+        return tr
+
+    def graph_count(self) -> int:
+        n = C.c_int64()
+        _check(_lib.snlp_graph_count(self._h, C.byref(n)))
+        return n.value
 
     # -- misc -------------------------------------------------------------------------------------
     def set_flag(self, flag: int, value: int):

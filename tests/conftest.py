@@ -10,6 +10,7 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); run with -m gpu")
+    config.addinivalue_line("markers", "slow: the oracle side takes tens of seconds of fp64 work; deselect with -m 'gpu and not slow'")
 
 
 def pytest_collection_modifyitems(config, items):

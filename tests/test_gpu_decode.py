@@ -25,9 +25,14 @@ def oracle_kv(cfg, B, ctx):
     return O.LayerKV(cfg.n_layer, B, ctx, cfg.n_head, cfg.head_dim)
 
 
+# relative state error the comparisons allow for: what the kernels are observed to stay within (bf16 paths 1.4-2.7e-3
+# on every parity case), not the 2e-2 acceptance bound, so that a wrong token cannot hide behind the tolerance
+STATE_ERR = {"fp32": 1e-5, "bf16": 5e-3}
+
+
 def margin_tau(cfg, W):
-    # |logit error| <= tol * ||x_norm|| * ||w_row||, for the two logits being compared
-    return 2.0 * TOL[cfg.dtype] * math.sqrt(cfg.d_model) * float(np.max(np.linalg.norm(W.lm_head.astype(np.float64), axis=1)))
+    # |logit error| <= state error * ||x_norm|| * ||w_row||, for the two logits being compared
+    return 2.0 * STATE_ERR[cfg.dtype] * math.sqrt(cfg.d_model) * float(np.max(np.linalg.norm(W.lm_head.astype(np.float64), axis=1)))
 
 
 @pytest.mark.parametrize("cfg,K", [(F32, 0), (F32, 2), (F32_HC, 0), (F32_HC, 2)])

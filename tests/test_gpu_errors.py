@@ -95,3 +95,93 @@ def test_cache_may_outlive_its_model(env):
         kv.truncate(1)
     assert e.value.code == snlp.ERR_STATE
     kv.close()                       # ... then the cache: must not touch the freed model
+
+
+def test_injected_device_error_is_reported_once(env):
+    """Failure detection without a GPU fault: the host writes the error word that a kernel raises when a bounded
+    wait expires; snlp_device_status must report SNLP_ERR_TIMEOUT for it exactly once and the handle keeps working."""
+    snlp, cfg, W = env
+    m = snlp.Model(cfg, max_rows=16, max_batch=1, max_ctx=16)
+    m.load_weights(W)
+    h0 = torch.from_numpy(synth.make_hidden(cfg, 1, 16, seed=3)).cuda()
+    before = m.forward_sequential(h0)
+    m.device_status()                       # healthy
+    m.set_flag(3, 1)                        # inject
+    with pytest.raises(snlp.SnlpError) as e:
+        m.device_status()
+    assert e.value.code == snlp.ERR_TIMEOUT and "bounded wait" in str(e.value)
+    m.device_status()                       # cleared by the report
+    m.set_flag(3, 1)
+    m.set_flag(3, 0)                        # the hook can also take it back
+    m.device_status()
+    after = m.forward_sequential(h0)
+    assert torch.equal(before, after)
+    m.close()
+
+
+def test_misaligned_pointers_are_rejected_on_the_host(env):
+    snlp, cfg, W = env
+    lib = snlp.raw_library()
+    m = snlp.Model(cfg, max_rows=16, max_batch=1, max_ctx=16)
+    m.load_weights(W)
+    buf = torch.zeros((16 * 64 + 8,), device="cuda")
+    tr = torch.zeros((5 * 16 * 64 + 8,), device="cuda")
+    odd = C.c_void_p(buf.data_ptr() + 4)    # 4-byte aligned only
+    ok = C.c_void_p(buf.data_ptr())
+    assert lib.snlp_forward_sequential(m._h, odd, 1, 16, None, None) == snlp.ERR_ARG
+    assert b"aligned" in lib.snlp_last_error()
+    assert lib.snlp_forward_sequential(m._h, ok, 1, 16, C.c_void_p(tr.data_ptr() + 8), None) == snlp.ERR_ARG
+    assert lib.snlp_forward_parallel(m._h, odd, 1, 16, 1, 0, None, None, None) == snlp.ERR_ARG
+    assert lib.snlp_lm_head(m._h, odd, 1, None, ok, None) == snlp.ERR_ARG
+    ids = torch.zeros((8,), dtype=torch.int32, device="cuda")
+    kv = m.kv_cache(1, 16)
+    assert lib.snlp_decode_step(m._h, kv._h, C.c_void_p(ids.data_ptr() + 2), 0, 0, C.c_void_p(ids.data_ptr()), None, None) == snlp.ERR_ARG
+    assert lib.snlp_copy_trace(m._h, 1, None, None) == snlp.ERR_ARG
+    assert lib.snlp_copy_trace(m._h, 1, ok, None) == snlp.ERR_STATE       # nothing has run on this handle yet
+    m.forward_sequential(buf[:16 * 64].view(1, 16, 1, 64))
+    assert lib.snlp_copy_trace(m._h, 3, C.c_void_p(tr.data_ptr()), None) == snlp.ERR_SHAPE
+    assert lib.snlp_copy_trace(m._h, 16, C.c_void_p(tr.data_ptr()), None) == snlp.OK
+    lm = torch.zeros((128 * 32 + 8,), dtype=torch.int16, device="cuda")
+    out = torch.zeros((4,), dtype=torch.int32, device="cuda")
+    rc = lib.snlp_lm_head_greedy_static(C.c_void_p(buf.data_ptr() + 4), C.c_void_p(lm.data_ptr()), 1, 1, 32, 128, C.c_float(1e-6),
+                                        C.c_void_p(out.data_ptr()), None)
+    assert rc == snlp.ERR_ARG
+    rc = lib.snlp_lm_head_greedy_static(C.c_void_p(buf.data_ptr()), C.c_void_p(lm.data_ptr() + 2), 1, 1, 32, 128, C.c_float(1e-6),
+                                        C.c_void_p(out.data_ptr()), None)
+    assert rc == snlp.ERR_ARG
+    torch.cuda.synchronize()
+    kv.close()
+    m.close()
+
+
+def test_decode_graphs_are_not_keyed_on_the_token_buffers():
+    """300 steps, each with a fresh output tensor (what a plain caller of the binding does): one captured graph per
+    attention grid size, not one per step, and the same tokens as with one fixed buffer."""
+    from paper_2605_17842_b200 import snlp
+    cfg = synth.ModelConfig(2, 256, 2, 128, 512, 1024, 1, "bf16")
+    W = synth.make_weights(cfg, seed=1234, std=0.05, embed_std=1.0)
+    m = snlp.Model(cfg, max_rows=16, max_batch=1, max_ctx=400)
+    m.load_weights(W)
+    ids = torch.from_numpy(synth.make_ids(cfg, 1, 16, seed=2)).cuda()
+    kv = m.kv_cache(1, 400)
+    t0 = m.prefill(kv, ids)
+    keep = []                                # hold every tensor so the allocator must hand out new addresses
+    t = t0
+    for _ in range(300):
+        t = m.decode_step(kv, t, 2)
+        keep.append(t)
+    torch.cuda.synchronize()
+    assert len({x.data_ptr() for x in keep}) == 300
+    chunks = (16 + 300 - 1) // 256 + 1       # 256-key chunks of the split-KV attention (2 heads x 1 sequence)
+    assert m.graph_count() == chunks, m.graph_count()
+    fresh = torch.stack(keep).flatten().tolist()
+    kv.truncate(16)
+    t = t0.clone()
+    fixed = []
+    for _ in range(300):
+        m.decode_step(kv, t, 2, tok_out=t)
+        fixed.append(int(t.item()))
+    assert m.graph_count() == chunks
+    assert fresh == fixed
+    m.device_status()
+    m.close()

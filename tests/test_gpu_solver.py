@@ -6,7 +6,7 @@ import torch
 
 from oracle import snlp_oracle as O
 from paper_2605_17842_b200 import synth
-from tests.gpu_util import TOL, dev, layer_relerr, make_model
+from tests.gpu_util import TOL, dev, layer_relerr, make_model, trace_err
 
 pytestmark = pytest.mark.gpu
 
@@ -30,7 +30,7 @@ def test_prefix_and_fwd_init_match_oracle(name):
     for S, init, K in [(2, O.INIT_H0, 1), (2, O.INIT_FWD, 1), (0, O.INIT_FWD, 2), (3, O.INIT_H0, 2), (0, O.INIT_FWD, 0)]:
         want, want_res = O.forward_snlp(cfg, W, h0.astype(np.float64), K, mode, S=S, init=init)
         tr, rn = m.forward_solver(dev(h0), snlp.Solver(K=K, mode=mode, prefix=S, init=init))
-        assert layer_relerr(tr.cpu().numpy(), want) <= TOL[cfg.dtype], (S, init, K)
+        assert trace_err(tr.cpu().numpy(), want, TOL[cfg.dtype]) <= TOL[cfg.dtype], (S, init, K)
         if K > 0:
             gr, wr = np.sqrt(rn.cpu().numpy()[:K, :, 0]), np.sqrt(want_res[..., 0])
             scale = np.sqrt(want_res[..., 1]).max() + 1e-30
@@ -120,11 +120,11 @@ def test_fused_chunks_match_oracle(name):
         tr, _ = m.forward_solver(dev(h0), snlp.Solver(K=K, mode=O.MODE_IDN, prefix=S, init=init, fuse=F))
         got = tr.cpu().numpy()[S::F]
         assert got.shape[0] == len(want)
-        assert layer_relerr(got, np.stack(want)) <= TOL[cfg.dtype], (S, F, K, init)
+        assert trace_err(got, np.stack(want), TOL[cfg.dtype]) <= TOL[cfg.dtype], (S, F, K, init)
         # sequential execution of the same fused model, and chunkwise finite-step exactness against it (bit for bit)
         fseq_want = O.forward_chunked(cfg, W, h0.astype(np.float64), None, F, S=S)
         fseq, _ = m.forward_solver(dev(h0), snlp.Solver(K=0, mode=snlp.MODE_SEQUENTIAL, prefix=S, fuse=F))
-        assert layer_relerr(fseq.cpu().numpy()[S::F], np.stack(fseq_want)) <= TOL[cfg.dtype], (S, F)
+        assert trace_err(fseq.cpu().numpy()[S::F], np.stack(fseq_want), TOL[cfg.dtype]) <= TOL[cfg.dtype], (S, F)
         nexact = min((L - S) // F, K + (1 if init == O.INIT_FWD else 0))
         assert torch.equal(tr[S::F][:nexact + 1], fseq[S::F][:nexact + 1]), (S, F, K, init)
     # fuse = 1 through the same entry point is the unfused algorithm
@@ -134,7 +134,7 @@ def test_fused_chunks_match_oracle(name):
     # without correction (A = 0) information moves one chunk per sweep
     want = O.forward_chunked(cfg, W, h0.astype(np.float64), 1, 2, correct=False)
     tr, _ = m.forward_solver(dev(h0), snlp.Solver(K=1, mode=O.MODE_NOCORR, fuse=2))
-    assert layer_relerr(tr.cpu().numpy()[0::2], np.stack(want)) <= TOL[cfg.dtype]
+    assert trace_err(tr.cpu().numpy()[0::2], np.stack(want), TOL[cfg.dtype]) <= TOL[cfg.dtype]
     m.device_status()
 
 
