@@ -90,6 +90,13 @@ def make_weights(cfg: ModelConfig, seed: int = 1234, mix_seed: int = 5, std: flo
     W.wo = normal((L, d, d), std * out_scale)
     W.wup = normal((L, ff, d), std)
     W.wdn = normal((L, d, ff), std * out_scale)
+    _add_mixing(W, cfg, mix_seed)
+    return W
+
+
+def _add_mixing(W: SimpleNamespace, cfg: ModelConfig, mix_seed: int) -> None:
+    """The stream-mixing maps of an n-stream model (their own generator: they do not depend on the dense weights)."""
+    L, n = cfg.n_layer, cfg.n_streams
     if n > 1:
         mrng = np.random.Generator(np.random.Philox(mix_seed))
         W.hc_res_attn = sinkhorn(mrng.standard_normal((L, n, n))).astype(np.float32)
@@ -106,7 +113,24 @@ def make_weights(cfg: ModelConfig, seed: int = 1234, mix_seed: int = 5, std: flo
     else:
         W.hc_res_attn = W.hc_res_mlp = None
         W.hc_pre_attn = W.hc_pre_mlp = W.hc_post_attn = W.hc_post_mlp = None
-    return W
+
+
+def with_mixing(W: SimpleNamespace, cfg: ModelConfig, mix_seed: int = 5) -> SimpleNamespace:
+    """The weights make_weights(cfg, same seed, mix_seed) would return, built from an already generated set `W` of a
+    model with the same dense shapes (the dense arrays are shared, not copied; only the mixing maps are drawn)."""
+    out = SimpleNamespace(**{k: getattr(W, k) for k in ("embed", "lm_head", "wqkv", "wo", "wup", "wdn")})
+    _add_mixing(out, cfg, mix_seed)
+    return out
+
+
+def with_embed_std(W: SimpleNamespace, cfg: ModelConfig, seed: int, embed_std: float) -> SimpleNamespace:
+    """The weights make_weights(cfg, seed, embed_std=embed_std) would return, built from `W` = make_weights(cfg, seed):
+    the embedding is the generator's first draw, so only it is drawn again, at the new scale."""
+    rng = np.random.Generator(np.random.Philox(seed))
+    e = rng.standard_normal((cfg.vocab, cfg.d_model), dtype=np.float32) * np.float32(embed_std)
+    out = SimpleNamespace(**vars(W))
+    out.embed = round_to_bf16(e) if cfg.dtype == "bf16" else e
+    return out
 
 
 def make_ids(cfg: ModelConfig, B: int, T: int, seed: int = 1) -> np.ndarray:
