@@ -18,6 +18,7 @@
 #include "generic.cuh"
 #include "umma_gemm.cuh"
 #include "umma_gemm2.cuh"
+#include "umma_gemv.cuh"
 #include "attn_umma.cuh"
 
 using namespace snlp;
@@ -57,7 +58,6 @@ void set_last_error(const char *msg) { g_err = msg; }  // for the library's othe
 // ------------------------------------------------------------------------------------------------
 // handles
 constexpr size_t kCorrExtraSmem = 32768;   // k_correct: shared memory beyond the operand ring (norm partials, staged coefficients)
-constexpr int kMaxSplits = 4;    // K-splits of the partial-sum GEMV outputs
 constexpr int kDecodeRows = 16;  // largest row count served by the decode-regime kernels
 constexpr size_t kCorrSmallSmem = 160 * 1024;
 
@@ -97,6 +97,9 @@ struct snlp_model {
   unsigned *counter = nullptr, *attn_counters = nullptr;
   int *zero = nullptr;
   unsigned *lm_counter = nullptr;   // arrival counter of the LM-head launch (zero between launches)
+  float *gemv_part = nullptr;       // decode-regime products: pieces of tiles split between CTAs
+  unsigned *gemv_ctr = nullptr;     // their arrival counters, one per CTA (zero between launches)
+  size_t gemv_ctr_bytes = 0;
   int32_t *spec = nullptr;  // [2 * (max_rows + 1)] ids / verifier tokens for draft-and-verify
   int32_t *tok_pin = nullptr, *tok_dev = nullptr;   // [2][max_batch] mapped pinned host memory (tokens in, tokens out) and its device address (snlp_decode_step_host)
   int logit_rows = 0;
@@ -261,8 +264,7 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
     A(&m->xm, L * R * d * 4);
   }
   A(&m->qkv_raw, L * R * 3 * d * 4);
-  // the decode-regime kernels write up to kMaxSplits partial sums for at most kDecodeRows rows
-  const size_t split_rows = std::max<size_t>(R, (size_t)kMaxSplits * std::min<size_t>(R, kDecodeRows));
+  const size_t split_rows = R;
   A(&m->a, L * split_rows * d * 4);
   A(&m->y_raw, L * R * ff * 4);
   A(&m->mb, L * split_rows * d * 4);
@@ -293,6 +295,14 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
   A(&m->attn_counters, L * (size_t)kDecodeRows * c.n_head * 4);
   A(&m->zero, 16);
   A(&m->lm_counter, 16);
+  {
+    cudaDeviceProp prop;
+    if (rc == SNLP_OK && cudaGetDeviceProperties(&prop, m->device) == cudaSuccess) m->n_sm = prop.multiProcessorCount;
+    const size_t rows = std::min<size_t>(R, kDecodeRows);
+    A(&m->gemv_part, (size_t)m->n_sm * kGemvMaxSlices * rows * 256 * sizeof(float));
+    m->gemv_ctr_bytes = (size_t)(m->n_sm + 1) * sizeof(unsigned);
+    A(&m->gemv_ctr, m->gemv_ctr_bytes);
+  }
   A(&m->spec, 2 * (R + 1) * 4);
   A(&m->tok_slot, 2 * sizeof(void *));
   if (rc == SNLP_OK && (cudaHostAlloc((void **)&m->tok_pin, (size_t)2 * c.max_batch * 4, cudaHostAllocMapped) != cudaSuccess ||
@@ -301,7 +311,7 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
     rc = fail(SNLP_ERR_OOM, "cudaHostAlloc of the token staging buffer failed");
   }
   if (rc == SNLP_OK) {
-    if (cudaMemset(m->dev_err, 0, 16) != cudaSuccess || cudaMemset(m->attn_counters, 0, L * (size_t)kDecodeRows * c.n_head * 4) != cudaSuccess || cudaMemset(m->counter, 0, 16) != cudaSuccess || cudaMemset(m->zero, 0, 16) != cudaSuccess || cudaMemset(m->lm_counter, 0, 16) != cudaSuccess)
+    if (cudaMemset(m->dev_err, 0, 16) != cudaSuccess || cudaMemset(m->attn_counters, 0, L * (size_t)kDecodeRows * c.n_head * 4) != cudaSuccess || cudaMemset(m->counter, 0, 16) != cudaSuccess || cudaMemset(m->zero, 0, 16) != cudaSuccess || cudaMemset(m->lm_counter, 0, 16) != cudaSuccess || cudaMemset(m->gemv_ctr, 0, m->gemv_ctr_bytes) != cudaSuccess)
       rc = fail(SNLP_ERR_CUDA, "cudaMemset failed");
   }
   if (rc == SNLP_OK) {
@@ -465,6 +475,11 @@ extern "C" int snlp_device_status(snlp_model *m, void *stream) {
   CU(cudaMemcpy(&flag, m->dev_err, sizeof flag, cudaMemcpyDeviceToHost));
   if (flag) {
     cudaMemset(m->dev_err, 0, sizeof flag);
+    // a kernel that gave up may have left arrival counters part-way: bring them back to zero for the calls that follow
+    cudaMemset(m->gemv_ctr, 0, m->gemv_ctr_bytes);
+    cudaMemset(m->lm_counter, 0, 16);
+    cudaMemset(m->counter, 0, 16);
+    cudaMemset(m->attn_counters, 0, (size_t)m->cfg.n_layer * kDecodeRows * m->cfg.n_head * 4);
     return fail(SNLP_ERR_TIMEOUT, "a device-side bounded wait expired; results of the calls since the last check are invalid");
   }
   return SNLP_OK;
@@ -592,23 +607,21 @@ static bool umma_path_ok(const snlp_model *m) {
 static bool fused_prefill_ok(const snlp_model *m, int M) { return umma_path_ok(m) && M > kDecodeRows; }
 static bool fast_decode_ok(const snlp_model *m, int M) { return umma_path_ok(m) && M <= kDecodeRows; }
 
-// Largest K split <= want whose slices are whole 64-element k-blocks.
-static int pick_ksplit(int K, int want) {
-  for (int s = want; s > 1; --s)
-    if (K % s == 0 && (K / s) % kUmmaBK == 0) return s;
-  return 1;
-}
-
 template <int BN, int AM, int EPI>
 static cudaError_t umma_attr() {
   return cudaFuncSetAttribute(k_umma_gemm<BN, AM, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<BN, AM>::kSmem);
 }
 template <int EPI>
+static cudaError_t gemv_attr() {
+  cudaError_t e = cudaFuncSetAttribute(k_umma_gemv<128, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<128, 16>::kSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_umma_gemv<256, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<256, 16>::kSmem);
+  return e;
+}
+template <int EPI>
 static cudaError_t umma_attr_all() {
   cudaError_t e = umma_attr<128, 128, EPI>();
   if (e == cudaSuccess) e = umma_attr<256, 128, EPI>();
-  if (e == cudaSuccess) e = umma_attr<128, 16, EPI>();
-  if (e == cudaSuccess) e = umma_attr<256, 16, EPI>();
+  if (e == cudaSuccess) e = gemv_attr<EPI>();
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_umma_gemm2<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kU2Smem);
   return e;
 }
@@ -636,15 +649,39 @@ static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat1
     KLAUNCH(m, st, cls, k_umma_gemm2<EPI><<<2 * pairs, kUmmaThreads, kU2Smem, st>>>(ta, w.tm_half, p));
     return SNLP_OK;
   }
-  // Decode regime: a launch that does not occupy every SM (a sequential step's single layer: 5-20 items) lasts as long
-  // as one item.  The column tiling does not touch the numbers (every output column is its own dot product), so a
-  // launch whose 128-wide items still fit one round over the SMs takes those: twice the CTAs, half the bytes each.
-  // Beyond that the 256-wide tile is the faster one (a 128-wide MMA costs as much as a 256-wide one, which caps a
-  // CTA streaming 128-wide tiles at ~50 GB/s).  The
-  // out-projection's partial sums of squares are per 128 columns in this regime, whatever the tile width.
-  int bn = w.BN;
-  if (small && w.BN == 256 && (N / 128) * ksplit * nl <= m->n_sm) bn = 128;
-  const CUtensorMap &tmw = bn == w.BN ? w.tm : w.tm_half;
+  if (small) {
+    // Decode regime: the reduction is cut into fixed slices (a function of the projection's shape only) and the
+    // (tile, slice) units are dealt to the SMs in equal contiguous ranges; see umma_gemv.cuh.
+    const int nkb1 = K / kUmmaBK, skb = gemv_kslice_kb(nkb1, p.kfuse);
+    p.kslice = skb * kUmmaBK; p.ksplit = nkb1 / skb;
+    const int kst = p.ksplit * p.kfuse;
+    if (kst > kGemvMaxSlices) return fail(SNLP_ERR_UNSUPPORTED, "decode-regime product: %d fused layers give %d slices per tile (limit %d)", p.kfuse, kst, kGemvMaxSlices);
+    // Column width of the tiles: it does not touch the numbers (every output column is its own dot product).  The
+    // launch lasts as long as its most loaded SM: ceil(units / SMs) units of BN x kslice weights.  256 columns put
+    // 8 KB of weights under each tcgen05.mma (an instruction costs the same ~155 cycles whatever its shape), so
+    // 128 columns are taken only where they shorten that critical path noticeably (launches of a few tiles).
+    auto critical = [&](int bn_) {
+      const long long U = (long long)(N / bn_) * nl * kst, G = U < m->n_sm ? U : m->n_sm;
+      return (U + G - 1) / G * bn_;
+    };
+    int bn = w.BN;
+    if (w.BN == 256 && critical(128) * 100 < critical(256) * 87) bn = 128;
+    const CUtensorMap &tmw = bn == w.BN ? w.tm : w.tm_half;
+    p.Nt = N / bn;
+    p.partial = m->gemv_part; p.tile_counters = m->gemv_ctr;
+    const long long U = (long long)p.Nt * nl * kst;
+    const int grid = (int)(U < m->n_sm ? U : m->n_sm);
+    if (bn == 256) {
+      p.nstages = UmmaCfg<256, 16>::kStages;
+      KLAUNCH(m, st, cls, k_umma_gemv<256, EPI><<<grid, kUmmaThreads, UmmaCfg<256, 16>::kSmem, st>>>(ta, tmw, p));
+    } else {
+      p.nstages = UmmaCfg<128, 16>::kStages;
+      KLAUNCH(m, st, cls, k_umma_gemv<128, EPI><<<grid, kUmmaThreads, UmmaCfg<128, 16>::kSmem, st>>>(ta, tmw, p));
+    }
+    return SNLP_OK;
+  }
+  const int bn = w.BN;
+  const CUtensorMap &tmw = w.tm;
   p.Nt = N / bn;
   const int items = p.Mt * p.Nt * ksplit * nl;
   const int grid = items < m->n_sm ? items : m->n_sm;
@@ -653,12 +690,9 @@ static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat1
     p.nstages = UmmaCfg<BN_, AM_>::kStages;                                                                                          \
     KLAUNCH(m, st, cls, k_umma_gemm<BN_, AM_, EPI><<<grid, kUmmaThreads, UmmaCfg<BN_, AM_>::kSmem, st>>>(ta, tmw, p));                \
   } while (0)
-  if (bn == 256) {
-    if (small) SNLP_UMMA_LAUNCH(256, 16);
-    else if (EPI != UEPI_LMHEAD) SNLP_UMMA_LAUNCH(256, 128);
-  } else {
-    if (small) SNLP_UMMA_LAUNCH(128, 16);
-    else if (EPI != UEPI_LMHEAD) SNLP_UMMA_LAUNCH(128, 128);
+  if (EPI != UEPI_LMHEAD) {
+    if (bn == 256) SNLP_UMMA_LAUNCH(256, 128);
+    else SNLP_UMMA_LAUNCH(128, 128);
   }
 #undef SNLP_UMMA_LAUNCH
   return SNLP_OK;
@@ -740,7 +774,8 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
 // K split of the decode-regime down-projection (its reduction is the longest); it does not depend on how many
 // layers a launch covers, so sequential execution and layer-parallel sweeps add the partial sums in the same order.
 static int down_splits(const snlp_model *m, int M) {
-  return (umma_path_ok(m) && M <= kDecodeRows) ? pick_ksplit(m->cfg.d_ff, kMaxSplits) : 1;
+  (void)m; (void)M;
+  return 1;   // both regimes reduce inside the product (the decode regime in fixed slices, see umma_gemv.cuh)
 }
 
 // bf16 branch inputs of layers l0 .. l0+nl-1 for blocks_umma (and the fp32 MLP pre-map of mHC models)
@@ -761,8 +796,7 @@ static int init_kernel_attributes() {
   CU(umma_attr_all<UEPI_RELU2_BF16>());
   CU(umma_attr_all<UEPI_QKV>());
   CU(umma_attr_all<UEPI_RESID>());
-  CU((umma_attr<128, 16, UEPI_LMHEAD>()));
-  CU((umma_attr<256, 16, UEPI_LMHEAD>()));
+  CU(gemv_attr<UEPI_LMHEAD>());
   CU(cudaFuncSetAttribute(k_attn_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, kFuSmem));
 #define ATTR(NS) CU(cudaFuncSetAttribute(k_correct<NS, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(corr_ring_bytes(NS, 256) + kCorrExtraSmem))); \
   CU(cudaFuncSetAttribute(k_correct<NS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(corr_ring_bytes(NS, 256) + kCorrExtraSmem)));

@@ -59,6 +59,9 @@ struct UmmaParams {
   // index) and then adds one to *bump (nullable).  lm_counter: zero on entry, left zero.
   // argmax_pp (nullable): the address of argmax is read from a device slot instead (replayed decode graphs).
   int32_t *argmax; int *bump; unsigned *lm_counter; int32_t *const *argmax_pp;
+  // decode regime (k_umma_gemv): pieces of tiles whose slices are spread over several CTAs, [#CTAs][slices per tile][M][BN]
+  // fp32, and one arrival counter per CTA (zero on entry, left zero)
+  float *partial; unsigned *tile_counters;
 };
 
 constexpr int kUmmaThreads = 320;   // warp 0: TMA, warp 1: MMA + TMEM allocation, warps 2-9: epilogue (two per TMEM lane quarter)
