@@ -229,6 +229,9 @@ int snlp_draft_and_verify_async(snlp_model *m, snlp_kv *kv, int32_t *last_tok, i
  * flag 1: force the generic SIMT kernels even where a specialised kernel exists (default 0; testing).
  * flag 2: time every launch with CUDA events on its stream, accumulated per kernel class (default 0;
  *         while on, decode steps are launched directly instead of replaying graphs).
+ * flag 4: programmatic dependent launch between the kernels of layer-by-layer execution (sequential forward, sequential
+ *         prefix; default 1): a kernel is scheduled while its predecessor finishes and requests its first weight tiles
+ *         before it waits for that kernel's results.  The launches of a sweep never use it.
  * flag 3: failure-detection test hook: waits for the device, then writes `value != 0` into the error word that a
  *         kernel raises when one of its bounded waits expires; snlp_device_status then reports it exactly as it
  *         would report a real expiry (no kernel is made to wait). */

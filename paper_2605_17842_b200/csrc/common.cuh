@@ -85,4 +85,12 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialisation attribute may start while the
+// kernel before it in the stream is still running; pdl_wait() returns once that kernel (and, by induction, every
+// earlier one) has completed and its writes are visible, so everything a kernel does before it must depend on nothing
+// an earlier kernel of the stream writes (set-up, weight prefetch).  pdl_trigger() lets the NEXT kernel of the stream be
+// scheduled as soon as every CTA of this grid has issued it (or exited).  Both are no-ops in a normal launch.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 }  // namespace snlp

@@ -319,6 +319,8 @@ __global__ void __launch_bounds__(256, NS == 1 ? 4 : 2) k_correct(CorrParams p) 
 template <int NS>
 __global__ void k_prep_rows(const float *__restrict__ trace, int l0, int M, int d, const HcCoef *__restrict__ coef,
                             __nv_bfloat16 *__restrict__ xb, float *__restrict__ ssq_x, float *__restrict__ xm) {
+  pdl_trigger();
+  pdl_wait();
   const int d4 = d >> 2, c4 = threadIdx.x, l = l0 + blockIdx.y;
   const size_t row = blockIdx.x, Md4 = (size_t)M * d4;
   const float4 *x = reinterpret_cast<const float4 *>(trace) + (size_t)l * Md4 * NS + row * NS * d4 + c4;
@@ -352,6 +354,8 @@ __global__ void k_init_rows(float *__restrict__ trace, int l0, int L, int M, int
                             __nv_bfloat16 *__restrict__ xb, float *__restrict__ ssq_x, float *__restrict__ xm, int write_trace,
                             const int32_t *__restrict__ ids = nullptr, const __nv_bfloat16 *__restrict__ table = nullptr, int vocab = 0,
                             const int32_t *const *__restrict__ ids_pp = nullptr) {
+  pdl_trigger();
+  pdl_wait();
   if (ids_pp != nullptr) ids = *ids_pp;   // the ids' address is read from a device slot (replayed decode graphs)
   const int d4 = d >> 2, c4 = threadIdx.x;
   const size_t row = blockIdx.x, Md4 = (size_t)M * d4;
@@ -427,6 +431,8 @@ constexpr int kCorrSmallWarps = 16;
 template <int NS>
 __global__ void __launch_bounds__(32 * kCorrSmallWarps) k_correct_small(CorrParams p) {
   extern __shared__ float4 s_buf[];
+  pdl_trigger();   // a few CTAs on a few SMs: the next kernel may move in beside it at once and fetch its first weights
+  pdl_wait();
   const int d4 = p.d >> 2;
   const int c = threadIdx.x & 31, ll = threadIdx.x >> 5;
   const int c4 = blockIdx.x * 32 + c;

@@ -33,6 +33,7 @@ static __global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat
   __shared__ float hacc[8][128];
   __shared__ float hm[8], hl[8];
   __shared__ bool s_last;
+  pdl_wait();
   const int chunk = blockIdx.x, nchunk = gridDim.x, bh = blockIdx.y, l = blockIdx.z;
   const int b = bh / H, h = bh % H, d = H * 128;
   const int pos0 = *pos_base, kbeg = chunk * csub * kAttnSub;
@@ -152,6 +153,7 @@ static __global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat
     __syncthreads();
   }
   // ---- last CTA of this (layer, sequence, head) merges the chunks in chunk order --------------------
+  pdl_trigger();   // the chunk has been streamed: only the merge is left
   __threadfence();
   __syncthreads();
   if (tid == 0) s_last = atomicAdd(&counters[(size_t)l * gridDim.y + bh], 1u) == (unsigned)nchunk - 1;

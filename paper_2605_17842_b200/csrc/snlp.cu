@@ -18,7 +18,6 @@
 #include "generic.cuh"
 #include "umma_gemm.cuh"
 #include "umma_gemm2.cuh"
-#include "umma_gemv.cuh"
 #include "attn_umma.cuh"
 
 using namespace snlp;
@@ -58,6 +57,7 @@ void set_last_error(const char *msg) { g_err = msg; }  // for the library's othe
 // ------------------------------------------------------------------------------------------------
 // handles
 constexpr size_t kCorrExtraSmem = 32768;   // k_correct: shared memory beyond the operand ring (norm partials, staged coefficients)
+constexpr int kMaxSplits = 4;    // K-splits of the partial-sum GEMV outputs
 constexpr int kDecodeRows = 16;  // largest row count served by the decode-regime kernels
 constexpr size_t kCorrSmallSmem = 160 * 1024;
 
@@ -97,15 +97,13 @@ struct snlp_model {
   unsigned *counter = nullptr, *attn_counters = nullptr;
   int *zero = nullptr;
   unsigned *lm_counter = nullptr;   // arrival counter of the LM-head launch (zero between launches)
-  float *gemv_part = nullptr;       // decode-regime products: pieces of tiles split between CTAs
-  unsigned *gemv_ctr = nullptr;     // their arrival counters, one per CTA (zero between launches)
-  size_t gemv_ctr_bytes = 0;
   int32_t *spec = nullptr;  // [2 * (max_rows + 1)] ids / verifier tokens for draft-and-verify
   int32_t *tok_pin = nullptr, *tok_dev = nullptr;   // [2][max_batch] mapped pinned host memory (tokens in, tokens out) and its device address (snlp_decode_step_host)
   int logit_rows = 0;
   std::vector<void *> allocs;
   // flags / stats
-  int use_graphs = 1, force_generic = 0, timing = 0;
+  int use_graphs = 1, force_generic = 0, timing = 0, use_pdl = 1;
+  bool pdl_now = false;   // launches issued right now carry the programmatic-serialisation attribute (layer-by-layer execution only)
   std::vector<PendingTime> pending;
   std::vector<cudaEvent_t> free_events;
   double class_ms[KC_COUNT] = {};
@@ -199,6 +197,20 @@ struct TimedLaunch {
     if (e_ != cudaSuccess) return fail(SNLP_ERR_CUDA, "kernel launch failed (%s:%d): %s", __FILE__, __LINE__, cudaGetErrorString(e_)); \
   } while (0)
 
+// Launch with the programmatic-serialisation attribute (see pdl_wait / pdl_trigger in common.cuh): the kernel may be
+// scheduled while the one before it in the stream is still finishing.  Works the same under stream capture (the
+// dependency becomes a programmatic edge of the graph).  pdl == false: an ordinary launch.
+template <typename... KArgs, typename... Args>
+static void launch_pdl(bool pdl, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
+  cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);   // a failure is picked up by the cudaGetLastError() that follows every launch
+}
+
 template <typename P>
 static int dalloc(snlp_model *m, P **p, size_t bytes) {
   void *q = nullptr;
@@ -264,7 +276,8 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
     A(&m->xm, L * R * d * 4);
   }
   A(&m->qkv_raw, L * R * 3 * d * 4);
-  const size_t split_rows = R;
+  // the decode-regime kernels write up to kMaxSplits partial sums for at most kDecodeRows rows
+  const size_t split_rows = std::max<size_t>(R, (size_t)kMaxSplits * std::min<size_t>(R, kDecodeRows));
   A(&m->a, L * split_rows * d * 4);
   A(&m->y_raw, L * R * ff * 4);
   A(&m->mb, L * split_rows * d * 4);
@@ -295,14 +308,6 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
   A(&m->attn_counters, L * (size_t)kDecodeRows * c.n_head * 4);
   A(&m->zero, 16);
   A(&m->lm_counter, 16);
-  {
-    cudaDeviceProp prop;
-    if (rc == SNLP_OK && cudaGetDeviceProperties(&prop, m->device) == cudaSuccess) m->n_sm = prop.multiProcessorCount;
-    const size_t rows = std::min<size_t>(R, kDecodeRows);
-    A(&m->gemv_part, (size_t)m->n_sm * kGemvMaxSlices * rows * 256 * sizeof(float));
-    m->gemv_ctr_bytes = (size_t)(m->n_sm + 1) * sizeof(unsigned);
-    A(&m->gemv_ctr, m->gemv_ctr_bytes);
-  }
   A(&m->spec, 2 * (R + 1) * 4);
   A(&m->tok_slot, 2 * sizeof(void *));
   if (rc == SNLP_OK && (cudaHostAlloc((void **)&m->tok_pin, (size_t)2 * c.max_batch * 4, cudaHostAllocMapped) != cudaSuccess ||
@@ -311,7 +316,7 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
     rc = fail(SNLP_ERR_OOM, "cudaHostAlloc of the token staging buffer failed");
   }
   if (rc == SNLP_OK) {
-    if (cudaMemset(m->dev_err, 0, 16) != cudaSuccess || cudaMemset(m->attn_counters, 0, L * (size_t)kDecodeRows * c.n_head * 4) != cudaSuccess || cudaMemset(m->counter, 0, 16) != cudaSuccess || cudaMemset(m->zero, 0, 16) != cudaSuccess || cudaMemset(m->lm_counter, 0, 16) != cudaSuccess || cudaMemset(m->gemv_ctr, 0, m->gemv_ctr_bytes) != cudaSuccess)
+    if (cudaMemset(m->dev_err, 0, 16) != cudaSuccess || cudaMemset(m->attn_counters, 0, L * (size_t)kDecodeRows * c.n_head * 4) != cudaSuccess || cudaMemset(m->counter, 0, 16) != cudaSuccess || cudaMemset(m->zero, 0, 16) != cudaSuccess || cudaMemset(m->lm_counter, 0, 16) != cudaSuccess)
       rc = fail(SNLP_ERR_CUDA, "cudaMemset failed");
   }
   if (rc == SNLP_OK) {
@@ -434,6 +439,14 @@ extern "C" int snlp_set_flag(snlp_model *m, int flag, int value) {
   if (flag == 0) m->use_graphs = value != 0;
   else if (flag == 1) m->force_generic = value != 0;
   else if (flag == 2) m->timing = value != 0;
+  else if (flag == 4) {
+    if (m->use_pdl != (value != 0)) {   // captured decode steps carry the launch attributes they were recorded with
+      CU(cudaDeviceSynchronize());
+      for (auto &g : m->graphs) cudaGraphExecDestroy(g.second.exec);
+      m->graphs.clear();
+    }
+    m->use_pdl = value != 0;
+  }
   else if (flag == 3) {   // host-side injection of the error word a kernel raises when a bounded wait expires
     const int v = value != 0;
     CU(cudaDeviceSynchronize());
@@ -476,7 +489,6 @@ extern "C" int snlp_device_status(snlp_model *m, void *stream) {
   if (flag) {
     cudaMemset(m->dev_err, 0, sizeof flag);
     // a kernel that gave up may have left arrival counters part-way: bring them back to zero for the calls that follow
-    cudaMemset(m->gemv_ctr, 0, m->gemv_ctr_bytes);
     cudaMemset(m->lm_counter, 0, 16);
     cudaMemset(m->counter, 0, 16);
     cudaMemset(m->attn_counters, 0, (size_t)m->cfg.n_layer * kDecodeRows * m->cfg.n_head * 4);
@@ -543,7 +555,7 @@ static int correct(snlp_model *m, const Fwd &f, int l0, int nsteps, int lstep, i
     dim3 grid((c.d_model / 4 + 31) / 32, f.M);
     TimedLaunch tl_(m, f.st, KC_CORRECT);
     switch (c.n_streams) {
-#define CASE(NS) case NS: k_correct_small<NS><<<grid, 32 * kCorrSmallWarps, sm_small, f.st>>>(p); break;
+#define CASE(NS) case NS: launch_pdl(m->pdl_now, k_correct_small<NS>, grid, dim3(32 * kCorrSmallWarps), sm_small, f.st, p); break;
       CASE(1) CASE(2) CASE(3) CASE(4)
 #undef CASE
     }
@@ -607,21 +619,23 @@ static bool umma_path_ok(const snlp_model *m) {
 static bool fused_prefill_ok(const snlp_model *m, int M) { return umma_path_ok(m) && M > kDecodeRows; }
 static bool fast_decode_ok(const snlp_model *m, int M) { return umma_path_ok(m) && M <= kDecodeRows; }
 
+// Largest K split <= want whose slices are whole 64-element k-blocks.
+static int pick_ksplit(int K, int want) {
+  for (int s = want; s > 1; --s)
+    if (K % s == 0 && (K / s) % kUmmaBK == 0) return s;
+  return 1;
+}
+
 template <int BN, int AM, int EPI>
 static cudaError_t umma_attr() {
   return cudaFuncSetAttribute(k_umma_gemm<BN, AM, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<BN, AM>::kSmem);
 }
 template <int EPI>
-static cudaError_t gemv_attr() {
-  cudaError_t e = cudaFuncSetAttribute(k_umma_gemv<128, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<128, 16>::kSmem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_umma_gemv<256, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<256, 16>::kSmem);
-  return e;
-}
-template <int EPI>
 static cudaError_t umma_attr_all() {
   cudaError_t e = umma_attr<128, 128, EPI>();
   if (e == cudaSuccess) e = umma_attr<256, 128, EPI>();
-  if (e == cudaSuccess) e = gemv_attr<EPI>();
+  if (e == cudaSuccess) e = umma_attr<128, 16, EPI>();
+  if (e == cudaSuccess) e = umma_attr<256, 16, EPI>();
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_umma_gemm2<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kU2Smem);
   return e;
 }
@@ -649,50 +663,29 @@ static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat1
     KLAUNCH(m, st, cls, k_umma_gemm2<EPI><<<2 * pairs, kUmmaThreads, kU2Smem, st>>>(ta, w.tm_half, p));
     return SNLP_OK;
   }
-  if (small) {
-    // Decode regime: the reduction is cut into fixed slices (a function of the projection's shape only) and the
-    // (tile, slice) units are dealt to the SMs in equal contiguous ranges; see umma_gemv.cuh.
-    const int nkb1 = K / kUmmaBK, skb = gemv_kslice_kb(nkb1, p.kfuse);
-    p.kslice = skb * kUmmaBK; p.ksplit = nkb1 / skb;
-    const int kst = p.ksplit * p.kfuse;
-    if (kst > kGemvMaxSlices) return fail(SNLP_ERR_UNSUPPORTED, "decode-regime product: %d fused layers give %d slices per tile (limit %d)", p.kfuse, kst, kGemvMaxSlices);
-    // Column width of the tiles: it does not touch the numbers (every output column is its own dot product).  The
-    // launch lasts as long as its most loaded SM: ceil(units / SMs) units of BN x kslice weights.  256 columns put
-    // 8 KB of weights under each tcgen05.mma (an instruction costs the same ~155 cycles whatever its shape), so
-    // 128 columns are taken only where they shorten that critical path noticeably (launches of a few tiles).
-    auto critical = [&](int bn_) {
-      const long long U = (long long)(N / bn_) * nl * kst, G = U < m->n_sm ? U : m->n_sm;
-      return (U + G - 1) / G * bn_;
-    };
-    int bn = w.BN;
-    if (w.BN == 256 && critical(128) * 100 < critical(256) * 87) bn = 128;
-    const CUtensorMap &tmw = bn == w.BN ? w.tm : w.tm_half;
-    p.Nt = N / bn;
-    p.partial = m->gemv_part; p.tile_counters = m->gemv_ctr;
-    const long long U = (long long)p.Nt * nl * kst;
-    const int grid = (int)(U < m->n_sm ? U : m->n_sm);
-    if (bn == 256) {
-      p.nstages = UmmaCfg<256, 16>::kStages;
-      KLAUNCH(m, st, cls, k_umma_gemv<256, EPI><<<grid, kUmmaThreads, UmmaCfg<256, 16>::kSmem, st>>>(ta, tmw, p));
-    } else {
-      p.nstages = UmmaCfg<128, 16>::kStages;
-      KLAUNCH(m, st, cls, k_umma_gemv<128, EPI><<<grid, kUmmaThreads, UmmaCfg<128, 16>::kSmem, st>>>(ta, tmw, p));
-    }
-    return SNLP_OK;
-  }
-  const int bn = w.BN;
-  const CUtensorMap &tmw = w.tm;
+  // Decode regime: a launch that does not occupy every SM (a sequential step's single layer: 5-20 items) lasts as long
+  // as one item.  The column tiling does not touch the numbers (every output column is its own dot product), so a
+  // launch whose 128-wide items still fit one round over the SMs takes those: twice the CTAs, half the bytes each.
+  // Beyond that the 256-wide tile is the faster one (a 128-wide MMA costs as much as a 256-wide one, which caps a
+  // CTA streaming 128-wide tiles at ~50 GB/s).  The
+  // out-projection's partial sums of squares are per 128 columns in this regime, whatever the tile width.
+  int bn = w.BN;
+  if (small && w.BN == 256 && (N / 128) * ksplit * nl <= m->n_sm) bn = 128;
+  const CUtensorMap &tmw = bn == w.BN ? w.tm : w.tm_half;
   p.Nt = N / bn;
   const int items = p.Mt * p.Nt * ksplit * nl;
   const int grid = items < m->n_sm ? items : m->n_sm;
 #define SNLP_UMMA_LAUNCH(BN_, AM_)                                                                                                   \
   do {                                                                                                                               \
     p.nstages = UmmaCfg<BN_, AM_>::kStages;                                                                                          \
-    KLAUNCH(m, st, cls, k_umma_gemm<BN_, AM_, EPI><<<grid, kUmmaThreads, UmmaCfg<BN_, AM_>::kSmem, st>>>(ta, tmw, p));                \
+    KLAUNCH(m, st, cls, launch_pdl(m->pdl_now, k_umma_gemm<BN_, AM_, EPI>, dim3(grid), dim3(kUmmaThreads), UmmaCfg<BN_, AM_>::kSmem, st, ta, tmw, p)); \
   } while (0)
-  if (EPI != UEPI_LMHEAD) {
-    if (bn == 256) SNLP_UMMA_LAUNCH(256, 128);
-    else SNLP_UMMA_LAUNCH(128, 128);
+  if (bn == 256) {
+    if (small) SNLP_UMMA_LAUNCH(256, 16);
+    else if (EPI != UEPI_LMHEAD) SNLP_UMMA_LAUNCH(256, 128);
+  } else {
+    if (small) SNLP_UMMA_LAUNCH(128, 16);
+    else if (EPI != UEPI_LMHEAD) SNLP_UMMA_LAUNCH(128, 128);
   }
 #undef SNLP_UMMA_LAUNCH
   return SNLP_OK;
@@ -732,8 +725,8 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
   if (small) {
     const int csub = attn_csub(f.B * H);
     const int nchunk = (f.pos_hi + f.T - 1) / (csub * kAttnSub) + 1;
-    KLAUNCH(m, st, KC_ATTN, k_attn_decode<<<dim3(nchunk, f.B * H, nl), 128, 0, st>>>(q, Md, kc, vc, f.kv_ls, f.kv_bs, m->attn_part, m->attn_counters, att, Md,
-                                                                            f.T, H, f.pos, csub));
+    KLAUNCH(m, st, KC_ATTN, launch_pdl(m->pdl_now, k_attn_decode, dim3(nchunk, f.B * H, nl), dim3(128), 0, st, (const __nv_bfloat16 *)q, Md, (const __nv_bfloat16 *)kc,
+                                       (const __nv_bfloat16 *)vc, f.kv_ls, f.kv_bs, m->attn_part, m->attn_counters, att, Md, f.T, H, f.pos, csub));
   } else {
     // tensor-core attention: 128-query items over the (layer, sequence, head, query tile) grid, persistent CTAs
     CUtensorMap tq, tk, tv, to;
@@ -774,8 +767,7 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
 // K split of the decode-regime down-projection (its reduction is the longest); it does not depend on how many
 // layers a launch covers, so sequential execution and layer-parallel sweeps add the partial sums in the same order.
 static int down_splits(const snlp_model *m, int M) {
-  (void)m; (void)M;
-  return 1;   // both regimes reduce inside the product (the decode regime in fixed slices, see umma_gemv.cuh)
+  return (umma_path_ok(m) && M <= kDecodeRows) ? pick_ksplit(m->cfg.d_ff, kMaxSplits) : 1;
 }
 
 // bf16 branch inputs of layers l0 .. l0+nl-1 for blocks_umma (and the fp32 MLP pre-map of mHC models)
@@ -784,7 +776,7 @@ static int prep_rows(snlp_model *m, const Fwd &f, int l0, int nl) {
   dim3 grid(f.M, nl);
   const int threads = c.d_model / 4;
   switch (c.n_streams) {
-#define CASE(NS) case NS: KLAUNCH(m, f.st, KC_OTHER, k_prep_rows<NS><<<grid, threads, 0, f.st>>>(m->trace, l0, f.M, c.d_model, m->coef, (__nv_bfloat16 *)m->xn, m->ssq_x, m->xm)); break;
+#define CASE(NS) case NS: KLAUNCH(m, f.st, KC_OTHER, launch_pdl(m->pdl_now, k_prep_rows<NS>, grid, dim3(threads), 0, f.st, (const float *)m->trace, l0, f.M, c.d_model, (const HcCoef *)m->coef, (__nv_bfloat16 *)m->xn, m->ssq_x, m->xm)); break;
     CASE(1) CASE(2) CASE(3) CASE(4) CASE(5) CASE(6) CASE(7) CASE(8)
 #undef CASE
   }
@@ -796,7 +788,8 @@ static int init_kernel_attributes() {
   CU(umma_attr_all<UEPI_RELU2_BF16>());
   CU(umma_attr_all<UEPI_QKV>());
   CU(umma_attr_all<UEPI_RESID>());
-  CU(gemv_attr<UEPI_LMHEAD>());
+  CU((umma_attr<128, 16, UEPI_LMHEAD>()));
+  CU((umma_attr<256, 16, UEPI_LMHEAD>()));
   CU(cudaFuncSetAttribute(k_attn_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, kFuSmem));
 #define ATTR(NS) CU(cudaFuncSetAttribute(k_correct<NS, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(corr_ring_bytes(NS, 256) + kCorrExtraSmem))); \
   CU(cudaFuncSetAttribute(k_correct<NS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(corr_ring_bytes(NS, 256) + kCorrExtraSmem)));
@@ -864,7 +857,17 @@ static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *res
   const bool fused_embed = have_ids && umma_path_ok(m) && S == 0 && !seq;
   if (have_ids && !fused_embed) TRY(embed_impl(m, f.st, f.embed_ids, f.M, m->trace, f.embed_ids_pp));
   if (resnorm_out && sol.K > 0 && !seq) CU(cudaMemsetAsync(resnorm_out, 0, (size_t)sol.K * L * 2 * sizeof(float), f.st));
+  // Layer-by-layer execution is a chain of short kernels on a few SMs each: there a kernel is launched with the
+  // programmatic-serialisation attribute, so that it is scheduled while its predecessor finishes and requests its
+  // first weight tiles before it waits for that kernel's results (measured: 4-5 % of a sequential decode step).  The
+  // launches of a sweep fill the GPU; they gain nothing from it (measured: 2-8 % slower) and are launched normally.
+  struct PdlScope {
+    snlp_model *m;
+    explicit PdlScope(snlp_model *m_) : m(m_) { m->pdl_now = m->use_pdl != 0; }
+    ~PdlScope() { m->pdl_now = false; }
+  };
   if (S > 0) {  // Alg. 2 lines 2-4
+    PdlScope pdl(m);
     if (umma_path_ok(m)) TRY(prep_rows(m, f, 0, 1));
     else TRY(premix(m, f, 0, 1));
     for (int l = 0; l < S; ++l) {
@@ -874,6 +877,7 @@ static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *res
   }
   if (S == L) return SNLP_OK;
   if (seq) {  // sequential execution of the fused model: chunk after chunk
+    PdlScope pdl(m);
     if (umma_path_ok(m)) TRY(prep_rows(m, f, S, 1));
     for (int h = S; h < L; h += F) {
       TRY(run_blocks(m, f, h, F, F));
@@ -884,7 +888,7 @@ static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *res
   // Alg. 2 line 5: every suffix state starts at h_S
   if (umma_path_ok(m)) {
     switch (c.n_streams) {   // one kernel: the copies and the layers' first branch inputs
-#define CASE(NS) case NS: KLAUNCH(m, f.st, KC_OTHER, k_init_rows<NS><<<f.M, c.d_model / 4, 0, f.st>>>(m->trace, S, L, f.M, c.d_model, m->coef, (__nv_bfloat16 *)m->xn, m->ssq_x, m->xm, 0, fused_embed ? f.embed_ids : nullptr, (const __nv_bfloat16 *)m->embed, c.vocab, fused_embed ? f.embed_ids_pp : nullptr)); break;
+#define CASE(NS) case NS: KLAUNCH(m, f.st, KC_OTHER, launch_pdl(m->pdl_now, k_init_rows<NS>, dim3(f.M), dim3(c.d_model / 4), 0, f.st, m->trace, S, L, f.M, c.d_model, (const HcCoef *)m->coef, (__nv_bfloat16 *)m->xn, m->ssq_x, m->xm, 0, fused_embed ? f.embed_ids : (const int32_t *)nullptr, (const __nv_bfloat16 *)m->embed, c.vocab, fused_embed ? f.embed_ids_pp : (const int32_t *const *)nullptr)); break;
       CASE(1) CASE(2) CASE(3) CASE(4) CASE(5) CASE(6) CASE(7) CASE(8)
 #undef CASE
     }

@@ -59,9 +59,6 @@ struct UmmaParams {
   // index) and then adds one to *bump (nullable).  lm_counter: zero on entry, left zero.
   // argmax_pp (nullable): the address of argmax is read from a device slot instead (replayed decode graphs).
   int32_t *argmax; int *bump; unsigned *lm_counter; int32_t *const *argmax_pp;
-  // decode regime (k_umma_gemv): pieces of tiles whose slices are spread over several CTAs, [#CTAs][slices per tile][M][BN]
-  // fp32, and one arrival counter per CTA (zero on entry, left zero)
-  float *partial; unsigned *tile_counters;
 };
 
 constexpr int kUmmaThreads = 320;   // warp 0: TMA, warp 1: MMA + TMEM allocation, warps 2-9: epilogue (two per TMEM lane quarter)
@@ -529,6 +526,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Everything up to here, and the weight tiles the producer requests first, depend on no earlier kernel of the stream.
+  if (!(warp == 0 && lane == 0)) pdl_wait();
 
   // item -> (row tile, column tile, K split, layer); row tiles fastest so that concurrent CTAs share a weight tile
 #define SNLP_DECODE_ITEM(i)                                       \
@@ -544,9 +543,30 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
     if (lane == 0) {
       int g = 0, issued = 0;
       bool ok = true;
-      for (int i = 0; i < my_items && ok; ++i) {
+      // The weight tiles of the first ring-ful of k-blocks are requested before the dependency wait (under a programmatic
+      // dependent launch they stream in while the previous kernel is still finishing); the activation tiles of the same
+      // stages follow once that kernel's results are visible.
+      const int total_kb = my_items * nkb, npre = total_kb < S ? total_kb : S;
+      for (int pass = 0; pass < 2; ++pass) {
+        if (pass == 1) pdl_wait();
+        for (int i = 0, gp = 0; gp < npre; ++i) {
+          SNLP_DECODE_ITEM(i)
+          for (int kb = 0; kb < nkb && gp < npre; ++kb, ++gp) {
+            const int j = kb / nkb1, k0 = ks * p.kslice + (kb % nkb1) * kUmmaBK;
+            if (pass == 0) {
+              mbar_expect_tx(&full[gp], Cfg::kABytes + Cfg::kBBytes);   // the stages are empty: first use
+              tma_load_3d(sB + (size_t)gp * Cfg::kBBytes, &tmB, &full[gp], k0, n_tile * BN, p.l0 + l + j);
+            } else {
+              tma_load_3d(sA + (size_t)gp * Cfg::kABytes, &tmA, &full[gp], k0, m_tile * kUmmaBM, la + j);
+            }
+          }
+        }
+      }
+      issued = npre;
+      for (int i = npre / nkb; i < my_items && ok; ++i) {
         SNLP_DECODE_ITEM(i)
-        for (int kb = 0; kb < nkb; ++kb, ++g) {
+        for (int kb = (i == npre / nkb ? npre % nkb : 0); kb < nkb; ++kb) {
+          g = i * nkb + kb;
           const int s = g % S;
           ok = mbar_wait(&empty[s], ((g / S) & 1) ^ 1u, abort_flag, p.err);
           if (!ok) break;
@@ -557,6 +577,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
           issued = g + 1;
         }
       }
+      // every load of this CTA has been requested: what is left is its tail, so the next kernel of the stream may be
+      // scheduled onto the SMs as they free up (it waits for this kernel to complete before it reads any result)
+      pdl_trigger();
       if (*abort_flag) {
         // let the copies still in flight land before the CTA's shared memory is handed on
         const int first = issued > S ? issued - S : 0;
