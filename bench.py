@@ -149,27 +149,35 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     def timed_decode(kv, first_tok, K, n_warm, n_steps, min_total_ms=0.0):
-        """Repeats of (cache cut back to CTX, n_warm untimed steps, n_steps timed steps between two events) until the
-        timed blocks add up to min_total_ms of device time (at least one repeat).  Every repeat is timed as the maximum
-        over the ranks.  Returns (median ms/step, min ms/step, repeats)."""
-        per_step, total = [], 0.0
-        while True:
-            kv.truncate(CTX)
-            tok = first_tok.clone()
-            for _ in range(n_warm):
-                model.decode_step(kv, tok, K, snlp.MODE_IDN, tok_out=tok)
-            barrier()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            for _ in range(n_steps):
-                model.decode_step(kv, tok, K, snlp.MODE_IDN, tok_out=tok)
-            e1.record()
-            barrier()
-            ms = replicas.max_over_ranks(rk, e0.elapsed_time(e1), "cuda")   # the same figure on every rank: same loop count
-            per_step.append(ms / n_steps)
-            total += ms
-            if total >= min_total_ms or len(per_step) >= 400:
-                break
+        """Repeats of (cache cut back to CTX, n_warm untimed steps, n_steps timed steps between two CUDA events).  One
+        calibration repeat fixes how many are needed for min_total_ms of timed device work; those are then enqueued back
+        to back (no host synchronisation in between, so the GPU never idles between repeats) inside one barrier +
+        synchronize bracket, and every repeat is reduced to the maximum over the ranks.
+        Returns (median ms/step, min ms/step, repeats)."""
+        def block(n):
+            evs = []
+            for _ in range(n):
+                kv.truncate(CTX)
+                tok = first_tok.clone()
+                for _ in range(n_warm):
+                    model.decode_step(kv, tok, K, snlp.MODE_IDN, tok_out=tok)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(n_steps):
+                    model.decode_step(kv, tok, K, snlp.MODE_IDN, tok_out=tok)
+                e1.record()
+                evs.append((e0, e1))
+            return evs
+
+        barrier()
+        evs = block(1)
+        barrier()
+        first = replicas.max_over_ranks(rk, evs[0][0].elapsed_time(evs[0][1]), "cuda")   # the same figure on every rank
+        n = max(1, min(400, int(min_total_ms / max(first, 1e-3)) + 1)) if min_total_ms > 0 else 1
+        barrier()
+        evs = block(n)
+        barrier()
+        per_step = [replicas.max_over_ranks(rk, a.elapsed_time(b), "cuda") / n_steps for a, b in evs]
         return statistics.median(per_step), min(per_step), len(per_step)
 
     results = {}
@@ -195,7 +203,7 @@ def run_ours(args):
         ms_main, ms_main_min, repeats = timed_decode(kv, first, K_MAIN, warmup, steps, min_total_ms=min_ms)
         launches = model.launch_count() - l0
         clocks = sampler.stop()
-        launches_timed = int(round(launches * steps / (steps + warmup) / repeats))   # per timed block of `steps` steps
+        launches_timed = int(round(launches * steps / (steps + warmup) / (repeats + 1)))   # per timed block of `steps` steps (one calibration repeat ran too)
         results[(1, K_MAIN)] = ms_main
 
         if args.only_main:
@@ -319,7 +327,8 @@ def run_ours(args):
                    "l2": "no flush: each step streams 2.1 GB of weights + KV (> 126 MB L2)"},
         "timing": {"repeats": repeats, "steps_per_repeat": steps, "ms_per_step_median": ms_main, "ms_per_step_min": ms_main_min,
                    "note": "value = median over the repeats; each repeat = cache cut back to 2048, warm-up steps, then `steps` "
-                           "steps between two CUDA events; repeated until >= 1 s of timed device work"},
+                           "steps between two CUDA events; enough repeats for >= 1 s of timed device work, enqueued back to back "
+                           "between one barrier + synchronize on each side"},
         "clocks": clocks,
         "e2e": {"value": world * 1e3 / ms_e2e, "unit": "tokens/s", "h2d_bytes_per_step": 4, "d2h_bytes_per_step": 4,
                 "steps": e2e_steps, "note": "snlp_decode_step_host every step: host token -> pinned staging, read across the bus by the step's first kernel; next token written back by its last kernel; stream sync"},

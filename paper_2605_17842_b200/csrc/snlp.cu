@@ -673,12 +673,13 @@ static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat1
   if (small && w.BN == 256 && (N / 128) * ksplit * nl <= m->n_sm) bn = 128;
   const CUtensorMap &tmw = bn == w.BN ? w.tm : w.tm_half;
   p.Nt = N / bn;
+  const bool pdl_ = m->pdl_now;
   const int items = p.Mt * p.Nt * ksplit * nl;
   const int grid = items < m->n_sm ? items : m->n_sm;
 #define SNLP_UMMA_LAUNCH(BN_, AM_)                                                                                                   \
   do {                                                                                                                               \
     p.nstages = UmmaCfg<BN_, AM_>::kStages;                                                                                          \
-    KLAUNCH(m, st, cls, launch_pdl(m->pdl_now, k_umma_gemm<BN_, AM_, EPI>, dim3(grid), dim3(kUmmaThreads), UmmaCfg<BN_, AM_>::kSmem, st, ta, tmw, p)); \
+    KLAUNCH(m, st, cls, launch_pdl(pdl_, k_umma_gemm<BN_, AM_, EPI>, dim3(grid), dim3(kUmmaThreads), UmmaCfg<BN_, AM_>::kSmem, st, ta, tmw, p)); \
   } while (0)
   if (bn == 256) {
     if (small) SNLP_UMMA_LAUNCH(256, 16);
