@@ -139,7 +139,7 @@ def run_ours(args):
     extra_steps = 32 if args.quick else 64
     W = synth.make_weights(cfg, seed=1234)
     max_ctx = CTX + warmup + max(steps, extra_steps) + 8
-    model = snlp.Model(cfg, max_rows=512 if args.only_main else 2048, max_batch=8, max_ctx=max_ctx)
+    model = snlp.Model(cfg, max_rows=512 * args.main_batch if args.only_main else 2048, max_batch=8, max_ctx=max_ctx)
     model.load_weights(W)
     stream = torch.cuda.Stream()
     hbm_peak, peak_src = peaks()
@@ -183,8 +183,8 @@ def run_ours(args):
     results = {}
     with torch.cuda.stream(stream):
         caches = {}
-        for B in (1, 8):
-            if B == 8 and (args.quick or args.only_main):
+        for B in ((args.main_batch,) if args.only_main else (1, 8)):
+            if B == 8 and args.quick:
                 continue
             ids = torch.from_numpy(synth.make_ids(cfg, B, CTX, seed=3)).cuda()
             kv = model.kv_cache(B, max_ctx)
@@ -193,7 +193,7 @@ def run_ours(args):
             caches[B] = (kv, first)
 
         # ---- headline: SNLP(K=2) IDN, batch 1 ------------------------------------------------
-        kv, first = caches[1]
+        kv, first = caches[args.main_batch if args.only_main else 1]
         sampler = ClockSampler(local)
         timed_decode(kv, first, K_MAIN, warmup, steps)  # untimed pass: CUDA graphs are captured here
         sampler.start()
@@ -209,8 +209,8 @@ def run_ours(args):
         if args.only_main:
             if rank == 0:
                 print(json.dumps({"metric": "d20 decode tokens/s SNLP(K) vs sequential; sweep HBM GB/s vs B200 peak",
-                                  "value": replicas.whole_job_rate(rk, 1, ms_main), "unit": "tokens/s", "ms_per_step": ms_main,
-                                  "steps": steps, "warmup": warmup, "note": "--only-main: headline point only"}))
+                                  "value": replicas.whole_job_rate(rk, args.main_batch, ms_main), "unit": "tokens/s", "ms_per_step": ms_main,
+                                  "steps": steps, "warmup": warmup, "batch": args.main_batch, "note": "--only-main: one point only"}))
             return
 
         # ---- the other points (fewer steps each) ---------------------------------------------
@@ -727,6 +727,7 @@ def main():
     ap.add_argument("--no-other", action="store_true", help="leave the other configurations out of the benchmark line")
     ap.add_argument("--only-main", action="store_true",
                     help="headline point only, small workspace: the light command used for ncu captures")
+    ap.add_argument("--main-batch", type=int, default=1, choices=[1, 8], help="with --only-main: the batch size of the one point that is run")
     ap.add_argument("--workload", default="d20_decode", choices=["d20_decode", "d12_prefill", "d20_hcn", "d20_spec", "paper_0p5b"],
                     help="d20_decode is the benchmark line; the others are side measurements of the remaining configurations")
     args = ap.parse_args()
