@@ -864,11 +864,11 @@ static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *res
   // launches of a sweep fill the GPU; they gain nothing from it (measured: 2-8 % slower) and are launched normally.
   struct PdlScope {
     snlp_model *m;
-    explicit PdlScope(snlp_model *m_) : m(m_) { m->pdl_now = m->use_pdl != 0; }
+    PdlScope(snlp_model *m_, int rows) : m(m_) { m->pdl_now = m->use_pdl != 0 && rows <= kDecodeRows; }   // decode regime only
     ~PdlScope() { m->pdl_now = false; }
   };
   if (S > 0) {  // Alg. 2 lines 2-4
-    PdlScope pdl(m);
+    PdlScope pdl(m, f.M);
     if (umma_path_ok(m)) TRY(prep_rows(m, f, 0, 1));
     else TRY(premix(m, f, 0, 1));
     for (int l = 0; l < S; ++l) {
@@ -878,7 +878,7 @@ static int solve(snlp_model *m, const Fwd &f, const snlp_solver &sol, float *res
   }
   if (S == L) return SNLP_OK;
   if (seq) {  // sequential execution of the fused model: chunk after chunk
-    PdlScope pdl(m);
+    PdlScope pdl(m, f.M);
     if (umma_path_ok(m)) TRY(prep_rows(m, f, S, 1));
     for (int h = S; h < L; h += F) {
       TRY(run_blocks(m, f, h, F, F));

@@ -67,3 +67,39 @@ def test_static_lm_head_rejects_sizes_beyond_its_fixed_scratch():
                                    1, cfg.rms_eps)
     assert e.value.code == snlp.ERR_UNSUPPORTED
     torch.cuda.synchronize()
+
+
+def _torch_logits(hL, head_bits, n_streams, eps):
+    """fp32 logits of the same bf16 product on the GPU (plain torch ops: a test-side check, not the product path)."""
+    x = hL.sum(dim=1) if hL.dim() == 3 else hL
+    rstd = torch.rsqrt((x * x).mean(-1, keepdim=True) + eps)
+    xb = x.to(torch.bfloat16).float()
+    w = head_bits.view(torch.bfloat16).float()
+    return (xb @ w.T) * rstd
+
+
+@pytest.mark.parametrize("rows,d_model,vocab,n_streams", [(16, 4096, 2048, 1), (16, 32, 262144, 1), (9, 1280, 65536, 4)])
+def test_static_lm_head_at_the_ends_of_its_limits(rows, d_model, vocab, n_streams):
+    """The largest row count with the widest model (the two-tile variant with its large shared-memory request), the
+    whole scratch array (largest vocabulary), and the benchmark's own head shape; and the property the entry point
+    exists for: the device's free memory is the same before and after a call."""
+    from paper_2605_17842_b200 import snlp
+    g = torch.Generator(device="cuda").manual_seed(1234 + rows + d_model)
+    hL = torch.randn((rows, n_streams, d_model), device="cuda", generator=g)
+    head = (torch.randn((vocab, d_model), device="cuda", generator=g) * 0.05).to(torch.bfloat16).view(torch.int16)
+    out = torch.full((rows,), -7, dtype=torch.int32, device="cuda")
+    snlp.lm_head_greedy_static(hL, head, n_streams, 1e-6, argmax=out)      # first call on the device does the set-up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    out.fill_(-7)
+    snlp.lm_head_greedy_static(hL, head, n_streams, 1e-6, argmax=out)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, (free0, free1)
+    logits = _torch_logits(hL, head, n_streams, 1e-6)
+    got = out.long()
+    assert int(got.min()) >= 0 and int(got.max()) < vocab
+    top = logits.max(dim=-1).values
+    chosen = logits.gather(1, got[:, None])[:, 0]
+    # the chosen token is the maximum up to the rounding noise of two fp32 sums of d_model bf16 products
+    assert bool(torch.all(top - chosen <= 2e-5 * logits.abs().max() + 1e-6)), (top - chosen)
