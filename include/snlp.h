@@ -232,6 +232,9 @@ int snlp_draft_and_verify_async(snlp_model *m, snlp_kv *kv, int32_t *last_tok, i
  * flag 4: programmatic dependent launch between the kernels of layer-by-layer execution (sequential forward, sequential
  *         prefix; default 1): a kernel is scheduled while its predecessor finishes and requests its first weight tiles
  *         before it waits for that kernel's results.  The launches of a sweep never use it.
+ * flag 5: decode regime: run the three products that follow the attention (out-projection, MLP up, MLP down) as one
+ *         cooperative launch with grid barriers between them (default 1); 0 = three launches.  Same results bit for bit.
+ *         Under flag 2 the one launch is booked under the MLP-up class.
  * flag 3: failure-detection test hook: waits for the device, then writes `value != 0` into the error word that a
  *         kernel raises when one of its bounded waits expires; snlp_device_status then reports it exactly as it
  *         would report a real expiry (no kernel is made to wait). */

@@ -18,6 +18,7 @@
 #include "generic.cuh"
 #include "umma_gemm.cuh"
 #include "umma_gemm2.cuh"
+#include "umma_chain.cuh"
 #include "attn_umma.cuh"
 
 using namespace snlp;
@@ -97,12 +98,13 @@ struct snlp_model {
   unsigned *counter = nullptr, *attn_counters = nullptr;
   int *zero = nullptr;
   unsigned *lm_counter = nullptr;   // arrival counter of the LM-head launch (zero between launches)
+  unsigned *chain_bar = nullptr;    // grid-barrier counter of the chained decode-regime products (zero between launches)
   int32_t *spec = nullptr;  // [2 * (max_rows + 1)] ids / verifier tokens for draft-and-verify
   int32_t *tok_pin = nullptr, *tok_dev = nullptr;   // [2][max_batch] mapped pinned host memory (tokens in, tokens out) and its device address (snlp_decode_step_host)
   int logit_rows = 0;
   std::vector<void *> allocs;
   // flags / stats
-  int use_graphs = 1, force_generic = 0, timing = 0, use_pdl = 1;
+  int use_graphs = 1, force_generic = 0, timing = 0, use_pdl = 1, use_chain = 1;
   bool pdl_now = false;   // launches issued right now carry the programmatic-serialisation attribute (layer-by-layer execution only)
   std::vector<PendingTime> pending;
   std::vector<cudaEvent_t> free_events;
@@ -308,6 +310,7 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
   A(&m->attn_counters, L * (size_t)kDecodeRows * c.n_head * 4);
   A(&m->zero, 16);
   A(&m->lm_counter, 16);
+  A(&m->chain_bar, 16);
   A(&m->spec, 2 * (R + 1) * 4);
   A(&m->tok_slot, 2 * sizeof(void *));
   if (rc == SNLP_OK && (cudaHostAlloc((void **)&m->tok_pin, (size_t)2 * c.max_batch * 4, cudaHostAllocMapped) != cudaSuccess ||
@@ -316,7 +319,7 @@ extern "C" int snlp_create(const snlp_config *cfg, snlp_model **out) {
     rc = fail(SNLP_ERR_OOM, "cudaHostAlloc of the token staging buffer failed");
   }
   if (rc == SNLP_OK) {
-    if (cudaMemset(m->dev_err, 0, 16) != cudaSuccess || cudaMemset(m->attn_counters, 0, L * (size_t)kDecodeRows * c.n_head * 4) != cudaSuccess || cudaMemset(m->counter, 0, 16) != cudaSuccess || cudaMemset(m->zero, 0, 16) != cudaSuccess || cudaMemset(m->lm_counter, 0, 16) != cudaSuccess)
+    if (cudaMemset(m->dev_err, 0, 16) != cudaSuccess || cudaMemset(m->attn_counters, 0, L * (size_t)kDecodeRows * c.n_head * 4) != cudaSuccess || cudaMemset(m->counter, 0, 16) != cudaSuccess || cudaMemset(m->zero, 0, 16) != cudaSuccess || cudaMemset(m->lm_counter, 0, 16) != cudaSuccess || cudaMemset(m->chain_bar, 0, 16) != cudaSuccess)
       rc = fail(SNLP_ERR_CUDA, "cudaMemset failed");
   }
   if (rc == SNLP_OK) {
@@ -447,6 +450,14 @@ extern "C" int snlp_set_flag(snlp_model *m, int flag, int value) {
     }
     m->use_pdl = value != 0;
   }
+  else if (flag == 5) {
+    if (m->use_chain != (value != 0)) {   // captured decode steps were recorded with the other launch sequence
+      CU(cudaDeviceSynchronize());
+      for (auto &g : m->graphs) cudaGraphExecDestroy(g.second.exec);
+      m->graphs.clear();
+    }
+    m->use_chain = value != 0;
+  }
   else if (flag == 3) {   // host-side injection of the error word a kernel raises when a bounded wait expires
     const int v = value != 0;
     CU(cudaDeviceSynchronize());
@@ -490,6 +501,7 @@ extern "C" int snlp_device_status(snlp_model *m, void *stream) {
     cudaMemset(m->dev_err, 0, sizeof flag);
     // a kernel that gave up may have left arrival counters part-way: bring them back to zero for the calls that follow
     cudaMemset(m->lm_counter, 0, 16);
+    cudaMemset(m->chain_bar, 0, 16);
     cudaMemset(m->counter, 0, 16);
     cudaMemset(m->attn_counters, 0, (size_t)m->cfg.n_layer * kDecodeRows * m->cfg.n_head * 4);
     return fail(SNLP_ERR_TIMEOUT, "a device-side bounded wait expired; results of the calls since the last check are invalid");
@@ -640,55 +652,105 @@ static cudaError_t umma_attr_all() {
   return e;
 }
 
-// C[l] = A[l] (M x K bf16, activations) * W[l0 + l]^T (N x K bf16, stacked weights), nl layers, `ksplit` K slices.
-template <int EPI>
-static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat16 *A, size_t a_ls, const WMap &w, int l0, UmmaParams p,
-                     int M, int N, int K, int ksplit, int nl) {
-  const bool small = M <= kDecodeRows;
-  if (EPI == UEPI_LMHEAD && !small) return fail(SNLP_ERR_UNSUPPORTED, "LM-head epilogue needs <= %d rows", kDecodeRows);
+// Column width of a decode-regime launch.  A launch that does not occupy every SM (a sequential step's single layer: 5-20
+// items) lasts as long as one item.  The column tiling does not touch the numbers (every output column is its own dot
+// product), so a launch whose 128-wide items still fit one round over the SMs takes those: twice the CTAs, half the bytes
+// each.  Beyond that the 256-wide tile is the faster one (a 128-wide MMA costs as much as a 256-wide one, which caps a
+// CTA streaming 128-wide tiles at ~50 GB/s).  The out-projection's partial sums of squares are per 128 columns in this
+// regime, whatever the tile width.
+static int decode_bn(const snlp_model *m, const WMap &w, int N, int ksplit, int nl) {
+  return (w.BN == 256 && (N / 128) * ksplit * nl <= m->n_sm) ? 128 : w.BN;
+}
+
+// A product ready to be launched: C[l] = A[l] (M x K bf16, activations) * W[l0 + l]^T (N x K bf16, stacked weights), nl
+// layers, `ksplit` K slices.
+struct GemmLaunch {
   CUtensorMap ta;
+  const CUtensorMap *tmw;
+  UmmaParams p;
+  int bn, grid;
+  bool small, pairs;
+};
+
+// bn_force: 0 = choose the column width; 128 / 256 = use that one (decode regime; the phases of a chained launch share it)
+static int umma_prepare(snlp_model *m, GemmLaunch &g, int epi, const __nv_bfloat16 *A, size_t a_ls, const WMap &w, int l0, UmmaParams p, int M, int N,
+                        int K, int ksplit, int nl, int bn_force = 0) {
+  const bool small = M <= kDecodeRows;
+  if (epi == UEPI_LMHEAD && !small) return fail(SNLP_ERR_UNSUPPORTED, "LM-head epilogue needs <= %d rows", kDecodeRows);
   if (p.a_share < 1) p.a_share = 1;
   if (p.kfuse < 1) p.kfuse = 1;
-  if (!make_tmap_bf16(m->encode_tiled, &ta, A, K, M, (uint64_t)nl * p.kfuse, a_ls ? a_ls : (size_t)M * K, small ? 16 : kUmmaBM))
+  if (!make_tmap_bf16(m->encode_tiled, &g.ta, A, K, M, (uint64_t)nl * p.kfuse, a_ls ? a_ls : (size_t)M * K, small ? 16 : kUmmaBM))
     return fail(SNLP_ERR_CUDA, "cuTensorMapEncodeTiled failed (M=%d K=%d)", M, K);
-  if (p.a_share < 1) p.a_share = 1;
-  if (p.kfuse < 1) p.kfuse = 1;
   p.M = M; p.N = N; p.K = K; p.ksplit = ksplit; p.kslice = K / ksplit;
   p.Mt = small ? 1 : (M + kUmmaBM - 1) / kUmmaBM; p.Nt = N / w.BN; p.nl = nl; p.l0 = l0; p.err = m->dev_err;
-  if (!small && w.BN == 256 && M > kUmmaBM && EPI != UEPI_LMHEAD) {
+  g.small = small;
+  g.pairs = !small && w.BN == 256 && M > kUmmaBM && epi != UEPI_LMHEAD;
+  if (g.pairs) {
     // prefill regime with more than one row tile: 256 x 256 tiles on CTA pairs (same results, less operand traffic per SM)
     p.Mt = (M + 2 * kUmmaBM - 1) / (2 * kUmmaBM);
     p.nstages = kU2Stages;
     const int items2 = p.Mt * p.Nt * ksplit * nl, pairs = items2 < m->n_sm / 2 ? items2 : m->n_sm / 2;
-    KLAUNCH(m, st, cls, k_umma_gemm2<EPI><<<2 * pairs, kUmmaThreads, kU2Smem, st>>>(ta, w.tm_half, p));
+    g.bn = 256; g.grid = 2 * pairs; g.tmw = &w.tm_half; g.p = p;
     return SNLP_OK;
   }
-  // Decode regime: a launch that does not occupy every SM (a sequential step's single layer: 5-20 items) lasts as long
-  // as one item.  The column tiling does not touch the numbers (every output column is its own dot product), so a
-  // launch whose 128-wide items still fit one round over the SMs takes those: twice the CTAs, half the bytes each.
-  // Beyond that the 256-wide tile is the faster one (a 128-wide MMA costs as much as a 256-wide one, which caps a
-  // CTA streaming 128-wide tiles at ~50 GB/s).  The
-  // out-projection's partial sums of squares are per 128 columns in this regime, whatever the tile width.
   int bn = w.BN;
-  if (small && w.BN == 256 && (N / 128) * ksplit * nl <= m->n_sm) bn = 128;
-  const CUtensorMap &tmw = bn == w.BN ? w.tm : w.tm_half;
+  if (small) bn = bn_force ? bn_force : decode_bn(m, w, N, ksplit, nl);
+  g.tmw = bn == w.BN ? &w.tm : &w.tm_half;
   p.Nt = N / bn;
-  const bool pdl_ = m->pdl_now;
   const int items = p.Mt * p.Nt * ksplit * nl;
-  const int grid = items < m->n_sm ? items : m->n_sm;
+  g.bn = bn; g.grid = items < m->n_sm ? items : m->n_sm;
+  g.p = p;
+  return SNLP_OK;
+}
+
+template <int EPI>
+static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat16 *A, size_t a_ls, const WMap &w, int l0, UmmaParams p,
+                     int M, int N, int K, int ksplit, int nl) {
+  GemmLaunch g;
+  TRY(umma_prepare(m, g, EPI, A, a_ls, w, l0, p, M, N, K, ksplit, nl));
+  if (g.pairs) {
+    KLAUNCH(m, st, cls, k_umma_gemm2<EPI><<<g.grid, kUmmaThreads, kU2Smem, st>>>(g.ta, *g.tmw, g.p));
+    return SNLP_OK;
+  }
+  const bool pdl_ = m->pdl_now;
 #define SNLP_UMMA_LAUNCH(BN_, AM_)                                                                                                   \
   do {                                                                                                                               \
-    p.nstages = UmmaCfg<BN_, AM_>::kStages;                                                                                          \
-    KLAUNCH(m, st, cls, launch_pdl(pdl_, k_umma_gemm<BN_, AM_, EPI>, dim3(grid), dim3(kUmmaThreads), UmmaCfg<BN_, AM_>::kSmem, st, ta, tmw, p)); \
+    g.p.nstages = UmmaCfg<BN_, AM_>::kStages;                                                                                        \
+    KLAUNCH(m, st, cls, launch_pdl(pdl_, k_umma_gemm<BN_, AM_, EPI>, dim3(g.grid), dim3(kUmmaThreads), UmmaCfg<BN_, AM_>::kSmem, st, g.ta, *g.tmw, g.p)); \
   } while (0)
-  if (bn == 256) {
-    if (small) SNLP_UMMA_LAUNCH(256, 16);
+  if (g.bn == 256) {
+    if (g.small) SNLP_UMMA_LAUNCH(256, 16);
     else if (EPI != UEPI_LMHEAD) SNLP_UMMA_LAUNCH(256, 128);
   } else {
-    if (small) SNLP_UMMA_LAUNCH(128, 16);
+    if (g.small) SNLP_UMMA_LAUNCH(128, 16);
     else if (EPI != UEPI_LMHEAD) SNLP_UMMA_LAUNCH(128, 128);
   }
 #undef SNLP_UMMA_LAUNCH
+  return SNLP_OK;
+}
+
+// Decode regime: the three products that follow the attention -- out-projection, MLP up, MLP down -- as one cooperative
+// launch whose phases are separated by grid barriers (umma_chain.cuh).  Same items and epilogues as three launches.
+static int umma_chain3(snlp_model *m, cudaStream_t st, GemmLaunch (&g)[3], const int (&epi)[3]) {
+  ChainParams cp{};
+  cp.nphase = 3;
+  cp.bar = m->chain_bar;
+  for (int i = 0; i < 3; ++i) {
+    cp.tmA[i] = g[i].ta; cp.tmB[i] = *g[i].tmw; cp.p[i] = g[i].p; cp.epi[i] = epi[i];
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(m->n_sm); cfg.blockDim = dim3(kUmmaThreads); cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;   // every CTA must be resident: they wait for one another at the phase barriers
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  if (g[0].bn == 256) {
+    cfg.dynamicSmemBytes = UmmaCfg<256, 16>::kSmem;
+    KLAUNCH(m, st, KC_UP, cudaLaunchKernelEx(&cfg, k_umma_chain<256>, cp));
+  } else {
+    cfg.dynamicSmemBytes = UmmaCfg<128, 16>::kSmem;
+    KLAUNCH(m, st, KC_UP, cudaLaunchKernelEx(&cfg, k_umma_chain<128>, cp));
+  }
   return SNLP_OK;
 }
 
@@ -742,26 +804,31 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
     const int grid = ap.n_items < m->n_sm ? ap.n_items : m->n_sm;
     KLAUNCH(m, st, KC_ATTN, k_attn_umma<<<grid, kFuThreads, kFuSmem, st>>>(tq, tk, tv, to, ap, nl));
   }
-  {
-    UmmaParams p{};
-    p.c = a; p.z = ub; p.out_ls = Md;
-    p.xm = xm_src; p.xm_ls = implicit ? 0 : Md; p.coef = m->coef + l0; p.ssq_out = m->ssq_u + (size_t)l0 * Pu * M;
-    p.kfuse = fuse;   // a chunk's out-projections are one product over the concatenated attention outputs
-    TRY(umma_gemm<UEPI_RESID>(m, st, KC_OPROJ, att, Md, m->w_o, l0, p, M, d, d, 1, nl / fuse));
+  UmmaParams po{}, pu{}, pd{};
+  po.c = a; po.z = ub; po.out_ls = Md;
+  po.xm = xm_src; po.xm_ls = implicit ? 0 : Md; po.coef = m->coef + l0; po.ssq_out = m->ssq_u + (size_t)l0 * Pu * M;
+  po.kfuse = fuse;   // a chunk's out-projections are one product over the concatenated attention outputs
+  pu.z = z; pu.out_ls = (size_t)M * ff;
+  pu.ssq = m->ssq_u + (size_t)l0 * Pu * M; pu.nparts = Pu; pu.eps = c.rms_eps;
+  pu.a_share = fuse;
+  pd.c = mb; pd.out_ls = Md; pd.out_ss = (size_t)L * Md;
+  pd.kfuse = fuse;
+  if (small && m->use_chain) {
+    // one cooperative launch for the three products; a common column width: 256 as soon as one of them wants it
+    const int b0 = decode_bn(m, m->w_o, d, 1, nl / fuse), b1 = decode_bn(m, m->w_up, ff, 1, nl), b2 = decode_bn(m, m->w_dn, d, sd, nl / fuse);
+    const bool all256 = m->w_o.BN == 256 && m->w_up.BN == 256 && m->w_dn.BN == 256;
+    const int bn = (all256 && (b0 == 256 || b1 == 256 || b2 == 256)) ? 256 : 128;
+    GemmLaunch g[3];
+    TRY(umma_prepare(m, g[0], UEPI_RESID, att, Md, m->w_o, l0, po, M, d, d, 1, nl / fuse, bn));
+    TRY(umma_prepare(m, g[1], UEPI_RELU2_BF16, ub, Md, m->w_up, l0, pu, M, ff, d, 1, nl, bn));
+    TRY(umma_prepare(m, g[2], UEPI_F32, z, (size_t)M * ff, m->w_dn, l0, pd, M, d, ff, sd, nl / fuse, bn));
+    const int epi[3] = {UEPI_RESID, UEPI_RELU2_BF16, UEPI_F32};
+    TRY(umma_chain3(m, st, g, epi));
+    return SNLP_OK;
   }
-  {
-    UmmaParams p{};
-    p.z = z; p.out_ls = (size_t)M * ff;
-    p.ssq = m->ssq_u + (size_t)l0 * Pu * M; p.nparts = Pu; p.eps = c.rms_eps;
-    p.a_share = fuse;
-    TRY(umma_gemm<UEPI_RELU2_BF16>(m, st, KC_UP, ub, Md, m->w_up, l0, p, M, ff, d, 1, nl));
-  }
-  {
-    UmmaParams p{};
-    p.c = mb; p.out_ls = Md; p.out_ss = (size_t)L * Md;
-    p.kfuse = fuse;
-    TRY(umma_gemm<UEPI_F32>(m, st, KC_DOWN, z, (size_t)M * ff, m->w_dn, l0, p, M, d, ff, sd, nl / fuse));
-  }
+  TRY(umma_gemm<UEPI_RESID>(m, st, KC_OPROJ, att, Md, m->w_o, l0, po, M, d, d, 1, nl / fuse));
+  TRY(umma_gemm<UEPI_RELU2_BF16>(m, st, KC_UP, ub, Md, m->w_up, l0, pu, M, ff, d, 1, nl));
+  TRY(umma_gemm<UEPI_F32>(m, st, KC_DOWN, z, (size_t)M * ff, m->w_dn, l0, pd, M, d, ff, sd, nl / fuse));
   return SNLP_OK;
 }
 
@@ -791,6 +858,8 @@ static int init_kernel_attributes() {
   CU(umma_attr_all<UEPI_RESID>());
   CU((umma_attr<128, 16, UEPI_LMHEAD>()));
   CU((umma_attr<256, 16, UEPI_LMHEAD>()));
+  CU(cudaFuncSetAttribute(k_umma_chain<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<128, 16>::kSmem));
+  CU(cudaFuncSetAttribute(k_umma_chain<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<256, 16>::kSmem));
   CU(cudaFuncSetAttribute(k_attn_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, kFuSmem));
 #define ATTR(NS) CU(cudaFuncSetAttribute(k_correct<NS, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(corr_ring_bytes(NS, 256) + kCorrExtraSmem))); \
   CU(cudaFuncSetAttribute(k_correct<NS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(corr_ring_bytes(NS, 256) + kCorrExtraSmem)));
