@@ -24,11 +24,29 @@ __device__ __forceinline__ uint4 ldg_stream(const void *p) {
 constexpr int kAttnPartStride = 132;
 constexpr int kAttnSub = 64;
 
+// One output row from the chunk partials of its (layer, sequence, head, query): the chunks are merged in chunk order.
+// src: [nchunk][kAttnPartStride]; e = the head feature this thread produces.  Used by k_attn_decode's last-arriver
+// merge and by the chained launch that follows the attention, so both give the same bits.
+__device__ __forceinline__ float attn_merge_row(const float *src, int nchunk, int e) {
+  float M = -INFINITY;
+  for (int c = 0; c < nchunk; ++c) M = fmaxf(M, __ldcg(src + (size_t)c * kAttnPartStride + 128));
+  float o = 0.f, den = 0.f;
+  for (int c = 0; c < nchunk; ++c) {
+    const float mc = __ldcg(src + (size_t)c * kAttnPartStride + 128);
+    const float w = mc == -INFINITY ? 0.f : __expf(mc - M);
+    o = fmaf(w, __ldcg(src + (size_t)c * kAttnPartStride + e), o);
+    den = fmaf(w, __ldcg(src + (size_t)c * kAttnPartStride + 129), den);
+  }
+  return o / den;
+}
+
+// merge_here == 0: the CTAs only leave their chunk partials behind (the kernel that follows merges them); no fence, no
+// arrival counter, no tail.
 static __global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat16 *__restrict__ q, size_t q_ls,
                                                         const __nv_bfloat16 *__restrict__ kc, const __nv_bfloat16 *__restrict__ vc,
                                                         size_t kv_ls, size_t kv_bs, float *__restrict__ part,
                                                         unsigned *__restrict__ counters, __nv_bfloat16 *__restrict__ out,
-                                                        size_t o_ls, int Tq, int H, const int *__restrict__ pos_base, int csub) {
+                                                        size_t o_ls, int Tq, int H, const int *__restrict__ pos_base, int csub, int merge_here) {
   __shared__ float qs[16][128];
   __shared__ float hacc[8][128];
   __shared__ float hm[8], hl[8];
@@ -154,6 +172,7 @@ static __global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat
   }
   // ---- last CTA of this (layer, sequence, head) merges the chunks in chunk order --------------------
   pdl_trigger();   // the chunk has been streamed: only the merge is left
+  if (!merge_here) return;
   __threadfence();
   __syncthreads();
   if (tid == 0) s_last = atomicAdd(&counters[(size_t)l * gridDim.y + bh], 1u) == (unsigned)nchunk - 1;
@@ -162,16 +181,7 @@ static __global__ void __launch_bounds__(128, 4) k_attn_decode(const __nv_bfloat
   __threadfence();
   for (int t = 0; t < Tq; ++t) {
     const float *src = pbase + (size_t)t * nchunk * kAttnPartStride;
-    float M = -INFINITY;
-    for (int c = 0; c < nchunk; ++c) M = fmaxf(M, __ldcg(src + (size_t)c * kAttnPartStride + 128));
-    float o = 0.f, den = 0.f;
-    for (int c = 0; c < nchunk; ++c) {
-      const float mc = __ldcg(src + (size_t)c * kAttnPartStride + 128);
-      const float w = mc == -INFINITY ? 0.f : __expf(mc - M);
-      o = fmaf(w, __ldcg(src + (size_t)c * kAttnPartStride + tid), o);
-      den = fmaf(w, __ldcg(src + (size_t)c * kAttnPartStride + 129), den);
-    }
-    out[(size_t)l * o_ls + (size_t)(b * Tq + t) * d + h * 128 + tid] = __float2bfloat16_rn(o / den);
+    out[(size_t)l * o_ls + (size_t)(b * Tq + t) * d + h * 128 + tid] = __float2bfloat16_rn(attn_merge_row(src, nchunk, tid));
   }
   if (tid == 0) counters[(size_t)l * gridDim.y + bh] = 0u;
 }

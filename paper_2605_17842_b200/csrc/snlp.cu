@@ -731,8 +731,7 @@ static int umma_gemm(snlp_model *m, cudaStream_t st, int cls, const __nv_bfloat1
 
 // Decode regime: the three products that follow the attention -- out-projection, MLP up, MLP down -- as one cooperative
 // launch whose phases are separated by grid barriers (umma_chain.cuh).  Same items and epilogues as three launches.
-static int umma_chain3(snlp_model *m, cudaStream_t st, GemmLaunch (&g)[3], const int (&epi)[3]) {
-  ChainParams cp{};
+static int umma_chain3(snlp_model *m, cudaStream_t st, GemmLaunch (&g)[3], const int (&epi)[3], ChainParams &cp) {
   cp.nphase = 3;
   cp.bar = m->chain_bar;
   for (int i = 0; i < 3; ++i) {
@@ -777,6 +776,9 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
   T *kc = (T *)f.kc + (size_t)l0 * f.kv_ls, *vc = (T *)f.vc + (size_t)l0 * f.kv_ls;
   const int Pu = small ? d / 128 : 2 * (d / m->w_o.BN);  // partials of sum u^2: one per 128 columns (decode regime), two per column tile of the out-projection
   const int sd = down_splits(m, M);
+  const bool chained = small && m->use_chain;   // the three products after the attention as one launch, which also merges the attention's chunk partials
+  int comb_nchunk = 0;
+  bool comb = false;
   {
     UmmaParams p{};
     p.ssq = m->ssq_x + (size_t)l0 * P * M; p.nparts = P; p.eps = c.rms_eps;
@@ -788,8 +790,17 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
   if (small) {
     const int csub = attn_csub(f.B * H);
     const int nchunk = (f.pos_hi + f.T - 1) / (csub * kAttnSub) + 1;
+    // Where the chunk partials are merged.  In the attention kernel itself the CTA that arrives last at its (layer,
+    // sequence, head) merges them, which puts a device-scope fence and an atomic round trip at the end of every CTA; with
+    // only a few waves of CTAs (a batch-1 sweep: ~3) that tail is a fifth of the launch, and the chained launch that
+    // follows merges them instead (measured: attention 46.6 -> 40.5 us, chained launch 105 -> 108 us).  With many waves
+    // (batch 8) or a single layer the tail is hidden or the chain's extra step costs as much: merged in place.  The same
+    // function merges in both places: no bit depends on the choice.
+    comb = chained && nl > 1 && (long long)nchunk * f.B * H * nl <= 16LL * m->n_sm;
     KLAUNCH(m, st, KC_ATTN, launch_pdl(m->pdl_now, k_attn_decode, dim3(nchunk, f.B * H, nl), dim3(128), 0, st, (const __nv_bfloat16 *)q, Md, (const __nv_bfloat16 *)kc,
-                                       (const __nv_bfloat16 *)vc, f.kv_ls, f.kv_bs, m->attn_part, m->attn_counters, att, Md, f.T, H, f.pos, csub));
+                                       (const __nv_bfloat16 *)vc, f.kv_ls, f.kv_bs, m->attn_part, m->attn_counters, att, Md, f.T, H, f.pos, csub,
+                                       comb ? 0 : 1));
+    comb_nchunk = nchunk;
   } else {
     // tensor-core attention: 128-query items over the (layer, sequence, head, query tile) grid, persistent CTAs
     CUtensorMap tq, tk, tv, to;
@@ -813,7 +824,7 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
   pu.a_share = fuse;
   pd.c = mb; pd.out_ls = Md; pd.out_ss = (size_t)L * Md;
   pd.kfuse = fuse;
-  if (small && m->use_chain) {
+  if (chained) {
     // one cooperative launch for the three products; a common column width: 256 as soon as one of them wants it
     const int b0 = decode_bn(m, m->w_o, d, 1, nl / fuse), b1 = decode_bn(m, m->w_up, ff, 1, nl), b2 = decode_bn(m, m->w_dn, d, sd, nl / fuse);
     const bool all256 = m->w_o.BN == 256 && m->w_up.BN == 256 && m->w_dn.BN == 256;
@@ -823,7 +834,10 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
     TRY(umma_prepare(m, g[1], UEPI_RELU2_BF16, ub, Md, m->w_up, l0, pu, M, ff, d, 1, nl, bn));
     TRY(umma_prepare(m, g[2], UEPI_F32, z, (size_t)M * ff, m->w_dn, l0, pd, M, d, ff, sd, nl / fuse, bn));
     const int epi[3] = {UEPI_RESID, UEPI_RELU2_BF16, UEPI_F32};
-    TRY(umma_chain3(m, st, g, epi));
+    ChainParams cp{};
+    cp.comb_part = m->attn_part; cp.comb_out = att; cp.comb_o_ls = Md;
+    cp.comb_rows = comb ? nl * f.B * H * f.T : 0; cp.comb_nchunk = comb_nchunk; cp.comb_Tq = f.T; cp.comb_BH = f.B * H; cp.comb_H = H; cp.comb_d = d;
+    TRY(umma_chain3(m, st, g, epi, cp));
     return SNLP_OK;
   }
   TRY(umma_gemm<UEPI_RESID>(m, st, KC_OPROJ, att, Md, m->w_o, l0, po, M, d, d, 1, nl / fuse));

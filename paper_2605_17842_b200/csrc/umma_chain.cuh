@@ -13,6 +13,7 @@
 // back to zero.  The kernel needs all its CTAs resident
 // (one per SM): it is launched cooperatively.  All waits are bounded as in k_umma_gemm.
 #pragma once
+#include "decode.cuh"
 #include "umma_gemm.cuh"
 
 namespace snlp {
@@ -25,6 +26,10 @@ struct ChainParams {
   int epi[kChainMax];                           // UEPI_* of the phase
   int nphase;
   unsigned *bar;                                // grid-barrier counter
+  // Optional first step: merge the split-KV partials the decode attention left behind (k_attn_decode with merge_here = 0)
+  // into the bf16 attention output that phase 0 reads.  comb_rows = layers x sequences x heads x queries (0 = no such step).
+  const float *comb_part; __nv_bfloat16 *comb_out; size_t comb_o_ls;
+  int comb_rows, comb_nchunk, comb_Tq, comb_BH, comb_H, comb_d;
 };
 
 __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned *p) {
@@ -78,6 +83,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_chain(const __grid_con
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = (int)gridDim.x;
+  const int pre = cp.comb_rows > 0 ? 1 : 0;   // barriers before phase 0
   int *err = cp.p[0].err;
   constexpr uint32_t kTmemCols = 2 * BN;
 
@@ -126,10 +132,10 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_chain(const __grid_con
         // The activation tiles of this phase may only be requested once the phase is open; its weight tiles go out at
         // once.  pend_*: the stages of this phase whose activation tile is still to be requested (at most S of them:
         // a stage cannot be reused before the product that reads it has run, and that needs its activations).
-        bool open = ph == 0;
+        bool open = ph == 0 && pre == 0;
         int pend_from = g;
         int pend_k0[S], pend_la[S];
-        const unsigned target = (unsigned)ph * (unsigned)G;
+        const unsigned target = (unsigned)(ph + pre) * (unsigned)G;
         auto flush = [&]() {
           asm volatile("fence.proxy.async;" ::: "memory");   // the other CTAs' stores, seen through the barrier, before the bulk copies that read them
           for (int q = pend_from; q < g; ++q)
@@ -201,6 +207,19 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_chain(const __grid_con
     const int quarter = warp & 3;
     int n = 0;
     bool alive = true;
+    if (pre) {
+      // merge the attention's chunk partials: one output row (128 head features) per group of four warps at a time
+      const int grp4 = et >> 7, e = et & 127;
+      for (int r = (int)blockIdx.x + G * grp4; r < cp.comb_rows; r += 2 * G) {
+        const int t = r % cp.comb_Tq, pair = r / cp.comb_Tq, bh = pair % cp.comb_BH, l = pair / cp.comb_BH;
+        const int b = bh / cp.comb_H, h = bh % cp.comb_H;
+        const float v = attn_merge_row(cp.comb_part + (size_t)r * cp.comb_nchunk * kAttnPartStride, cp.comb_nchunk, e);
+        cp.comb_out[(size_t)l * cp.comb_o_ls + (size_t)(b * cp.comb_Tq + t) * cp.comb_d + h * 128 + e] = __float2bfloat16_rn(v);
+      }
+      __threadfence();
+      epi_bar_sync();
+      if (et == 0) atomicAdd(cp.bar, 1u);
+    }
     for (int ph = 0; ph < cp.nphase; ++ph) {
       SNLP_CHAIN_PHASE(ph)
       (void)nkb;
@@ -233,9 +252,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_chain(const __grid_con
       __threadfence();
       epi_bar_sync();
       if (et == 0) {
-        if (ph > 0 && my_items == 0 && alive) chain_wait(cp.bar, (unsigned)ph * (unsigned)G, abort_flag, err);
+        if (ph + pre > 0 && my_items == 0 && alive) chain_wait(cp.bar, (unsigned)(ph + pre) * (unsigned)G, abort_flag, err);
         const unsigned old = atomicAdd(cp.bar, 1u);
-        if (old == (unsigned)cp.nphase * (unsigned)G - 1u) *cp.bar = 0u;   // the last arrival of the last phase: nobody polls any more
+        if (old == (unsigned)(cp.nphase + pre) * (unsigned)G - 1u) *cp.bar = 0u;   // the last arrival of the last phase: nobody polls any more
       }
     }
   }
