@@ -199,8 +199,10 @@ int snlp_decode_step(snlp_model *m, snlp_kv *kv, const int32_t *tok_in, int K, i
 
 /* snlp_decode_step for a caller that keeps its tokens on the host: tok_in_host and tok_out_host are HOST int32 [B]
  * (pageable or pinned; they may alias).  The tokens go through the library's own mapped pinned staging buffer, which
- * the step's kernels read and write across the bus; the call synchronises `stream` before returning, so tok_out_host
- * is valid on return.  One staging buffer per model: calls on the same model must not overlap.  Errors as
+ * the step's kernels read and write across the bus; the call returns once every output token has arrived in host memory
+ * (it watches the staging buffer; should the tokens not arrive within 50 ms it synchronises `stream` instead), so
+ * tok_out_host is valid on return.  The step's last kernel may still be retiring at that moment; later calls on the same
+ * stream are ordered behind it as usual.  One staging buffer per model: calls on the same model must not overlap.  Errors as
  * snlp_decode_step, plus CUDA. */
 int snlp_decode_step_host(snlp_model *m, snlp_kv *kv, const int32_t *tok_in_host, int K, int mode, int32_t *tok_out_host,
                           void *stream);

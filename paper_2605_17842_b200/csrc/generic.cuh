@@ -260,6 +260,7 @@ __global__ void k_argmax_rows(const float *__restrict__ logits, int vocab, int32
     for (int i = 1; i < nw; ++i)
       if (sv[i] > bv || (sv[i] == bv && si[i] < bi)) { bv = sv[i]; bi = si[i]; }
     out[blockIdx.x] = bi == 0x7fffffff ? 0 : bi;
+    __threadfence_system();   // the token buffer may be mapped host memory that the host is watching
   }
 }
 

@@ -3,6 +3,8 @@
 #include "../../include/snlp.h"
 
 #include <algorithm>
+#include <atomic>
+#include <chrono>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -1427,8 +1429,25 @@ extern "C" int snlp_decode_step_host(snlp_model *m, snlp_kv *kv, const int32_t *
   // gather fetches B ids across the bus and the LM-head kernel posts B ids back, with no copy operations around the graph.
   const size_t bytes = (size_t)kv->B * sizeof(int32_t);
   memcpy(m->tok_pin, tok_in_host, bytes);
+  // The host does not go through the stream's completion machinery (tens of microseconds of wake-up latency) to learn
+  // that the step is done: it marks the output slots with a value no token can take and watches them until the step's
+  // last kernel has stored every token (the stores travel straight over the bus).  If they do not arrive within a
+  // generous limit -- an error in the step, a device that is busy with other work -- it falls back to synchronising.
+  volatile int32_t *out = m->tok_pin + m->cfg.max_batch;
+  constexpr int32_t kNoToken = INT32_MIN;
+  for (int i = 0; i < kv->B; ++i) out[i] = kNoToken;
   TRY(snlp_decode_step(m, kv, m->tok_dev, K, mode, m->tok_dev + m->cfg.max_batch, nullptr, stream));
-  CU(cudaStreamSynchronize((cudaStream_t)stream));
+  bool seen = false;
+  const auto t0 = std::chrono::steady_clock::now();
+  for (uint32_t it = 0; !seen; ++it) {
+    seen = true;
+    for (int i = 0; i < kv->B; ++i) seen = seen && out[i] != kNoToken;
+    if (seen) break;
+    __builtin_ia32_pause();
+    if ((it & 1023u) == 1023u && std::chrono::steady_clock::now() - t0 > std::chrono::milliseconds(50)) break;
+  }
+  if (!seen) CU(cudaStreamSynchronize((cudaStream_t)stream));
+  std::atomic_thread_fence(std::memory_order_acquire);
   memcpy(tok_out_host, m->tok_pin + m->cfg.max_batch, bytes);
   return SNLP_OK;
 }

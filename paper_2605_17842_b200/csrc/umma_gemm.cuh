@@ -684,7 +684,10 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
             const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
             if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
           }
-          if (lane == 0) amax[tok] = (unsigned)bi < (unsigned)p.N ? bi : 0;
+          if (lane == 0) {
+            amax[tok] = (unsigned)bi < (unsigned)p.N ? bi : 0;
+            __threadfence_system();   // the token buffer may be mapped host memory that the host is watching
+          }
         }
         if (et == 0) {
           if (p.bump != nullptr) *p.bump += 1;

@@ -246,3 +246,31 @@ def test_decode_through_host_buffers_gives_the_same_tokens(cfg, B):
     with pytest.raises(snlp.SnlpError) as e:
         m.decode_step_host(kv, th, -1)
     assert e.value.code == snlp.ERR_ARG
+
+
+@pytest.mark.parametrize("cfg,B", [(BF16, 1), (BF16, 3), (synth.ModelConfig(3, 256, 2, 128, 512, 1024, 4, "bf16"), 2)])
+def test_chained_launch_gives_the_same_bits_as_three_launches(cfg, B):
+    """The decode regime runs out-projection, MLP up and MLP down as one cooperative launch (and, for a sweep with few
+    attention CTAs, merges the attention's chunk partials there); with flag 5 off they are three launches and the
+    attention merges its own partials.  Same items, same order of every sum: states and tokens must be identical."""
+    W = synth.make_weights(cfg, seed=1234, mix_seed=5, std=0.05, embed_std=1.0)
+    Tp = 300
+    ids = dev(synth.make_ids(cfg, B, Tp, seed=12))
+    mode = O.MODE_HCN if cfg.n_streams > 1 else O.MODE_IDN
+    outs = []
+    for chain in (1, 0):
+        m = make_model(cfg, W, max_rows=B * 100, max_batch=B, max_ctx=Tp + 16)
+        m.set_flag(5, chain)
+        kv = m.kv_cache(B, Tp + 16)
+        t = m.prefill(kv, ids)
+        rec = []
+        for K in (0, 2, cfg.n_layer, 2):
+            t = m.decode_step(kv, t, K, mode)
+            rec.append((t.clone(), m.copy_trace(B)))
+        tr, _ = m.forward_parallel(m.embed(ids[:, :5].contiguous()), 2, mode)   # 5 rows per sequence: still the decode regime
+        rec.append((tr, tr))
+        m.device_status()
+        outs.append(rec)
+        m.close()
+    for (t1, s1), (t0, s0) in zip(*outs):
+        assert torch.equal(t1, t0) and torch.equal(s1, s0)
