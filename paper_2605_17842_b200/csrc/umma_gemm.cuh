@@ -419,6 +419,11 @@ __device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const f
       const float *xs = p.xm + (size_t)l * p.xm_ls + (size_t)tok * p.N + n0;
       float *adst = p.c + (size_t)l * p.out_ls + (size_t)tok * p.N + n0;
       __nv_bfloat16 *udst = p.z + (size_t)l * p.out_ls + (size_t)tok * p.N + n0;
+      // (all the residual-stream values first: loads left between the stores below would be issued one at a time, one
+      // memory round trip each, and this epilogue is on the path between two phases of a chained launch)
+      float xv[BN / 32];
+#pragma unroll
+      for (int j = 0; j < BN / 32; ++j) xv[j] = xs[lane + 32 * j];
       // one partial sum of u^2 per 128 columns, so that 128- and 256-wide tiles leave the same numbers behind
 #pragma unroll
       for (int h = 0; h < BN / 128; ++h) {
@@ -426,7 +431,7 @@ __device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const f
 #pragma unroll
         for (int j = 4 * h; j < 4 * h + 4; ++j) {
           const float a = y[lane + 32 * j];
-          const float u = fmaf(kappa, a, xs[lane + 32 * j]);
+          const float u = fmaf(kappa, a, xv[j]);
           adst[lane + 32 * j] = a;
           udst[lane + 32 * j] = __float2bfloat16_rn(u);
           ss = fmaf(u, u, ss);
@@ -436,7 +441,10 @@ __device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const f
       }
     } else if (EPI == UEPI_QKV) {
       const int b = tok / p.T, pos = *p.pos_base + (tok % p.T);
-#pragma unroll 1
+      // the rotation table entries of this position, for every head of the tile, before anything is stored (a load
+      // that follows a store is not issued ahead of it: one memory round trip per head otherwise)
+      const float2 c0 = p.rope[(size_t)pos * 64 + lane], c1 = p.rope[(size_t)pos * 64 + lane + 32];
+#pragma unroll
       for (int hh = 0; hh < BN / 128; ++hh) {
         const int n = (int)n0 + hh * 128, kind = n / p.d, hcol = n % p.d;
         const float *yh = y + hh * 128;
@@ -447,7 +455,6 @@ __device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const f
 #pragma unroll
           for (int j = 0; j < 4; ++j) dst[lane + 32 * j] = __float2bfloat16_rn(yh[lane + 32 * j] * rstd);
         } else {
-          const float2 c0 = p.rope[(size_t)pos * 64 + lane], c1 = p.rope[(size_t)pos * 64 + lane + 32];
           const float a1 = yh[lane] * rstd, a2 = yh[lane + 64] * rstd, b1 = yh[lane + 32] * rstd, b2 = yh[lane + 96] * rstd;
           const float ya1 = a1 * c0.x - a2 * c0.y, ya2 = a1 * c0.y + a2 * c0.x;
           const float yb1 = b1 * c1.x - b2 * c1.y, yb2 = b1 * c1.y + b2 * c1.x;
