@@ -38,14 +38,6 @@ struct FaUmmaParams {
   int *err;
 };
 
-__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *tm, uint64_t *bar, int c0, int c1, int c2, int c3) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(
-          smem_u32(dst)),
-      "l"(tm), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-      : "memory");
-}
-
 // Shared-memory descriptor of an MN-major operand: rows of 128 bytes = 64 consecutive MN elements of one K index,
 // 128-byte swizzle; the next 8 K indices are 1024 bytes on, the next 64 MN elements `mn_stride` bytes on.
 __device__ __forceinline__ uint64_t umma_desc_sw128_mn(uint32_t smem_addr, uint32_t mn_stride) {

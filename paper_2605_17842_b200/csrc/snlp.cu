@@ -10,6 +10,7 @@
 #include <cstdio>
 #include <cstring>
 #include <map>
+#include <numeric>
 #include <string>
 #include <tuple>
 #include <vector>
@@ -76,7 +77,10 @@ struct GraphKey {
 };
 struct GraphEntry { cudaGraphExec_t exec; int64_t nodes; };
 struct PendingTime { int cls; cudaEvent_t e0, e1; };
-struct WMap { CUtensorMap tm, tm_half; int BN; };  // TMA maps over one stacked weight array, boxes {64, BN, 1} and (for CTA pairs) {64, 128, 1}
+// TMA maps over one stacked weight array: boxes {64, BN, 1} and (for CTA pairs) {64, 128, 1}; for the decode regime
+// td128[i] / td256[i] with boxes of 2^i k-blocks of 128 / 256 rows (those that divide nkb1, the k-blocks one decode-regime
+// item reduces over; td256 only when BN == 256).
+struct WMap { CUtensorMap tm, tm_half, td128[3], td256[2]; int BN, nkb1; };
 enum { KC_QKV = 0, KC_ATTN, KC_OPROJ, KC_UP, KC_DOWN, KC_CORRECT, KC_LMHEAD, KC_OTHER, KC_COUNT };
 static_assert(KC_COUNT == SNLP_NUM_KERNEL_CLASSES, "kernel class count");
 
@@ -159,6 +163,8 @@ static inline void count(snlp_model *m, int n = 1) {
   if (m->capturing) m->cap_nodes += n;
   else m->launches += n;
 }
+
+static int pick_ksplit(int K, int want);
 
 // Optional device timing of every launch, by kernel class (CUDA events on the launching stream).
 struct TimedLaunch {
@@ -427,13 +433,21 @@ extern "C" int snlp_load_weights(snlp_model *m, const snlp_weights *w) {
   CU(cudaMemcpy(m->coef, co.data(), L * sizeof(HcCoef), cudaMemcpyHostToDevice));
   m->have_wmaps = false;
   if (m->encode_tiled && c.dtype == SNLP_DTYPE_BF16 && d % 128 == 0 && ff % 128 == 0 && V % 128 == 0) {
-    auto mk = [&](WMap &w, const void *base, uint64_t K, uint64_t N, uint64_t layers) {
+    // kslice: the K range one decode-regime item reduces over (K, or a K-split slice of it)
+    auto mk = [&](WMap &w, const void *base, uint64_t K, uint64_t N, uint64_t layers, uint64_t kslice) {
       w.BN = N % 256 == 0 ? 256 : 128;
-      return make_tmap_bf16(m->encode_tiled, &w.tm, base, K, N, layers, N * K, w.BN) &&
-             make_tmap_bf16(m->encode_tiled, &w.tm_half, base, K, N, layers, N * K, 128);
+      w.nkb1 = (int)(kslice / kUmmaBK);
+      bool ok = make_tmap_bf16(m->encode_tiled, &w.tm, base, K, N, layers, N * K, w.BN) &&
+                make_tmap_bf16(m->encode_tiled, &w.tm_half, base, K, N, layers, N * K, 128);
+      for (int i = 0; i < 3 && ok; ++i)
+        if (w.nkb1 % (1 << i) == 0) ok = make_tmap_bf16_kb(m->encode_tiled, &w.td128[i], base, K, N, layers, N * K, 128, 1u << i);
+      for (int i = 0; i < 2 && ok; ++i)
+        if (w.BN == 256 && w.nkb1 % (1 << i) == 0) ok = make_tmap_bf16_kb(m->encode_tiled, &w.td256[i], base, K, N, layers, N * K, 256, 1u << i);
+      return ok;
     };
-    m->have_wmaps = mk(m->w_qkv, m->wqkv, d, 3 * d, L) && mk(m->w_o, m->wo, d, d, L) && mk(m->w_up, m->wup, d, ff, L) &&
-                    mk(m->w_dn, m->wdn, ff, d, L) && mk(m->w_lm, m->lm_head, d, V, 1);
+    const uint64_t dn_slice = ff / pick_ksplit(ff, kMaxSplits);
+    m->have_wmaps = mk(m->w_qkv, m->wqkv, d, 3 * d, L, d) && mk(m->w_o, m->wo, d, d, L, d) && mk(m->w_up, m->wup, d, ff, L, d) &&
+                    mk(m->w_dn, m->wdn, ff, d, L, dn_slice) && mk(m->w_lm, m->lm_head, d, V, 1, d);
   }
   m->loaded = true;
   return SNLP_OK;
@@ -674,15 +688,24 @@ struct GemmLaunch {
   bool small, pairs;
 };
 
-// bn_force: 0 = choose the column width; 128 / 256 = use that one (decode regime; the phases of a chained launch share it)
+// k-blocks per bulk-tensor copy of a decode-regime product whose items reduce over nkb1 k-blocks: as many as divide it,
+// up to 64 KB of weights per copy
+static int best_kbox(int bn, int nkb1) {
+  if (bn == 128 && nkb1 % 4 == 0) return 4;
+  return nkb1 % 2 == 0 ? 2 : 1;
+}
+
+// bn_force: 0 = choose the column width; 128 / 256 = use that one (decode regime; the phases of a chained launch share it,
+// and the box depth kbox_force)
 static int umma_prepare(snlp_model *m, GemmLaunch &g, int epi, const __nv_bfloat16 *A, size_t a_ls, const WMap &w, int l0, UmmaParams p, int M, int N,
-                        int K, int ksplit, int nl, int bn_force = 0) {
+                        int K, int ksplit, int nl, int bn_force = 0, int kbox_force = 0) {
   const bool small = M <= kDecodeRows;
   if (epi == UEPI_LMHEAD && !small) return fail(SNLP_ERR_UNSUPPORTED, "LM-head epilogue needs <= %d rows", kDecodeRows);
   if (p.a_share < 1) p.a_share = 1;
   if (p.kfuse < 1) p.kfuse = 1;
-  if (!make_tmap_bf16(m->encode_tiled, &g.ta, A, K, M, (uint64_t)nl * p.kfuse, a_ls ? a_ls : (size_t)M * K, small ? 16 : kUmmaBM))
+  if (!small && !make_tmap_bf16(m->encode_tiled, &g.ta, A, K, M, (uint64_t)nl * p.kfuse, a_ls ? a_ls : (size_t)M * K, kUmmaBM))
     return fail(SNLP_ERR_CUDA, "cuTensorMapEncodeTiled failed (M=%d K=%d)", M, K);
+  p.kbox = 1;
   p.M = M; p.N = N; p.K = K; p.ksplit = ksplit; p.kslice = K / ksplit;
   p.Mt = small ? 1 : (M + kUmmaBM - 1) / kUmmaBM; p.Nt = N / w.BN; p.nl = nl; p.l0 = l0; p.err = m->dev_err;
   g.small = small;
@@ -696,8 +719,17 @@ static int umma_prepare(snlp_model *m, GemmLaunch &g, int epi, const __nv_bfloat
     return SNLP_OK;
   }
   int bn = w.BN;
-  if (small) bn = bn_force ? bn_force : decode_bn(m, w, N, ksplit, nl);
-  g.tmw = bn == w.BN ? &w.tm : &w.tm_half;
+  if (small) {
+    bn = bn_force ? bn_force : decode_bn(m, w, N, ksplit, nl);
+    if (K / ksplit / kUmmaBK != w.nkb1) return fail(SNLP_ERR_UNSUPPORTED, "decode-regime product: K slice %d does not match the weight maps", K / ksplit);
+    p.kbox = kbox_force ? kbox_force : best_kbox(bn, w.nkb1);
+    const int ki = p.kbox == 4 ? 2 : p.kbox == 2 ? 1 : 0;
+    g.tmw = bn == 256 ? &w.td256[ki] : &w.td128[ki];
+    if (!make_tmap_bf16_kb(m->encode_tiled, &g.ta, A, K, M, (uint64_t)nl * p.kfuse, a_ls ? a_ls : (size_t)M * K, 16, p.kbox))
+      return fail(SNLP_ERR_CUDA, "cuTensorMapEncodeTiled failed (M=%d K=%d)", M, K);
+  } else {
+    g.tmw = bn == w.BN ? &w.tm : &w.tm_half;
+  }
   p.Nt = N / bn;
   const int items = p.Mt * p.Nt * ksplit * nl;
   g.bn = bn; g.grid = items < m->n_sm ? items : m->n_sm;
@@ -831,12 +863,15 @@ static int blocks_umma(snlp_model *m, const Fwd &f, int l0, int nl, int fuse) {
     const int b0 = decode_bn(m, m->w_o, d, 1, nl / fuse), b1 = decode_bn(m, m->w_up, ff, 1, nl), b2 = decode_bn(m, m->w_dn, d, sd, nl / fuse);
     const bool all256 = m->w_o.BN == 256 && m->w_up.BN == 256 && m->w_dn.BN == 256;
     const int bn = (all256 && (b0 == 256 || b1 == 256 || b2 == 256)) ? 256 : 128;
+    // ... and a common box depth: the three products share the ring
+    const int kbox = best_kbox(bn, std::gcd(std::gcd(m->w_o.nkb1, m->w_up.nkb1), m->w_dn.nkb1));
     GemmLaunch g[3];
-    TRY(umma_prepare(m, g[0], UEPI_RESID, att, Md, m->w_o, l0, po, M, d, d, 1, nl / fuse, bn));
-    TRY(umma_prepare(m, g[1], UEPI_RELU2_BF16, ub, Md, m->w_up, l0, pu, M, ff, d, 1, nl, bn));
-    TRY(umma_prepare(m, g[2], UEPI_F32, z, (size_t)M * ff, m->w_dn, l0, pd, M, d, ff, sd, nl / fuse, bn));
+    TRY(umma_prepare(m, g[0], UEPI_RESID, att, Md, m->w_o, l0, po, M, d, d, 1, nl / fuse, bn, kbox));
+    TRY(umma_prepare(m, g[1], UEPI_RELU2_BF16, ub, Md, m->w_up, l0, pu, M, ff, d, 1, nl, bn, kbox));
+    TRY(umma_prepare(m, g[2], UEPI_F32, z, (size_t)M * ff, m->w_dn, l0, pd, M, d, ff, sd, nl / fuse, bn, kbox));
     const int epi[3] = {UEPI_RESID, UEPI_RELU2_BF16, UEPI_F32};
     ChainParams cp{};
+    cp.kbox = kbox;
     cp.comb_part = m->attn_part; cp.comb_out = att; cp.comb_o_ls = Md;
     cp.comb_rows = comb ? nl * f.B * H * f.T : 0; cp.comb_nchunk = comb_nchunk; cp.comb_Tq = f.T; cp.comb_BH = f.B * H; cp.comb_H = H; cp.comb_d = d;
     TRY(umma_chain3(m, st, g, epi, cp));

@@ -21,10 +21,11 @@ namespace snlp {
 constexpr int kChainMax = 3;
 
 struct ChainParams {
-  CUtensorMap tmA[kChainMax], tmB[kChainMax];   // per phase: activations {K, M, layers}, box {64, 16, 1}; weights {K, N, L}, box {64, BN, 1}
+  CUtensorMap tmA[kChainMax], tmB[kChainMax];   // per phase: activations {64, M, K / 64, layers}, box {64, 16, kbox, 1}; weights {64, N, K / 64, L}, box {64, BN, kbox, 1}
   UmmaParams p[kChainMax];
   int epi[kChainMax];                           // UEPI_* of the phase
   int nphase;
+  int kbox;                                     // k-blocks per bulk-tensor copy, the same in every phase (the ring is shared)
   unsigned *bar;                                // grid-barrier counter
   // Optional first step: merge the split-KV partials the decode attention left behind (k_attn_decode with merge_here = 0)
   // into the bf16 attention output that phase 0 reads.  comb_rows = layers x sequences x heads x queries (0 = no such step).
@@ -136,29 +137,30 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_chain(const __grid_con
         int pend_from = g;
         int pend_k0[S], pend_la[S];
         const unsigned target = (unsigned)(ph + pre) * (unsigned)G;
+        const int kbox = cp.kbox;   // k-blocks per request (the same in every phase): kbox consecutive ring slots, signalled on the first one's barrier, handed back on the last one's
         auto flush = [&]() {
           asm volatile("fence.proxy.async;" ::: "memory");   // the other CTAs' stores, seen through the barrier, before the bulk copies that read them
-          for (int q = pend_from; q < g; ++q)
-            tma_load_3d(sA + (size_t)(q % S) * Cfg::kABytes, &cp.tmA[ph], &full[q % S], pend_k0[q % S], 0, pend_la[q % S]);
+          for (int q = pend_from; q < g; q += kbox)
+            tma_load_4d(sA + (size_t)(q % S) * Cfg::kABytes, &cp.tmA[ph], &full[q % S], 0, 0, pend_k0[q % S] / kUmmaBK, pend_la[q % S]);
           pend_from = g;
         };
         for (int i = 0; i < my_items && ok; ++i) {
           SNLP_CHAIN_ITEM(i)
-          for (int kb = 0; kb < nkb && ok; ++kb, ++g) {
+          for (int kb = 0; kb < nkb && ok; kb += kbox, g += kbox) {
             if (!open) {
               if (g - pend_from >= S) { ok = chain_wait(cp.bar, target, abort_flag, err); open = ok; if (ok) flush(); }
               else if (ld_acquire_gpu(cp.bar) >= target) { open = true; flush(); }
               if (!ok) break;
             }
             const int s = g % S;
-            ok = mbar_wait(&empty[s], ((g / S) & 1) ^ 1u, abort_flag, err);
+            ok = mbar_wait(&empty[s + kbox - 1], ((g / S) & 1) ^ 1u, abort_flag, err);
             if (!ok) break;
-            mbar_expect_tx(&full[s], Cfg::kABytes + Cfg::kBBytes);
+            mbar_expect_tx(&full[s], (Cfg::kABytes + Cfg::kBBytes) * kbox);
             const int j = kb / nkb1, k0 = ks * p.kslice + (kb % nkb1) * kUmmaBK;   // j: layer inside a K-concatenated chunk
-            tma_load_3d(sB + (size_t)s * Cfg::kBBytes, &cp.tmB[ph], &full[s], k0, n_tile * BN, p.l0 + l + j);
-            if (open) tma_load_3d(sA + (size_t)s * Cfg::kABytes, &cp.tmA[ph], &full[s], k0, 0, la + j);
+            tma_load_4d(sB + (size_t)s * Cfg::kBBytes, &cp.tmB[ph], &full[s], 0, n_tile * BN, k0 / kUmmaBK, p.l0 + l + j);
+            if (open) tma_load_4d(sA + (size_t)s * Cfg::kABytes, &cp.tmA[ph], &full[s], 0, 0, k0 / kUmmaBK, la + j);
             else { pend_k0[s] = k0; pend_la[s] = la + j; }
-            issued = g + 1;
+            issued = g + kbox;
           }
         }
         if (ok && !open && pend_from < g) { ok = chain_wait(cp.bar, target, abort_flag, err); if (ok) flush(); }
@@ -167,7 +169,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_chain(const __grid_con
         // let the copies still in flight land before the CTA's shared memory is handed on (stages whose activation
         // tile was never requested cannot complete: their wait runs into its limit)
         const int first = issued > S ? issued - S : 0;
-        for (int q = first; q < issued; ++q) {
+        for (int q = first; q < issued; q += cp.kbox) {
           const unsigned long long t0 = global_ns();
           while (!mbar_try_wait(&full[q % S], (q / S) & 1) && global_ns() - t0 < kWaitLimitNs / 16) {}
         }
@@ -187,16 +189,18 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_chain(const __grid_con
           if (!ok) break;
           tc_fence_after();
           const uint32_t dcol = tmem_base + b * BN;
-          for (int kb = 0; kb < nkb; ++kb, ++g) {
+          for (int kb = 0; kb < nkb; kb += cp.kbox, g += cp.kbox) {   // one wait and one commit per request
             const int s = g % S;
             ok = mbar_wait(&full[s], (g / S) & 1, abort_flag, err);
             if (!ok) break;
             tc_fence_after();
-            const uint64_t da = umma_desc_sw128(smem_u32(sA + (size_t)s * Cfg::kABytes));
-            const uint64_t db = umma_desc_sw128(smem_u32(sB + (size_t)s * Cfg::kBBytes));
+            uint64_t da = umma_desc_sw128(smem_u32(sA + (size_t)s * Cfg::kABytes));
+            uint64_t db = umma_desc_sw128(smem_u32(sB + (size_t)s * Cfg::kBBytes));
+            for (int q = 0; q < cp.kbox; ++q, da += Cfg::kABytes >> 4, db += Cfg::kBBytes >> 4) {
 #pragma unroll
-            for (int k = 0; k < kUmmaBK / 16; ++k) umma_bf16(dcol, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
-            umma_commit(&empty[s]);
+              for (int k = 0; k < kUmmaBK / 16; ++k) umma_bf16(dcol, da + 2 * k, db + 2 * k, idesc, (kb | q | k) != 0);
+            }
+            umma_commit(&empty[s + cp.kbox - 1]);
           }
           if (ok) umma_commit(&accfull[b]);
         }

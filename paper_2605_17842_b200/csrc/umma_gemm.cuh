@@ -44,6 +44,12 @@ struct UmmaParams {
   // kfuse layers' A rows and weights in turn and accumulates into one output -- the K-concatenated form
   // (attention out-projection, MLP down); outputs and epilogue inputs are indexed by the chunk's first layer.
   int a_share, kfuse;
+  // Decode regime: k-blocks fetched by one bulk-tensor copy (1, 2 or 4; divides kslice / 64 and the ring depth).  One
+  // thread requests the copies and one issues the products; each spends several hundred cycles per ring step whatever
+  // the step's size (~590 per copy request, ~500 per k-block of four products with its barrier wait and commit), which
+  // caps a CTA streaming 128-wide tiles one k-block at a time at ~55 GB/s.  With boxes of several k-blocks there is one
+  // request, one wait and one commit per box.
+  int kbox;
   float *c;                // UEPI_F32 / UEPI_RESID: [ksplit][nl][M][N] fp32
   __nv_bfloat16 *z;        // UEPI_RELU2_BF16: [nl][M][N] bf16;  UEPI_RESID: bf16(u) [nl][M][N]
   size_t out_ls, out_ss;   // layer / split stride of the outputs above (elements)
@@ -117,6 +123,14 @@ __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *tm, ui
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(
           smem_u32(dst)),
       "l"(tm), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *tm, uint64_t *bar, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(
+          smem_u32(dst)),
+      "l"(tm), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
 }
 
@@ -212,7 +226,8 @@ struct UmmaCfg {
   static constexpr int kOuts = AM == 16 ? 16 * (BN + 1) * 4 : 8 * 4096;
   static constexpr int kFixed = kOuts + 1024 /*alignment slack*/ + 512 /*barriers*/;
   static constexpr int kStagesMax = (kUmmaSmemBudget - kFixed) / (kABytes + kBBytes);
-  static constexpr int kStages = kStagesMax > 10 ? 10 : kStagesMax;
+  // decode regime: a whole number of the largest boxes (4 k-blocks at BN = 128, 2 at BN = 256)
+  static constexpr int kStages = AM == 16 ? (BN == 128 ? (kStagesMax / 4) * 4 : (kStagesMax / 2) * 2) : (kStagesMax > 10 ? 10 : kStagesMax);
   static constexpr int kSmem = kStages * (kABytes + kBBytes) + kFixed;
 };
 
@@ -553,18 +568,29 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
       // The weight tiles of the first ring-ful of k-blocks are requested before the dependency wait (under a programmatic
       // dependent launch they stream in while the previous kernel is still finishing); the activation tiles of the same
       // stages follow once that kernel's results are visible.
+      // (decode regime: a request covers kbox consecutive k-blocks = kbox consecutive ring slots; it is signalled on the
+      // first slot's barrier and handed back on the last slot's)
+      const int kbox = AM == 16 ? p.kbox : 1;
+      auto load_a = [&](int s, int k0, int m_tile, int layer) {
+        if (AM == 16) tma_load_4d(sA + (size_t)s * Cfg::kABytes, &tmA, &full[s], 0, 0, k0 / kUmmaBK, layer);
+        else tma_load_3d(sA + (size_t)s * Cfg::kABytes, &tmA, &full[s], k0, m_tile * kUmmaBM, layer);
+      };
+      auto load_b = [&](int s, int k0, int n_tile, int layer) {
+        if (AM == 16) tma_load_4d(sB + (size_t)s * Cfg::kBBytes, &tmB, &full[s], 0, n_tile * BN, k0 / kUmmaBK, layer);
+        else tma_load_3d(sB + (size_t)s * Cfg::kBBytes, &tmB, &full[s], k0, n_tile * BN, layer);
+      };
       const int total_kb = my_items * nkb, npre = total_kb < S ? total_kb : S;
       for (int pass = 0; pass < 2; ++pass) {
         if (pass == 1) pdl_wait();
         for (int i = 0, gp = 0; gp < npre; ++i) {
           SNLP_DECODE_ITEM(i)
-          for (int kb = 0; kb < nkb && gp < npre; ++kb, ++gp) {
+          for (int kb = 0; kb < nkb && gp < npre; kb += kbox, gp += kbox) {
             const int j = kb / nkb1, k0 = ks * p.kslice + (kb % nkb1) * kUmmaBK;
             if (pass == 0) {
-              mbar_expect_tx(&full[gp], Cfg::kABytes + Cfg::kBBytes);   // the stages are empty: first use
-              tma_load_3d(sB + (size_t)gp * Cfg::kBBytes, &tmB, &full[gp], k0, n_tile * BN, p.l0 + l + j);
+              mbar_expect_tx(&full[gp], (Cfg::kABytes + Cfg::kBBytes) * kbox);   // the stages are empty: first use
+              load_b(gp, k0, n_tile, p.l0 + l + j);
             } else {
-              tma_load_3d(sA + (size_t)gp * Cfg::kABytes, &tmA, &full[gp], k0, m_tile * kUmmaBM, la + j);
+              load_a(gp, k0, m_tile, la + j);
             }
           }
         }
@@ -572,16 +598,16 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
       issued = npre;
       for (int i = npre / nkb; i < my_items && ok; ++i) {
         SNLP_DECODE_ITEM(i)
-        for (int kb = (i == npre / nkb ? npre % nkb : 0); kb < nkb; ++kb) {
+        for (int kb = (i == npre / nkb ? npre % nkb : 0); kb < nkb; kb += kbox) {
           g = i * nkb + kb;
           const int s = g % S;
-          ok = mbar_wait(&empty[s], ((g / S) & 1) ^ 1u, abort_flag, p.err);
+          ok = mbar_wait(&empty[s + kbox - 1], ((g / S) & 1) ^ 1u, abort_flag, p.err);
           if (!ok) break;
-          mbar_expect_tx(&full[s], Cfg::kABytes + Cfg::kBBytes);
+          mbar_expect_tx(&full[s], (Cfg::kABytes + Cfg::kBBytes) * kbox);
           const int j = kb / nkb1, k0 = ks * p.kslice + (kb % nkb1) * kUmmaBK;   // j: layer inside a K-concatenated chunk
-          tma_load_3d(sA + (size_t)s * Cfg::kABytes, &tmA, &full[s], k0, m_tile * kUmmaBM, la + j);
-          tma_load_3d(sB + (size_t)s * Cfg::kBBytes, &tmB, &full[s], k0, n_tile * BN, p.l0 + l + j);
-          issued = g + 1;
+          load_a(s, k0, m_tile, la + j);
+          load_b(s, k0, n_tile, p.l0 + l + j);
+          issued = g + kbox;
         }
       }
       // every load of this CTA has been requested: what is left is its tail, so the next kernel of the stream may be
@@ -590,7 +616,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
       if (*abort_flag) {
         // let the copies still in flight land before the CTA's shared memory is handed on
         const int first = issued > S ? issued - S : 0;
-        for (int q = first; q < issued; ++q) {
+        for (int q = first; q < issued; q += kbox) {
           const unsigned long long t0 = global_ns();
           while (!mbar_try_wait(&full[q % S], (q / S) & 1) && global_ns() - t0 < kWaitLimitNs) {}
         }
@@ -607,17 +633,20 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
         if (!ok) break;
         tc_fence_after();
         const uint32_t dcol = tmem_base + b * BN;
-        for (int kb = 0; kb < nkb; ++kb, ++g) {
+        const int kbox = AM == 16 ? p.kbox : 1;
+        for (int kb = 0; kb < nkb; kb += kbox, g += kbox) {   // one wait and one commit per request
           const int s = g % S;
           ok = mbar_wait(&full[s], (g / S) & 1, abort_flag, p.err);
           if (!ok) break;
           tc_fence_after();
-          const uint64_t da = umma_desc_sw128(smem_u32(sA + (size_t)s * Cfg::kABytes));
-          const uint64_t db = umma_desc_sw128(smem_u32(sB + (size_t)s * Cfg::kBBytes));
+          uint64_t da = umma_desc_sw128(smem_u32(sA + (size_t)s * Cfg::kABytes));
+          uint64_t db = umma_desc_sw128(smem_u32(sB + (size_t)s * Cfg::kBBytes));
+          for (int q = 0; q < kbox; ++q, da += Cfg::kABytes >> 4, db += Cfg::kBBytes >> 4) {
 #pragma unroll
-          for (int k = 0; k < kUmmaBK / 16; ++k)  // 16 bf16 = 32 bytes = 2 descriptor address units per step
-            umma_bf16(dcol, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
-          umma_commit(&empty[s]);
+            for (int k = 0; k < kUmmaBK / 16; ++k)  // 16 bf16 = 32 bytes = 2 descriptor address units per step
+              umma_bf16(dcol, da + 2 * k, db + 2 * k, idesc, (kb | q | k) != 0);
+          }
+          umma_commit(&empty[s + kbox - 1]);
         }
         if (ok) umma_commit(&accfull[b]);
       }
@@ -722,6 +751,19 @@ inline bool make_tmap_bf16(EncodeTiledFn fn, CUtensorMap *tm, const void *base, 
   cuuint32_t box[3] = {(cuuint32_t)kUmmaBK, box_rows, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// 4-D bf16 map over the same [layers][rows][K] array with K split into k-blocks: dims {64, rows, K / 64, layers}, box
+// {64, box_rows, kbox, 1}: one copy brings kbox consecutive k-blocks of box_rows rows, each laid out like a {64, box_rows} box
+// of the 3-D map, one after the other.
+inline bool make_tmap_bf16_kb(EncodeTiledFn fn, CUtensorMap *tm, const void *base, uint64_t K, uint64_t rows, uint64_t layers,
+                              uint64_t layer_stride_elems, uint32_t box_rows, uint32_t kbox) {
+  cuuint64_t dims[4] = {(cuuint64_t)kUmmaBK, rows, K / kUmmaBK, layers};
+  cuuint64_t strides[3] = {K * 2, (cuuint64_t)kUmmaBK * 2, layer_stride_elems * 2};
+  cuuint32_t box[4] = {(cuuint32_t)kUmmaBK, box_rows, kbox, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
