@@ -671,9 +671,9 @@ static cudaError_t umma_attr_all() {
 // Column width of a decode-regime launch.  A launch that does not occupy every SM (a sequential step's single layer: 5-20
 // items) lasts as long as one item.  The column tiling does not touch the numbers (every output column is its own dot
 // product), so a launch whose 128-wide items still fit one round over the SMs takes those: twice the CTAs, half the bytes
-// each.  Beyond that the 256-wide tile is the faster one (a 128-wide MMA costs as much as a 256-wide one, which caps a
-// CTA streaming 128-wide tiles at ~50 GB/s).  The out-projection's partial sums of squares are per 128 columns in this
-// regime, whatever the tile width.
+// each.  Beyond that the 256-wide tile is the faster one (the thread that issues the products spends 55-100 cycles per
+// instruction of any width, so 128-wide tiles, 4 KB of weights per instruction, stream at roughly half the rate per CTA).
+// The out-projection's partial sums of squares are per 128 columns in this regime, whatever the tile width.
 static int decode_bn(const snlp_model *m, const WMap &w, int N, int ksplit, int nl) {
   return (w.BN == 256 && (N / 128) * ksplit * nl <= m->n_sm) ? 128 : w.BN;
 }

@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_chain(const __grid_con
   extern __shared__ unsigned char umma_smem_raw[];
   unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)umma_smem_raw + 1023) & ~(uintptr_t)1023);
   constexpr int S = Cfg::kStages;
-  unsigned char *sA = smem;                                   // [S][16 x 128 B]; the A descriptor reads 128 rows from a slot
+  unsigned char *sA = smem;                                   // [S][16 x 128 B]; the A descriptor reads 64 rows from a slot
   unsigned char *sB = smem + (size_t)S * Cfg::kABytes;        // [S][BN x 128 B]
   float *outs = reinterpret_cast<float *>(sB + (size_t)S * Cfg::kBBytes);
   uint64_t *full = reinterpret_cast<uint64_t *>(reinterpret_cast<unsigned char *>(outs) + Cfg::kOuts);
@@ -177,7 +177,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_chain(const __grid_con
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(kUmmaBM, BN);
+      constexpr uint32_t idesc = umma_idesc_bf16(64, BN);
       int g = 0, n = 0;   // stages / items so far, over all phases
       bool ok = true;
       for (int ph = 0; ph < cp.nphase && ok; ++ph) {

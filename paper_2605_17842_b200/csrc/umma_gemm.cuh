@@ -3,15 +3,17 @@
 // Persistent CTAs (one per SM) walk (row tile, column tile, K split, layer) items.  Operand tiles -- AM x 64
 // activations and BN x 64 weights, 128-byte swizzle -- are brought into a shared-memory ring by TMA (one
 // elected thread) that keeps running across item boundaries; a second elected thread issues tcgen05.mma
-// (UMMA 128 x BN x 16, fp32 accumulators in tensor memory, two accumulators so the epilogue of one item
+// (UMMA 128 x BN x 16 -- 64 x BN x 16 in the decode regime --, fp32 accumulators in tensor memory, two accumulators so the epilogue of one item
 // overlaps the main loop of the next) and releases ring slots with tcgen05.commit; four epilogue warps read
 // the accumulator back with tcgen05.ld and apply the fused epilogue.
 //   AM = 128: prefill regime, one accumulator row per epilogue thread.
-//   AM = 16 : decode regime (<= 16 rows).  The weights stay the 256-wide operand -- a tcgen05.mma costs the
-//             same ~155 cycles whatever its shape, so streaming needs 8 KB of weights per instruction -- and
-//             the token box is only 16 rows high (rows 16..127 of the A operand are whatever follows in shared
-//             memory and land in accumulator rows nobody reads).  The kernel is then bound by the weight stream
-//             from HBM; the accumulator is transposed through shared memory so all 128 epilogue threads work.
+//   AM = 16 : decode regime (<= 16 rows).  The weights stay the 256-wide operand: a 64 x 256 x 16 instruction takes the
+//             tensor pipe 128 cycles and covers 8 KB of weights (as many cycles as the 128-row form -- the time goes with
+//             the columns -- but half the multiply-adds, which shows under the board's power cap; a 128-wide one takes
+//             64 cycles for 4 KB, and the issuing thread spends 55-100 cycles per instruction of any shape), and the token
+//             box is only 16 rows high (rows 16..63 of the A operand are whatever follows in shared memory and land in
+//             accumulator rows nobody reads).  The kernel is then bound by the weight stream from HBM; the accumulator is
+//             transposed through shared memory so all 256 epilogue threads work.
 // Every wait on an mbarrier is bounded: on expiry the kernel raises a flag in global memory, lets its
 // copies in flight land, frees its tensor memory and returns.
 #pragma once
@@ -512,7 +514,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
   extern __shared__ unsigned char umma_smem_raw[];
   unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)umma_smem_raw + 1023) & ~(uintptr_t)1023);
   const int S = p.nstages;
-  unsigned char *sA = smem;                                   // [S][AM x 128 B]; the A descriptor reads 128 rows from a slot
+  unsigned char *sA = smem;                                   // [S][AM x 128 B]; the A descriptor reads 128 (decode regime: 64) rows from a slot
   unsigned char *sB = smem + (size_t)S * Cfg::kABytes;        // [S][BN x 128 B]   (>= 14 KB, so those reads stay in bounds)
   float *outs = reinterpret_cast<float *>(sB + (size_t)S * Cfg::kBBytes);
   uint64_t *full = reinterpret_cast<uint64_t *>(reinterpret_cast<unsigned char *>(outs) + Cfg::kOuts);
@@ -624,7 +626,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(kUmmaBM, BN);
+      constexpr uint32_t idesc = umma_idesc_bf16(AM == 16 ? 64 : kUmmaBM, BN);
       int g = 0;
       bool ok = true;
       for (int i = 0; i < my_items && ok; ++i) {
