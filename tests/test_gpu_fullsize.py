@@ -146,3 +146,36 @@ def test_d20_mhc_config_matches_oracle():
     assert trace_err(got.cpu().numpy(), want, TOL["bf16"]) <= TOL["bf16"]
     m.device_status()
     m.close()
+
+
+@pytest.mark.slow
+def test_paper_shaped_model_solver_configurations_match_oracle():
+    """The 32-layer paper-shaped model (L32 d640 H5x128 ff2560) in the solver configurations of the paper's 0.5B
+    inference table (prefix + suffix sweeps, `fwd` initialisation, fused chunks), on the shape itself: a decode-regime
+    call (12 rows) and a prefill-regime call (one ragged 150-row sequence), every layer's state against the oracle."""
+    from paper_2605_17842_b200 import snlp
+    cfg = synth.CONFIGS["paper_0p5b"]
+    W = synth.make_weights(cfg, seed=1234)
+    L = cfg.n_layer
+    for B, T in ((2, 6), (1, 150)):
+        m = make_model(cfg, W, max_rows=B * T, max_batch=B, max_ctx=256)
+        h0 = O.embed(cfg, W, synth.make_ids(cfg, B, T, seed=8)).astype(np.float32)
+        h64 = h0.astype(np.float64)
+        # PxF1: prefix S = L - P, K sweeps (24xF1-h0 K=2, 12xF1-fwd K=2, 8xF1-h0 K=4, 32xF1-h0 K=2)
+        for S, K, init in ((8, 2, O.INIT_H0), (20, 2, O.INIT_FWD), (24, 4, O.INIT_H0), (0, 2, O.INIT_H0)):
+            want, _ = O.forward_snlp(cfg, W, h64, K, O.MODE_IDN, S=S, init=init)
+            got, _ = m.forward_solver(dev(h0), snlp.Solver(K=K, mode=O.MODE_IDN, prefix=S, init=init))
+            err = trace_err(got.cpu().numpy(), want, TOL["bf16"])
+            print(f"paper-shaped B{B}xT{T} S={S} K={K} init={init}: worst layer error {err:.2e}")
+            assert err <= TOL["bf16"], (B, T, S, K, init)
+        # PxF2 / 1xF12: fused chunks behind a prefix (12xF2-h0 K=1, 12xF2-h0 K=2, 1xF12-h0 K=1)
+        for S, F, K in ((8, 2, 1), (8, 2, 2), (20, 12, 1)):
+            want = O.forward_chunked(cfg, W, h64, K, F, S=S)
+            got, _ = m.forward_solver(dev(h0), snlp.Solver(K=K, mode=O.MODE_IDN, prefix=S, fuse=F))
+            err = trace_err(got.cpu().numpy()[S::F], np.stack(want), TOL["bf16"])
+            print(f"paper-shaped B{B}xT{T} S={S} fuse={F} K={K}: worst chunk-boundary error {err:.2e}")
+            assert err <= TOL["bf16"], (B, T, S, F, K)
+        seq = m.forward_sequential(dev(h0)).cpu().numpy()
+        assert trace_err(seq, O.forward_sequential(cfg, W, h64), TOL["bf16"]) <= TOL["bf16"]
+        m.device_status()
+        m.close()
