@@ -131,6 +131,39 @@ def test_decode_step_trace_matches_oracle_mhc():
     m.close()
 
 
+def test_decode_step_with_solver_options_matches_oracle():
+    """KV-cached decode steps through snlp_decode_step_solver: sequential prefix, `fwd` initialisation and fused chunks
+    (the configurations of the paper's inference table) against the oracle on the same cache, several chunks of keys."""
+    from paper_2605_17842_b200 import snlp
+    cfg = synth.ModelConfig(6, 256, 2, 128, 512, 1024, 1, "bf16")
+    W = synth.make_weights(cfg, seed=1234, std=0.05, embed_std=1.0)
+    T = 700
+    ids, m, kv, kv_o = prefilled(cfg, W, 2, T, 2 * 350, seed=6)
+    L = cfg.n_layer
+    worst = 0.0
+    for ctx in (699, 300):
+        tok = ids[:, ctx].copy()
+        h0 = O.embed(cfg, W, tok.reshape(2, 1))
+        cases = [(2, 2, O.INIT_H0, 1), (2, 1, O.INIT_FWD, 1), (0, 1, O.INIT_H0, 2), (2, 2, O.INIT_H0, 2), (0, 1, O.INIT_H0, 3)]
+        for S, K, init, F in cases:
+            kv.truncate(ctx)
+            kv_o.len = ctx
+            m.decode_step_solver(kv, dev(tok), snlp.Solver(K=K, mode=O.MODE_IDN, prefix=S, init=init, fuse=F))
+            got = m.copy_trace(2).cpu().numpy()                           # [L+1, B, n, d]
+            if F == 1:
+                want = O.forward_snlp(cfg, W, h0, K, O.MODE_IDN, kv_o, ctx, S=S, init=init)[0][:, :, 0]
+                err = trace_err(got, want, TOL["bf16"])
+            else:
+                want = np.stack(O.forward_chunked(cfg, W, h0, K, F, kv_o, ctx, S=S, init=init))[:, :, 0]
+                err = trace_err(got[S::F], want, TOL["bf16"])
+            assert err <= TOL["bf16"], (ctx, S, K, init, F, err)
+            assert len(kv) == ctx + 1
+            worst = max(worst, err)
+    print(f"decode step with solver options: worst layer error {worst:.2e}")
+    m.device_status()
+    m.close()
+
+
 def test_async_draft_and_verify_rounds_match_the_synchronous_form():
     """Rounds issued back to back without reading the accepted count: same tokens, same cache length, and the
     host-side bound of the length is only resolved by snlp_kv_len."""
