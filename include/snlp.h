@@ -274,7 +274,7 @@ int snlp_graph_count(const snlp_model *m, int64_t *captured);
  * SNLP_STATIC_LM_HEAD_MAX_D_MODEL (multiple of 32); larger sizes return SNLP_ERR_SHAPE before anything
  * is launched.  Neither this call nor anything it uses calls cudaMalloc/cudaFree.
  * The first call on a device looks up the array's device address and sets two kernel attributes; make
- * that first call outside any stream capture, with the device current.
+ * that first call during set-up, with the device current.
  * All calls on a device share the one array, which keeps whatever the previous call left in it (nothing
  * needs to start at zero: every slot a call reads, it has written first).  Two calls that overlap on the
  * GPU -- different streams without ordering, or two host threads -- race on it: serialise them.
