@@ -340,7 +340,7 @@ def run_ours(args):
                            "between one barrier + synchronize on each side"},
         "clocks": clocks,
         "e2e": {"value": world * 1e3 / ms_e2e, "unit": "tokens/s", "h2d_bytes_per_step": 4, "d2h_bytes_per_step": 4,
-                "steps": e2e_steps, "note": "snlp_decode_step_host every step: host token -> pinned staging, read across the bus by the step's first kernel; next token written back by its last kernel; stream sync"},
+                "steps": e2e_steps, "note": "snlp_decode_step_host every step: host token -> mapped pinned staging, read across the bus by the step's first kernel; next token written back by its last kernel and awaited by the host in that buffer"},
         "gpu_launches": launches_timed,
         "roofline": {"bound": "hbm", "kernel": dom_name,
                      "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak, "peak_source": peak_src,
@@ -350,8 +350,11 @@ def run_ours(args):
                                      "(traffic grows in proportion to the layers covered)" if traffic_full else "no ncu table found",
                      "alg_bytes_per_launch": dom_bytes, "alg_bytes_untrimmed": cls_full[dom], "layers_per_launch": ev,
                      "ms_per_launch": dom_ms,
+                     "sum_of_timed_launches_ms_per_step": sum(v[0] for v in ktimes.values()) / n_prof,
                      "note": "duration = CUDA events recorded by the library around every launch of the class (graphs off), "
-                             "which adds a few microseconds per launch; the whole-step figure under `sweep` has no such overhead"},
+                             "which adds a few microseconds per launch (compare sum_of_timed_launches_ms_per_step with "
+                             "ms_per_step, the same launches replayed as a graph without events; event-record nodes inside "
+                             "the graph were measured to cost the same); the whole-step figure under `sweep` has no such overhead"},
         "sweep": {"alg_bytes_per_step": step_bytes, "alg_bytes_untrimmed": step_bytes_untrimmed, "achieved_GBs": step_gbs,
                   "frac_of_hbm_peak": step_gbs / hbm_peak, "frac_of_nominal": step_gbs / HBM_NOMINAL_GBS, "target_frac": 0.70,
                   "note": "whole decode step (K sweeps + lm head) under CUDA-graph replay; bytes count the layers each sweep "
