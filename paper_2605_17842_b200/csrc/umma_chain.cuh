@@ -56,12 +56,25 @@ __device__ __forceinline__ bool chain_wait(const unsigned *bar, unsigned target,
   }
 }
 
+// pre: the out-projection's inputs, fetched before the accumulator wait (they come from earlier launches); the other
+// epilogues read what the previous phase of this launch wrote and fetch it here, after their phase has opened.
 template <int BN>
-__device__ __forceinline__ void chain_epilogue(int epi, const UmmaParams &p, const float *outs, int ew, int lane, int n_tile, int ks, int l, int ls) {
+__device__ __forceinline__ void chain_epilogue(int epi, const UmmaParams &p, const float *outs, int ew, int lane, int n_tile, int ks, int l, int ls,
+                                               const SmallPre<BN, UEPI_RESID> &pre) {
   switch (epi) {
-    case UEPI_F32: umma_epilogue_small<BN, UEPI_F32>(p, outs, ew, lane, n_tile, ks, l, ls); break;
-    case UEPI_RELU2_BF16: umma_epilogue_small<BN, UEPI_RELU2_BF16>(p, outs, ew, lane, n_tile, ks, l, ls); break;
-    case UEPI_RESID: umma_epilogue_small<BN, UEPI_RESID>(p, outs, ew, lane, n_tile, ks, l, ls); break;
+    case UEPI_F32: {
+      SmallPre<BN, UEPI_F32> q;
+      umma_epilogue_small_pre<BN, UEPI_F32>(p, ew, lane, n_tile, l, ls, q);
+      umma_epilogue_small<BN, UEPI_F32>(p, outs, ew, lane, n_tile, ks, l, ls, q);
+      break;
+    }
+    case UEPI_RELU2_BF16: {
+      SmallPre<BN, UEPI_RELU2_BF16> q;
+      umma_epilogue_small_pre<BN, UEPI_RELU2_BF16>(p, ew, lane, n_tile, l, ls, q);
+      umma_epilogue_small<BN, UEPI_RELU2_BF16>(p, outs, ew, lane, n_tile, ks, l, ls, q);
+      break;
+    }
+    case UEPI_RESID: umma_epilogue_small<BN, UEPI_RESID>(p, outs, ew, lane, n_tile, ks, l, ls, pre); break;
     default: break;
   }
 }
@@ -230,6 +243,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_chain(const __grid_con
       for (int i = 0; i < my_items && alive; ++i, ++n) {
         SNLP_CHAIN_ITEM(i)
         const int b = n & 1;
+        SmallPre<BN, UEPI_RESID> pre;
+        if (cp.epi[ph] == UEPI_RESID) umma_epilogue_small_pre<BN, UEPI_RESID>(p, ew, lane, n_tile, l, la, pre);
         if (!epi_all(mbar_wait(&accfull[b], (n >> 1) & 1, abort_flag, err))) { alive = false; break; }
         tc_fence_after();
         const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * BN;
@@ -247,7 +262,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_chain(const __grid_con
         tc_fence_before();
         epi_bar_sync();
         if (et == 0) mbar_arrive(&accempty[b]);
-        chain_epilogue<BN>(cp.epi[ph], p, outs, ew, lane, n_tile, ks, l, la);
+        chain_epilogue<BN>(cp.epi[ph], p, outs, ew, lane, n_tile, ks, l, la, pre);
         epi_bar_sync();  // outs is reused by the next item
       }
       // This CTA's part of the phase is complete: publish its results and count it in.  A CTA counts itself into phase

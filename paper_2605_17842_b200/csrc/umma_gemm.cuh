@@ -408,17 +408,57 @@ __device__ __forceinline__ void umma_epilogue_rows(const UmmaParams &p, uint32_t
 }
 
 // ---- epilogue of the decode regime: accumulator rows (tokens) already transposed into outs[16][BN+1] ----
+// What an item's epilogue reads from global memory besides its accumulator (a warp serves tokens ew and ew + 8): row
+// scales, the residual-stream values, the rotation-table entries.  Fetched by umma_epilogue_small_pre, which a kernel may
+// call before it waits for the accumulator when those values come from an earlier launch, so that the round trip is
+// over when the products are (the last item's epilogue of a launch or phase is on the critical path).
+template <int BN, int EPI>
+struct SmallPre {
+  float rstd[2];
+  float xv[2][EPI == UEPI_RESID ? BN / 32 : 1];
+  float kappa;
+  float2 c0[2], c1[2];
+  int pos[2];
+};
+
+template <int BN, int EPI>
+__device__ __forceinline__ void umma_epilogue_small_pre(const UmmaParams &p, int ew, int lane, int n_tile, int l, int ls, SmallPre<BN, EPI> &q) {
+#pragma unroll
+  for (int tt = 0; tt < 2; ++tt) {
+    const int tok = ew + 8 * tt;
+    q.rstd[tt] = 1.f;
+    if (tok < p.M) {
+      if ((EPI == UEPI_QKV || EPI == UEPI_RELU2_BF16 || EPI == UEPI_LMHEAD) && p.ssq != nullptr) {
+        float ss = 0.f;
+        for (int i = 0; i < p.nparts; ++i) ss += p.ssq[((size_t)ls * p.nparts + i) * p.M + tok];
+        q.rstd[tt] = rsqrtf(ss / (float)p.K + p.eps);
+      }
+      if (EPI == UEPI_RESID) {
+        const float *xs = p.xm + (size_t)l * p.xm_ls + (size_t)tok * p.N + (size_t)n_tile * BN;
+#pragma unroll
+        for (int j = 0; j < BN / 32; ++j) q.xv[tt][EPI == UEPI_RESID ? j : 0] = xs[lane + 32 * j];
+      }
+      if (EPI == UEPI_QKV) {
+        const int pos = *p.pos_base + (tok % p.T);
+        q.pos[tt] = pos;
+        q.c0[tt] = p.rope[(size_t)pos * 64 + lane];
+        q.c1[tt] = p.rope[(size_t)pos * 64 + lane + 32];
+      }
+    }
+  }
+  if (EPI == UEPI_RESID) q.kappa = p.coef[l].kappa;
+}
+
 // ew = epilogue warp 0..7, lane; one warp per token, lanes across the tile's columns.
 template <int BN, int EPI>
-__device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const float *outs, int ew, int lane, int n_tile, int ks, int l, int ls) {
-  for (int tok = ew; tok < p.M; tok += 8) {
+__device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const float *outs, int ew, int lane, int n_tile, int ks, int l, int ls,
+                                                    const SmallPre<BN, EPI> &q) {
+#pragma unroll
+  for (int tt = 0; tt < 2; ++tt) {
+    const int tok = ew + 8 * tt;
+    if (tok >= p.M) break;
     const float *y = outs + tok * (BN + 1);
-    float rstd = 1.f;
-    if ((EPI == UEPI_QKV || EPI == UEPI_RELU2_BF16 || EPI == UEPI_LMHEAD) && p.ssq != nullptr) {
-      float ss = 0.f;
-      for (int i = 0; i < p.nparts; ++i) ss += p.ssq[((size_t)ls * p.nparts + i) * p.M + tok];
-      rstd = rsqrtf(ss / (float)p.K + p.eps);
-    }
+    const float rstd = q.rstd[tt];
     const size_t n0 = (size_t)n_tile * BN;
     if (EPI == UEPI_F32) {
       float *dst = p.c + (size_t)ks * p.out_ss + (size_t)l * p.out_ls + (size_t)tok * p.N + n0;
@@ -432,15 +472,12 @@ __device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const f
         dst[lane + 32 * j] = __float2bfloat16_rn(v * v);
       }
     } else if (EPI == UEPI_RESID) {
-      const float kappa = p.coef[l].kappa;
-      const float *xs = p.xm + (size_t)l * p.xm_ls + (size_t)tok * p.N + n0;
+      const float kappa = q.kappa;
       float *adst = p.c + (size_t)l * p.out_ls + (size_t)tok * p.N + n0;
       __nv_bfloat16 *udst = p.z + (size_t)l * p.out_ls + (size_t)tok * p.N + n0;
-      // (all the residual-stream values first: loads left between the stores below would be issued one at a time, one
-      // memory round trip each, and this epilogue is on the path between two phases of a chained launch)
-      float xv[BN / 32];
-#pragma unroll
-      for (int j = 0; j < BN / 32; ++j) xv[j] = xs[lane + 32 * j];
+      // (the residual-stream values were all fetched before: loads left between the stores below would be issued one at
+      // a time, one memory round trip each, and this epilogue is on the path between two phases of a chained launch)
+      const float *xv = q.xv[tt];
       // one partial sum of u^2 per 128 columns, so that 128- and 256-wide tiles leave the same numbers behind
 #pragma unroll
       for (int h = 0; h < BN / 128; ++h) {
@@ -448,7 +485,7 @@ __device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const f
 #pragma unroll
         for (int j = 4 * h; j < 4 * h + 4; ++j) {
           const float a = y[lane + 32 * j];
-          const float u = fmaf(kappa, a, xv[j]);
+          const float u = fmaf(kappa, a, xv[EPI == UEPI_RESID ? j : 0]);
           adst[lane + 32 * j] = a;
           udst[lane + 32 * j] = __float2bfloat16_rn(u);
           ss = fmaf(u, u, ss);
@@ -457,10 +494,10 @@ __device__ __forceinline__ void umma_epilogue_small(const UmmaParams &p, const f
         if (lane == 0) p.ssq_out[((size_t)l * p.Nt * (BN / 128) + n_tile * (BN / 128) + h) * p.M + tok] = ss;
       }
     } else if (EPI == UEPI_QKV) {
-      const int b = tok / p.T, pos = *p.pos_base + (tok % p.T);
-      // the rotation table entries of this position, for every head of the tile, before anything is stored (a load
-      // that follows a store is not issued ahead of it: one memory round trip per head otherwise)
-      const float2 c0 = p.rope[(size_t)pos * 64 + lane], c1 = p.rope[(size_t)pos * 64 + lane + 32];
+      const int b = tok / p.T, pos = q.pos[tt];
+      // (the rotation-table entries of this position serve every head of the tile and were fetched before anything is
+      // stored: a load that follows a store is not issued ahead of it)
+      const float2 c0 = q.c0[tt], c1 = q.c1[tt];
 #pragma unroll
       for (int hh = 0; hh < BN / 128; ++hh) {
         const int n = (int)n0 + hh * 128, kind = n / p.d, hcol = n % p.d;
@@ -669,6 +706,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
           for (int c = 0; c < BN / 64; ++c) asm volatile("prefetch.global.L2 [%0];" ::"l"(px + c * 32));
         }
       }
+      SmallPre<BN, EPI> pre;
+      if (AM != kUmmaBM) umma_epilogue_small_pre<BN, EPI>(p, ew, lane, n_tile, l, la, pre);   // every input is an earlier launch's
       if (!epi_all(mbar_wait(&accfull[b], (i >> 1) & 1, abort_flag, p.err))) break;
       tc_fence_after();
       const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * BN;
@@ -693,7 +732,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
         tc_fence_before();
         epi_bar_sync();
         if (et == 0) mbar_arrive(&accempty[b]);
-        umma_epilogue_small<BN, EPI>(p, outs, ew, lane, n_tile, ks, l, la);
+        umma_epilogue_small<BN, EPI>(p, outs, ew, lane, n_tile, ks, l, la, pre);
         epi_bar_sync();  // outs is reused by the next item
       }
     }
