@@ -56,11 +56,12 @@ __device__ __forceinline__ bool chain_wait(const unsigned *bar, unsigned target,
   }
 }
 
-// pre: the out-projection's inputs, fetched before the accumulator wait (they come from earlier launches); the other
-// epilogues read what the previous phase of this launch wrote and fetch it here, after their phase has opened.
+// pre_o / pre_u: the inputs of the out-projection's and the MLP-up epilogue, fetched before the accumulator wait -- the
+// former come from earlier launches, the latter from the previous phase of this launch, so they are fetched once the phase
+// is known to be open.
 template <int BN>
 __device__ __forceinline__ void chain_epilogue(int epi, const UmmaParams &p, const float *outs, int ew, int lane, int n_tile, int ks, int l, int ls,
-                                               const SmallPre<BN, UEPI_RESID> &pre) {
+                                               const SmallPre<BN, UEPI_RESID> &pre_o, const SmallPre<BN, UEPI_RELU2_BF16> &pre_u) {
   switch (epi) {
     case UEPI_F32: {
       SmallPre<BN, UEPI_F32> q;
@@ -68,13 +69,8 @@ __device__ __forceinline__ void chain_epilogue(int epi, const UmmaParams &p, con
       umma_epilogue_small<BN, UEPI_F32>(p, outs, ew, lane, n_tile, ks, l, ls, q);
       break;
     }
-    case UEPI_RELU2_BF16: {
-      SmallPre<BN, UEPI_RELU2_BF16> q;
-      umma_epilogue_small_pre<BN, UEPI_RELU2_BF16>(p, ew, lane, n_tile, l, ls, q);
-      umma_epilogue_small<BN, UEPI_RELU2_BF16>(p, outs, ew, lane, n_tile, ks, l, ls, q);
-      break;
-    }
-    case UEPI_RESID: umma_epilogue_small<BN, UEPI_RESID>(p, outs, ew, lane, n_tile, ks, l, ls, pre); break;
+    case UEPI_RELU2_BF16: umma_epilogue_small<BN, UEPI_RELU2_BF16>(p, outs, ew, lane, n_tile, ks, l, ls, pre_u); break;
+    case UEPI_RESID: umma_epilogue_small<BN, UEPI_RESID>(p, outs, ew, lane, n_tile, ks, l, ls, pre_o); break;
     default: break;
   }
 }
@@ -243,8 +239,18 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_chain(const __grid_con
       for (int i = 0; i < my_items && alive; ++i, ++n) {
         SNLP_CHAIN_ITEM(i)
         const int b = n & 1;
-        SmallPre<BN, UEPI_RESID> pre;
-        if (cp.epi[ph] == UEPI_RESID) umma_epilogue_small_pre<BN, UEPI_RESID>(p, ew, lane, n_tile, l, la, pre);
+        SmallPre<BN, UEPI_RESID> pre_o;
+        SmallPre<BN, UEPI_RELU2_BF16> pre_u;
+        if (cp.epi[ph] == UEPI_RESID) {
+          umma_epilogue_small_pre<BN, UEPI_RESID>(p, ew, lane, n_tile, l, la, pre_o);
+        } else if (cp.epi[ph] == UEPI_RELU2_BF16) {
+          if (i == 0 && ph + pre > 0) {   // the row scales are the previous phase's results: wait until this phase is open
+            bool open_ = true;
+            if (et == 0) open_ = chain_wait(cp.bar, (unsigned)(ph + pre) * (unsigned)G, abort_flag, err);
+            if (!epi_all(open_)) { alive = false; break; }
+          }
+          umma_epilogue_small_pre<BN, UEPI_RELU2_BF16>(p, ew, lane, n_tile, l, la, pre_u);
+        }
         if (!epi_all(mbar_wait(&accfull[b], (n >> 1) & 1, abort_flag, err))) { alive = false; break; }
         tc_fence_after();
         const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * BN;
@@ -262,7 +268,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_chain(const __grid_con
         tc_fence_before();
         epi_bar_sync();
         if (et == 0) mbar_arrive(&accempty[b]);
-        chain_epilogue<BN>(cp.epi[ph], p, outs, ew, lane, n_tile, ks, l, la, pre);
+        chain_epilogue<BN>(cp.epi[ph], p, outs, ew, lane, n_tile, ks, l, la, pre_o, pre_u);
         epi_bar_sync();  // outs is reused by the next item
       }
       // This CTA's part of the phase is complete: publish its results and count it in.  A CTA counts itself into phase
