@@ -567,6 +567,29 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
   const int my_items = (int)blockIdx.x < n_items ? (n_items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
   constexpr uint32_t kTmemCols = 2 * BN;
 
+  // item -> (row tile, column tile, K split, layer); row tiles fastest so that concurrent CTAs share a weight tile
+#define SNLP_DECODE_ITEM(i)                                       \
+  const int it_ = (int)blockIdx.x + (i) * (int)gridDim.x;         \
+  const int m_tile = it_ % p.Mt;                                  \
+  const int n_tile = (it_ / p.Mt) % p.Nt;                         \
+  const int ks = (it_ / (p.Mt * p.Nt)) % p.ksplit;                \
+  const int li_ = it_ / (p.Mt * p.Nt * p.ksplit);                 /* layer (or chunk) of the launch */ \
+  const int la = p.a_share > 1 ? (li_ / p.a_share) * p.a_share : li_ * p.kfuse; /* A rows' layer slot */ \
+  const int l = li_ * p.kfuse;                                    /* output / weight layer slot */
+
+  // (decode regime: a request covers kbox consecutive k-blocks = kbox consecutive ring slots; it is signalled on the
+  // first slot's barrier and handed back on the last slot's)
+  const int kbox = AM == 16 ? p.kbox : 1;
+  auto load_a = [&](int s, int k0, int m_tile, int layer) {
+    if (AM == 16) tma_load_4d(sA + (size_t)s * Cfg::kABytes, &tmA, &full[s], 0, 0, k0 / kUmmaBK, layer);
+    else tma_load_3d(sA + (size_t)s * Cfg::kABytes, &tmA, &full[s], k0, m_tile * kUmmaBM, layer);
+  };
+  auto load_b = [&](int s, int k0, int n_tile, int layer) {
+    if (AM == 16) tma_load_4d(sB + (size_t)s * Cfg::kBBytes, &tmB, &full[s], 0, n_tile * BN, k0 / kUmmaBK, layer);
+    else tma_load_3d(sB + (size_t)s * Cfg::kBBytes, &tmB, &full[s], k0, n_tile * BN, layer);
+  };
+  const int total_kb = my_items * nkb, npre = total_kb < S ? total_kb : S;   // the first ring-ful of k-blocks
+
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(&full[s], 1);
@@ -578,6 +601,19 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // The weight tiles of the first ring-ful of k-blocks depend on nothing -- not on the tensor-memory allocation the
+    // rest of the CTA is waiting for below, not on an earlier kernel of the stream: this thread, which is also the
+    // producer, requests them at once (under a programmatic dependent launch they stream in while the previous kernel
+    // is still finishing).  The activation tiles of the same stages follow behind the dependency wait.
+    for (int i = 0, gp = 0; gp < npre; ++i) {
+      SNLP_DECODE_ITEM(i)
+      (void)m_tile; (void)la;
+      for (int kb = 0; kb < nkb && gp < npre; kb += kbox, gp += kbox) {
+        const int j = kb / nkb1, k0 = ks * p.kslice + (kb % nkb1) * kUmmaBK;
+        mbar_expect_tx(&full[gp], (Cfg::kABytes + Cfg::kBBytes) * kbox);   // the stages are empty: first use
+        load_b(gp, k0, n_tile, p.l0 + l + j);
+      }
+    }
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, kTmemCols);
@@ -587,51 +623,20 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // Everything up to here, and the weight tiles the producer requests first, depend on no earlier kernel of the stream.
+  // Everything up to here, and the weight tiles requested above, depend on no earlier kernel of the stream.
   if (!(warp == 0 && lane == 0)) pdl_wait();
-
-  // item -> (row tile, column tile, K split, layer); row tiles fastest so that concurrent CTAs share a weight tile
-#define SNLP_DECODE_ITEM(i)                                       \
-  const int it_ = (int)blockIdx.x + (i) * (int)gridDim.x;         \
-  const int m_tile = it_ % p.Mt;                                  \
-  const int n_tile = (it_ / p.Mt) % p.Nt;                         \
-  const int ks = (it_ / (p.Mt * p.Nt)) % p.ksplit;                \
-  const int li_ = it_ / (p.Mt * p.Nt * p.ksplit);                 /* layer (or chunk) of the launch */ \
-  const int la = p.a_share > 1 ? (li_ / p.a_share) * p.a_share : li_ * p.kfuse; /* A rows' layer slot */ \
-  const int l = li_ * p.kfuse;                                    /* output / weight layer slot */
 
   if (warp == 0) {
     if (lane == 0) {
       int g = 0, issued = 0;
       bool ok = true;
-      // The weight tiles of the first ring-ful of k-blocks are requested before the dependency wait (under a programmatic
-      // dependent launch they stream in while the previous kernel is still finishing); the activation tiles of the same
-      // stages follow once that kernel's results are visible.
-      // (decode regime: a request covers kbox consecutive k-blocks = kbox consecutive ring slots; it is signalled on the
-      // first slot's barrier and handed back on the last slot's)
-      const int kbox = AM == 16 ? p.kbox : 1;
-      auto load_a = [&](int s, int k0, int m_tile, int layer) {
-        if (AM == 16) tma_load_4d(sA + (size_t)s * Cfg::kABytes, &tmA, &full[s], 0, 0, k0 / kUmmaBK, layer);
-        else tma_load_3d(sA + (size_t)s * Cfg::kABytes, &tmA, &full[s], k0, m_tile * kUmmaBM, layer);
-      };
-      auto load_b = [&](int s, int k0, int n_tile, int layer) {
-        if (AM == 16) tma_load_4d(sB + (size_t)s * Cfg::kBBytes, &tmB, &full[s], 0, n_tile * BN, k0 / kUmmaBK, layer);
-        else tma_load_3d(sB + (size_t)s * Cfg::kBBytes, &tmB, &full[s], k0, n_tile * BN, layer);
-      };
-      const int total_kb = my_items * nkb, npre = total_kb < S ? total_kb : S;
-      for (int pass = 0; pass < 2; ++pass) {
-        if (pass == 1) pdl_wait();
-        for (int i = 0, gp = 0; gp < npre; ++i) {
-          SNLP_DECODE_ITEM(i)
-          for (int kb = 0; kb < nkb && gp < npre; kb += kbox, gp += kbox) {
-            const int j = kb / nkb1, k0 = ks * p.kslice + (kb % nkb1) * kUmmaBK;
-            if (pass == 0) {
-              mbar_expect_tx(&full[gp], (Cfg::kABytes + Cfg::kBBytes) * kbox);   // the stages are empty: first use
-              load_b(gp, k0, n_tile, p.l0 + l + j);
-            } else {
-              load_a(gp, k0, m_tile, la + j);
-            }
-          }
+      pdl_wait();
+      for (int i = 0, gp = 0; gp < npre; ++i) {   // the activation tiles of the stages whose weights are already on their way
+        SNLP_DECODE_ITEM(i)
+        (void)n_tile; (void)l;
+        for (int kb = 0; kb < nkb && gp < npre; kb += kbox, gp += kbox) {
+          const int j = kb / nkb1, k0 = ks * p.kslice + (kb % nkb1) * kUmmaBK;
+          load_a(gp, k0, m_tile, la + j);
         }
       }
       issued = npre;
@@ -672,7 +677,6 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) k_umma_gemm(const __grid_cons
         if (!ok) break;
         tc_fence_after();
         const uint32_t dcol = tmem_base + b * BN;
-        const int kbox = AM == 16 ? p.kbox : 1;
         for (int kb = 0; kb < nkb; kb += kbox, g += kbox) {   // one wait and one commit per request
           const int s = g % S;
           ok = mbar_wait(&full[s], (g / S) & 1, abort_flag, p.err);
